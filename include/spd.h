@@ -1,0 +1,147 @@
+/*
+ * spd.h -- C ABI of the partitioned decode-attention library (libspd.so) for NVIDIA B200 (sm_100a).
+ *
+ * The library computes one decode step of attention split across two KV partitions, as in
+ * Secure Partitioned Decoding: every user's private ("input") partition holds the KV of its
+ * prompt, the public ("output") partition holds the KV of generated tokens.  A partition yields a
+ * partial result per (user, query head): an unnormalised output O, the running maximum m of the
+ * scaled scores and the sum l of exp(score - m).  Two partials merge by log-sum-exp rescaling into
+ * exactly the attention over the concatenated keys (Theorem 1, Eq. 1; stabilised form Sec. 4.2).
+ *
+ * Conventions for every call
+ *   - "device" pointers are CUDA device memory owned by the caller, 16-byte aligned (pools 128-byte
+ *     aligned).  The library allocates and frees no device memory.
+ *   - Calls enqueue work on `cuda_stream` (a cudaStream_t cast to void*, NULL = default stream)
+ *     and return without waiting, except where stated.
+ *   - Host-checkable mistakes (null pointer, unsupported shape, workspace too small) return an error
+ *     code and launch nothing.  Mistakes only the device can see (a page index outside the pool, a
+ *     length larger than the pages listed) never fault: the user concerned gets zeros as output, and
+ *     a sticky flag is raised in the workspace, read by spd_query_device_status().
+ *   - Layouts:  q [batch][num_q_heads][head_dim] in `dtype`;
+ *               pools [num_pages][num_kv_heads][page_size][head_dim] in `dtype`;
+ *               token t of user u lives in page page_indices[page_indptr[u] + t / page_size],
+ *               slot t % page_size; slots at or beyond seq_lens[u] are never used in a result.
+ *   - Query head h reads KV head h / (num_q_heads / num_kv_heads).
+ *   - m and l are in natural-log units of the scaled score, so a partial can be handed from one
+ *     call (or process) to another as is.  An empty partition gives O = 0, m = -inf, l = 0.
+ *   - Supported: head_dim 64 or 128, page_size 16, dtype F32 or BF16 (q and KV alike),
+ *     num_q_heads a multiple of num_kv_heads with a group size of 1, 2, 4, 8 or a multiple of 8.
+ */
+#ifndef SPD_H_
+#define SPD_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+    SPD_OK = 0,
+    SPD_ERR_INVALID_ARG = 1,   /* null pointer, negative size, misaligned pointer            */
+    SPD_ERR_UNSUPPORTED = 2,   /* shape or dtype outside the supported set                     */
+    SPD_ERR_WORKSPACE = 3,     /* workspace smaller than spd_workspace_size() reports          */
+    SPD_ERR_BAD_PAGE = 4,      /* device saw a page index or length out of range (sticky flag) */
+    SPD_ERR_CUDA = 5,          /* a CUDA runtime or driver call failed                         */
+    SPD_ERR_TIMEOUT = 6        /* a bounded wait inside a kernel ran out (sticky flag)         */
+} spd_status;
+
+typedef enum { SPD_F32 = 0, SPD_BF16 = 1 } spd_dtype;
+
+typedef struct {
+    int32_t   batch;          /* users in the batch (one query token each) */
+    int32_t   num_q_heads;
+    int32_t   num_kv_heads;
+    int32_t   head_dim;       /* 64 or 128 */
+    int32_t   page_size;      /* 16 */
+    spd_dtype dtype;          /* of q and of both pools */
+    float     sm_scale;       /* multiplies q.k before the softmax (the paper's Eq. 1 has scale 1) */
+} spd_shape;
+
+/* One KV partition.  All pointers are device memory. */
+typedef struct {
+    const void    *k_pool;        /* [num_pages][num_kv_heads][page_size][head_dim] */
+    const void    *v_pool;
+    int32_t        num_pages;
+    const int32_t *page_indptr;   /* [batch+1], page_indptr[0] = 0, non-decreasing                  */
+    const int32_t *page_indices;  /* [page_indptr[batch]], each in [0, num_pages)                   */
+    const int32_t *seq_lens;      /* [batch], 0 <= len <= page_size * (pages listed for the user)   */
+} spd_paged_kv;
+
+/* A partial attention result (device memory, fp32): the message between the two halves. */
+typedef struct {
+    float *o;   /* [batch][num_q_heads][head_dim], unnormalised */
+    float *m;   /* [batch][num_q_heads] */
+    float *l;   /* [batch][num_q_heads] */
+} spd_partial;
+
+/*
+ * Bytes of device workspace the calls below need for `shape` on the current device.
+ * The workspace holds the per-call plan, split-K scratch and the sticky status words; zero it
+ * once (cudaMemset) before first use.  One workspace serves one stream at a time.
+ */
+spd_status spd_workspace_size(const spd_shape *shape, size_t *bytes);
+
+/*
+ * Private partial attention (protocol step 3b; Fig. 3 step 4; Sec. 4.2): for every user and
+ * query head, (O, m, l) over the user's private partition.  Long partitions are split across
+ * warps and recombined by a second-level log-sum-exp merge.  `out` is fully overwritten.
+ */
+spd_status spd_partial_attn(const spd_shape *shape, const void *q, const spd_paged_kv *priv,
+                            spd_partial out, void *ws, size_t ws_bytes, void *cuda_stream);
+
+/*
+ * Public partial attention batched over users, fused with the merge (protocol step 3c; Fig. 3
+ * steps 3 and 5; Theorem 1): computes the partial over the public partition, merges it with `in`
+ * (the private partial) and writes the normalised attention output
+ *   out [batch][num_q_heads][head_dim] in `out_dtype` (F32 or BF16).
+ * A user whose two partitions are both empty gets zeros.
+ */
+spd_status spd_service_attn_merge(const spd_shape *shape, const void *q, const spd_paged_kv *pub,
+                                  spd_partial in, void *out, spd_dtype out_dtype,
+                                  void *ws, size_t ws_bytes, void *cuda_stream);
+
+/*
+ * One whole decode step of attention for one layer (protocol step 3, b and c): the private
+ * partial, the public partial and their merge.  `fused` = 0 chains spd_partial_attn and
+ * spd_service_attn_merge through a partial held in the workspace; `fused` != 0 streams both
+ * partitions of a user through one running log-sum-exp (the same merge algebra applied tile by
+ * tile), which saves the round trip of the partial.  Same result up to fp32 rounding order.
+ */
+spd_status spd_decode_step(const spd_shape *shape, const void *q, const spd_paged_kv *priv,
+                           const spd_paged_kv *pub, void *out, spd_dtype out_dtype, int32_t fused,
+                           void *ws, size_t ws_bytes, void *cuda_stream);
+
+/*
+ * spd_decode_step for a caller whose per-step data lives in HOST memory: q, both partitions'
+ * page_indptr / page_indices / seq_lens and `out` are host pointers (pinned memory makes the
+ * copies asynchronous); only k_pool / v_pool inside `priv` and `pub` are device pointers (the KV
+ * cache stays resident).  The call copies the host inputs into `staging` (device memory of at
+ * least spd_host_staging_size() bytes), runs the fused step, copies `out` back and waits for
+ * the stream.  Returns the device status as spd_query_device_status() would.
+ */
+spd_status spd_host_staging_size(const spd_shape *shape, int64_t priv_pages_listed,
+                                 int64_t pub_pages_listed, spd_dtype out_dtype, size_t *bytes);
+spd_status spd_decode_step_host(const spd_shape *shape, const void *q_host, const spd_paged_kv *priv,
+                                const spd_paged_kv *pub, void *out_host, spd_dtype out_dtype,
+                                void *staging, size_t staging_bytes,
+                                void *ws, size_t ws_bytes, void *cuda_stream);
+
+/*
+ * Waits for `cuda_stream`, then reads and clears the workspace's sticky status.  Returns SPD_OK,
+ * SPD_ERR_BAD_PAGE or SPD_ERR_TIMEOUT; *first_bad_user (may be NULL) receives the lowest user
+ * index that was flagged, or -1.
+ */
+spd_status spd_query_device_status(void *ws, void *cuda_stream, int32_t *first_bad_user);
+
+/* Number of kernels the library has launched in this process (for accounting in benchmarks). */
+int64_t spd_kernel_launch_count(void);
+
+/* Static text for a status code. */
+const char *spd_status_string(spd_status status);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* SPD_H_ */

@@ -1,0 +1,185 @@
+"""Thin ctypes binding over libspd.so: same names as the C ABI, argument marshalling only.
+
+PyTorch supplies device memory and streams; every step of the path runs in the library's
+kernels.  There is no fallback: if the library is missing, loading raises.
+"""
+from __future__ import annotations
+
+import ctypes as C
+import os
+from typing import Optional, Tuple
+
+import torch
+
+from .build import LIB_PATH
+
+SPD_OK = 0
+SPD_F32, SPD_BF16 = 0, 1
+_STATUS_NAMES = {0: "SPD_OK", 1: "SPD_ERR_INVALID_ARG", 2: "SPD_ERR_UNSUPPORTED", 3: "SPD_ERR_WORKSPACE",
+                 4: "SPD_ERR_BAD_PAGE", 5: "SPD_ERR_CUDA", 6: "SPD_ERR_TIMEOUT"}
+
+EXPORTS = ["spd_workspace_size", "spd_partial_attn", "spd_service_attn_merge", "spd_decode_step",
+           "spd_host_staging_size", "spd_decode_step_host", "spd_query_device_status",
+           "spd_kernel_launch_count", "spd_status_string"]
+
+
+class SpdError(RuntimeError):
+    def __init__(self, code: int, where: str):
+        self.code = code
+        super().__init__(f"{where}: {_STATUS_NAMES.get(code, code)} ({status_string(code)})")
+
+
+class Shape(C.Structure):
+    _fields_ = [("batch", C.c_int32), ("num_q_heads", C.c_int32), ("num_kv_heads", C.c_int32),
+                ("head_dim", C.c_int32), ("page_size", C.c_int32), ("dtype", C.c_int32), ("sm_scale", C.c_float)]
+
+
+class PagedKV(C.Structure):
+    _fields_ = [("k_pool", C.c_void_p), ("v_pool", C.c_void_p), ("num_pages", C.c_int32),
+                ("page_indptr", C.c_void_p), ("page_indices", C.c_void_p), ("seq_lens", C.c_void_p)]
+
+
+class Partial(C.Structure):
+    _fields_ = [("o", C.c_void_p), ("m", C.c_void_p), ("l", C.c_void_p)]
+
+
+_lib = None
+
+
+def lib() -> C.CDLL:
+    """Load libspd.so (built in-tree by build.py).  Raises if it is missing."""
+    global _lib
+    if _lib is None:
+        if not os.path.exists(LIB_PATH):
+            raise FileNotFoundError(f"{LIB_PATH} not built: run `python -m paper_2409_19134_b200.build`")
+        L = C.CDLL(LIB_PATH)
+        vp, sz = C.c_void_p, C.c_size_t
+        L.spd_workspace_size.argtypes = [C.POINTER(Shape), C.POINTER(sz)]
+        L.spd_partial_attn.argtypes = [C.POINTER(Shape), vp, C.POINTER(PagedKV), Partial, vp, sz, vp]
+        L.spd_service_attn_merge.argtypes = [C.POINTER(Shape), vp, C.POINTER(PagedKV), Partial, vp, C.c_int, vp, sz, vp]
+        L.spd_decode_step.argtypes = [C.POINTER(Shape), vp, C.POINTER(PagedKV), C.POINTER(PagedKV), vp, C.c_int,
+                                      C.c_int32, vp, sz, vp]
+        L.spd_host_staging_size.argtypes = [C.POINTER(Shape), C.c_int64, C.c_int64, C.c_int, C.POINTER(sz)]
+        L.spd_decode_step_host.argtypes = [C.POINTER(Shape), vp, C.POINTER(PagedKV), C.POINTER(PagedKV), vp, C.c_int,
+                                           vp, sz, vp, sz, vp]
+        L.spd_query_device_status.argtypes = [vp, vp, C.POINTER(C.c_int32)]
+        L.spd_kernel_launch_count.restype = C.c_int64
+        L.spd_status_string.restype = C.c_char_p
+        L.spd_status_string.argtypes = [C.c_int]
+        for name in EXPORTS[:7]:
+            getattr(L, name).restype = C.c_int
+        _lib = L
+    return _lib
+
+
+def status_string(code: int) -> str:
+    return lib().spd_status_string(int(code)).decode()
+
+
+def _check(code: int, where: str) -> None:
+    if code != SPD_OK:
+        raise SpdError(code, where)
+
+
+def _dtype_code(dt: torch.dtype) -> int:
+    if dt == torch.float32:
+        return SPD_F32
+    if dt == torch.bfloat16:
+        return SPD_BF16
+    raise TypeError(f"unsupported dtype {dt}")
+
+
+def make_shape(batch, num_q_heads, num_kv_heads, head_dim, dtype, sm_scale, page_size=16) -> Shape:
+    return Shape(batch, num_q_heads, num_kv_heads, head_dim, page_size, _dtype_code(dtype), float(sm_scale))
+
+
+def _ptr(t: Optional[torch.Tensor]) -> Optional[int]:
+    return None if t is None or t.numel() == 0 else t.data_ptr()
+
+
+def paged_kv(part) -> PagedKV:
+    """Marshal an object with k_pool, v_pool, page_indptr, page_indices, seq_lens tensors."""
+    for t in (part.k_pool, part.v_pool, part.page_indptr, part.page_indices, part.seq_lens):
+        assert t.is_contiguous()
+    assert part.page_indptr.dtype == torch.int32 and part.page_indices.dtype == torch.int32
+    assert part.seq_lens.dtype == torch.int32
+    return PagedKV(_ptr(part.k_pool), _ptr(part.v_pool), int(part.k_pool.shape[0]),
+                   part.page_indptr.data_ptr(), _ptr(part.page_indices), part.seq_lens.data_ptr())
+
+
+def _stream_ptr(stream: Optional[torch.cuda.Stream]) -> int:
+    s = stream if stream is not None else torch.cuda.current_stream()
+    return s.cuda_stream
+
+
+def spd_workspace_size(shape: Shape) -> int:
+    n = C.c_size_t(0)
+    _check(lib().spd_workspace_size(C.byref(shape), C.byref(n)), "spd_workspace_size")
+    return int(n.value)
+
+
+def alloc_workspace(shape: Shape, device="cuda") -> torch.Tensor:
+    """A zeroed workspace tensor of the size the library asks for."""
+    return torch.zeros(spd_workspace_size(shape), dtype=torch.uint8, device=device)
+
+
+def alloc_partial(shape: Shape, device="cuda") -> Tuple[torch.Tensor, torch.Tensor, torch.Tensor]:
+    B, H, D = shape.batch, shape.num_q_heads, shape.head_dim
+    return (torch.empty((B, H, D), dtype=torch.float32, device=device),
+            torch.empty((B, H), dtype=torch.float32, device=device),
+            torch.empty((B, H), dtype=torch.float32, device=device))
+
+
+def spd_partial_attn(shape, q, priv, out, ws, stream=None) -> None:
+    kv = paged_kv(priv)
+    part = Partial(out[0].data_ptr(), out[1].data_ptr(), out[2].data_ptr())
+    _check(lib().spd_partial_attn(C.byref(shape), q.data_ptr(), C.byref(kv), part, ws.data_ptr(), ws.numel(),
+                                  _stream_ptr(stream)), "spd_partial_attn")
+
+
+def spd_service_attn_merge(shape, q, pub, partial_in, out, ws, stream=None) -> None:
+    kv = paged_kv(pub)
+    part = Partial(partial_in[0].data_ptr(), partial_in[1].data_ptr(), partial_in[2].data_ptr())
+    _check(lib().spd_service_attn_merge(C.byref(shape), q.data_ptr(), C.byref(kv), part, out.data_ptr(),
+                                        _dtype_code(out.dtype), ws.data_ptr(), ws.numel(), _stream_ptr(stream)),
+           "spd_service_attn_merge")
+
+
+def spd_decode_step(shape, q, priv, pub, out, ws, fused=True, stream=None) -> None:
+    a, b = paged_kv(priv), paged_kv(pub)
+    _check(lib().spd_decode_step(C.byref(shape), q.data_ptr(), C.byref(a), C.byref(b), out.data_ptr(),
+                                 _dtype_code(out.dtype), 1 if fused else 0, ws.data_ptr(), ws.numel(),
+                                 _stream_ptr(stream)), "spd_decode_step")
+
+
+def spd_host_staging_size(shape, priv_pages_listed: int, pub_pages_listed: int, out_dtype) -> int:
+    n = C.c_size_t(0)
+    _check(lib().spd_host_staging_size(C.byref(shape), priv_pages_listed, pub_pages_listed,
+                                       _dtype_code(out_dtype), C.byref(n)), "spd_host_staging_size")
+    return int(n.value)
+
+
+def spd_decode_step_host(shape, q_host, priv_pools, priv_tables, pub_pools, pub_tables, out_host, staging, ws,
+                         stream=None) -> None:
+    """q_host / *_tables (indptr, indices, lens) / out_host are HOST tensors (pinned for async copies);
+    *_pools are (k_pool, v_pool) device tensors."""
+    def kv(pools, tables):
+        indptr, indices, lens = tables
+        return PagedKV(_ptr(pools[0]), _ptr(pools[1]), int(pools[0].shape[0]), indptr.data_ptr(),
+                       _ptr(indices), lens.data_ptr())
+    a, b = kv(priv_pools, priv_tables), kv(pub_pools, pub_tables)
+    _check(lib().spd_decode_step_host(C.byref(shape), q_host.data_ptr(), C.byref(a), C.byref(b),
+                                      out_host.data_ptr(), _dtype_code(out_host.dtype), staging.data_ptr(),
+                                      staging.numel(), ws.data_ptr(), ws.numel(), _stream_ptr(stream)),
+           "spd_decode_step_host")
+
+
+def spd_query_device_status(ws, stream=None) -> Tuple[int, int]:
+    """Waits for the stream; returns (status code, first flagged user or -1) and clears the flag."""
+    bad = C.c_int32(-1)
+    code = lib().spd_query_device_status(ws.data_ptr(), _stream_ptr(stream), C.byref(bad))
+    return int(code), int(bad.value)
+
+
+def spd_kernel_launch_count() -> int:
+    return int(lib().spd_kernel_launch_count())

@@ -1,0 +1,35 @@
+"""Builds libspd.so in-tree with nvcc for sm_100a (cross-compiles without a GPU)."""
+from __future__ import annotations
+
+import os
+import subprocess
+import sys
+
+_PKG = os.path.dirname(os.path.abspath(__file__))
+_ROOT = os.path.dirname(_PKG)
+LIB_PATH = os.path.join(_PKG, "libspd.so")
+SOURCES = [os.path.join(_PKG, "csrc", "spd_api.cu")]
+HEADERS = [os.path.join(_PKG, "csrc", "spd_kernels.cuh"), os.path.join(_PKG, "csrc", "spd_device.cuh"),
+           os.path.join(_ROOT, "include", "spd.h")]
+
+
+def nvcc_command(verbose: bool = False):
+    nvcc = os.environ.get("NVCC", "/usr/local/cuda/bin/nvcc")
+    cmd = [nvcc, "-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
+           "-shared", "-Xcompiler", "-fPIC", "-I", os.path.join(_ROOT, "include"), "-o", LIB_PATH] + SOURCES
+    if verbose:
+        cmd[1:1] = ["-Xptxas", "-v"]
+    return cmd
+
+
+def build(force: bool = False, verbose: bool = False) -> str:
+    deps = SOURCES + HEADERS
+    if (not force and os.path.exists(LIB_PATH)
+            and all(os.path.getmtime(LIB_PATH) >= os.path.getmtime(d) for d in deps)):
+        return LIB_PATH
+    subprocess.check_call(nvcc_command(verbose))
+    return LIB_PATH
+
+
+if __name__ == "__main__":
+    print(build(force="--force" in sys.argv, verbose="-v" in sys.argv))

@@ -1,0 +1,410 @@
+// Host side of libspd.so: argument checks, workspace layout, TMA descriptors, kernel launches.
+// The C ABI is declared in include/spd.h.
+#include "spd.h"
+
+#include <atomic>
+#include <cstdio>
+#include <cstring>
+#include <mutex>
+
+#include "spd_kernels.cuh"
+
+namespace {
+
+using namespace spd;
+
+std::atomic<int64_t> g_launches{0};
+
+struct DeviceInfo {
+    int sms = 0;
+    bool ok = false;
+};
+
+// Per-device facts, looked up once.
+spd_status device_info(DeviceInfo *out) {
+    static std::mutex mu;
+    static DeviceInfo cache[64];
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return SPD_ERR_CUDA;
+    std::lock_guard<std::mutex> lock(mu);
+    if (!cache[dev].ok) {
+        int sms = 0, major = 0;
+        if (cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess) return SPD_ERR_CUDA;
+        if (cudaDeviceGetAttribute(&major, cudaDevAttrComputeCapabilityMajor, dev) != cudaSuccess) return SPD_ERR_CUDA;
+        if (major != 10) return SPD_ERR_UNSUPPORTED;   // built for sm_100a only
+        cache[dev].sms = sms;
+        cache[dev].ok = true;
+    }
+    *out = cache[dev];
+    return SPD_OK;
+}
+
+typedef CUresult (*EncodeTiledFn)(CUtensorMap *, CUtensorMapDataType, cuuint32_t, void *, const cuuint64_t *,
+                                  const cuuint64_t *, const cuuint32_t *, const cuuint32_t *, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+EncodeTiledFn encode_fn() {
+    static EncodeTiledFn fn = nullptr;
+    static std::once_flag once;
+    std::call_once(once, [] {
+        void *ptr = nullptr;
+        cudaDriverEntryPointQueryResult q;
+        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &ptr, cudaEnableDefault, &q) == cudaSuccess &&
+            q == cudaDriverEntryPointSuccess)
+            fn = reinterpret_cast<EncodeTiledFn>(ptr);
+    });
+    return fn;
+}
+
+constexpr size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
+
+// Workspace layout.  The header and the bad-user array come first so that the status query can
+// find them without knowing the shape.
+struct WsLayout {
+    size_t hdr, bad, pfx, np0, np1, scratch, partial_o, partial_m, partial_l, total;
+};
+
+WsLayout ws_layout(const spd_shape &s, int sms) {
+    WsLayout L;
+    size_t off = 0;
+    const size_t B = s.batch;
+    L.hdr = off;       off = align_up(off + HDR_WORDS * 4, 256);
+    L.bad = off;       off = align_up(off + B * 4, 256);
+    L.pfx = off;       off = align_up(off + (B + 1) * 4, 256);
+    L.np0 = off;       off = align_up(off + B * 4, 256);
+    L.np1 = off;       off = align_up(off + B * 4, 256);
+    const size_t max_warps = static_cast<size_t>(sms) * 8;
+    L.scratch = off;   off = align_up(off + 2 * max_warps * slot_floats(s.head_dim) * 4, 256);
+    const size_t rows = B * s.num_q_heads;
+    L.partial_o = off; off = align_up(off + rows * s.head_dim * 4, 256);
+    L.partial_m = off; off = align_up(off + rows * 4, 256);
+    L.partial_l = off; off = align_up(off + rows * 4, 256);
+    L.total = off;
+    return L;
+}
+
+spd_status check_shape(const spd_shape *s) {
+    if (!s) return SPD_ERR_INVALID_ARG;
+    if (s->batch <= 0 || s->num_q_heads <= 0 || s->num_kv_heads <= 0) return SPD_ERR_INVALID_ARG;
+    if (s->head_dim != 64 && s->head_dim != 128) return SPD_ERR_UNSUPPORTED;
+    if (s->page_size != kPage) return SPD_ERR_UNSUPPORTED;
+    if (s->dtype != SPD_F32 && s->dtype != SPD_BF16) return SPD_ERR_UNSUPPORTED;
+    if (s->num_q_heads % s->num_kv_heads != 0) return SPD_ERR_UNSUPPORTED;
+    const int g = s->num_q_heads / s->num_kv_heads;
+    if (!(g == 1 || g == 2 || g == 4 || g % 8 == 0)) return SPD_ERR_UNSUPPORTED;
+    if (!(s->sm_scale == s->sm_scale)) return SPD_ERR_INVALID_ARG;
+    return SPD_OK;
+}
+
+bool misaligned(const void *p, size_t a) { return (reinterpret_cast<uintptr_t>(p) & (a - 1)) != 0; }
+
+spd_status check_kv(const spd_shape *s, const spd_paged_kv *kv) {
+    if (!kv) return SPD_ERR_INVALID_ARG;
+    if (kv->num_pages < 0) return SPD_ERR_INVALID_ARG;
+    if (!kv->page_indptr || !kv->seq_lens) return SPD_ERR_INVALID_ARG;
+    if (kv->num_pages > 0 && (!kv->k_pool || !kv->v_pool || !kv->page_indices)) return SPD_ERR_INVALID_ARG;
+    if (misaligned(kv->k_pool, 128) || misaligned(kv->v_pool, 128)) return SPD_ERR_INVALID_ARG;
+    // TMA row coordinates are 32-bit
+    if (static_cast<int64_t>(kv->num_pages) * s->num_kv_heads * kPage >= (1ll << 31)) return SPD_ERR_UNSUPPORTED;
+    return SPD_OK;
+}
+
+spd_status make_map(CUtensorMap *map, const spd_shape &s, const void *pool, int64_t num_pages) {
+    EncodeTiledFn fn = encode_fn();
+    if (!fn) return SPD_ERR_CUDA;
+    const bool bf = s.dtype == SPD_BF16;
+    const cuuint64_t es = bf ? 2 : 4;
+    cuuint64_t dims[2] = {static_cast<cuuint64_t>(s.head_dim),
+                          static_cast<cuuint64_t>(num_pages) * s.num_kv_heads * kPage};
+    cuuint64_t strides[1] = {static_cast<cuuint64_t>(s.head_dim) * es};
+    cuuint32_t box[2] = {static_cast<cuuint32_t>(bf ? 64 : s.head_dim), static_cast<cuuint32_t>(kPage)};
+    cuuint32_t estr[2] = {1, 1};
+    CUresult r = fn(map, bf ? CU_TENSOR_MAP_DATA_TYPE_BFLOAT16 : CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 2,
+                    const_cast<void *>(pool), dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
+                    bf ? CU_TENSOR_MAP_SWIZZLE_128B : CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                    CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    return r == CUDA_SUCCESS ? SPD_OK : SPD_ERR_CUDA;
+}
+
+template <class Math>
+constexpr size_t attn_smem_bytes() {
+    return 1024 + static_cast<size_t>(Math::kWarps) * Math::kStages * (2 * Math::kTileBytes + 8 + 16) +
+           static_cast<size_t>(Math::kWarps) * Math::kExtraBytes;
+}
+
+template <class Math>
+spd_status launch_attn(const Params &p, const CUtensorMap *maps, int sms, cudaStream_t st) {
+    constexpr size_t smem = attn_smem_bytes<Math>();
+    static std::once_flag once[64];
+    int dev = 0;
+    cudaGetDevice(&dev);
+    cudaError_t attr_err = cudaSuccess;
+    std::call_once(once[dev & 63], [&] {
+        attr_err = cudaFuncSetAttribute(attn_kernel<Math>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                        static_cast<int>(smem));
+    });
+    if (attr_err != cudaSuccess) return SPD_ERR_CUDA;
+    attn_kernel<Math><<<sms, Math::kWarps * 32, smem, st>>>(p, maps[0], maps[1], maps[2], maps[3]);
+    ++g_launches;
+    return cudaGetLastError() == cudaSuccess ? SPD_OK : SPD_ERR_CUDA;
+}
+
+template <class Math>
+int warps_of() { return Math::kWarps; }
+
+// What one library call boils down to: plan -> attention -> second-level merge.
+struct Job {
+    const spd_shape *shape;
+    const void *q;
+    const spd_paged_kv *part[2];   // private, public; either may be null (absent)
+    int mode;
+    spd_partial pout;              // OUT_PARTIAL
+    const spd_partial *pin;        // OUT_FINAL, optional
+    void *out;
+    spd_dtype out_dtype;
+};
+
+spd_status run_job(const Job &job, void *ws, size_t ws_bytes, void *stream) {
+    const spd_shape &s = *job.shape;
+    DeviceInfo di;
+    spd_status rc = device_info(&di);
+    if (rc != SPD_OK) return rc;
+    const WsLayout L = ws_layout(s, di.sms);
+    if (!ws || misaligned(ws, 256)) return SPD_ERR_INVALID_ARG;
+    if (ws_bytes < L.total) return SPD_ERR_WORKSPACE;
+    if (!job.q || misaligned(job.q, 16)) return SPD_ERR_INVALID_ARG;
+    uint8_t *w = static_cast<uint8_t *>(ws);
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+
+    Params p;
+    memset(&p, 0, sizeof p);
+    p.B = s.batch; p.Hq = s.num_q_heads; p.Hkv = s.num_kv_heads; p.g = p.Hq / p.Hkv;
+    p.hgroups = p.g > kHeadsPerItem ? p.g / kHeadsPerItem : 1;
+    p.geff = p.g > kHeadsPerItem ? kHeadsPerItem : p.g;
+    p.S = p.Hkv * p.hgroups;
+    p.sm_scale = s.sm_scale;
+    p.q = job.q;
+    const bool bf = s.dtype == SPD_BF16;
+    const int warps_per_cta = bf ? MathBF16<128>::kWarps : MathF32<128, 1>::kWarps;
+    p.num_warps = di.sms * warps_per_cta;
+    p.hdr = reinterpret_cast<int32_t *>(w + L.hdr);
+    p.bad = reinterpret_cast<int32_t *>(w + L.bad);
+    p.pfx = reinterpret_cast<int32_t *>(w + L.pfx);
+    p.np0 = reinterpret_cast<int32_t *>(w + L.np0);
+    p.np1 = reinterpret_cast<int32_t *>(w + L.np1);
+    p.scratch = reinterpret_cast<float *>(w + L.scratch);
+    p.mode = job.mode;
+    p.po = job.pout.o; p.pm = job.pout.m; p.pl = job.pout.l;
+    if (job.pin) { p.in_o = job.pin->o; p.in_m = job.pin->m; p.in_l = job.pin->l; }
+    p.out = job.out;
+    p.out_bf16 = job.out_dtype == SPD_BF16;
+
+    CUtensorMap maps[4];
+    int have = -1;
+    for (int i = 0; i < 2; ++i) {
+        const spd_paged_kv *kv = job.part[i];
+        if (!kv) continue;
+        p.part[i].indptr = kv->page_indptr;
+        p.part[i].indices = kv->page_indices;
+        p.part[i].lens = kv->seq_lens;
+        p.part[i].num_pages = kv->num_pages;
+        p.part[i].present = 1;
+        if (kv->num_pages > 0) {
+            if ((rc = make_map(&maps[2 * i], s, kv->k_pool, kv->num_pages)) != SPD_OK) return rc;
+            if ((rc = make_map(&maps[2 * i + 1], s, kv->v_pool, kv->num_pages)) != SPD_OK) return rc;
+            have = i;
+        }
+    }
+    for (int i = 0; i < 2 && have >= 0; ++i)   // a partition without pages borrows a descriptor it never uses
+        if (!job.part[i] || job.part[i]->num_pages == 0) {
+            maps[2 * i] = maps[2 * have];
+            maps[2 * i + 1] = maps[2 * have + 1];
+        }
+
+    plan_kernel<<<1, 1024, 0, st>>>(p);
+    ++g_launches;
+    if (cudaGetLastError() != cudaSuccess) return SPD_ERR_CUDA;
+
+    if (have >= 0) {
+        const int D = s.head_dim;
+        if (bf) {
+            rc = D == 128 ? launch_attn<MathBF16<128>>(p, maps, di.sms, st) : launch_attn<MathBF16<64>>(p, maps, di.sms, st);
+        } else {
+#define SPD_F32_CASE(DD, GG) if (D == DD && p.geff == GG) rc = launch_attn<MathF32<DD, GG>>(p, maps, di.sms, st);
+            SPD_F32_CASE(64, 1) SPD_F32_CASE(64, 2) SPD_F32_CASE(64, 4) SPD_F32_CASE(64, 8)
+            SPD_F32_CASE(128, 1) SPD_F32_CASE(128, 2) SPD_F32_CASE(128, 4) SPD_F32_CASE(128, 8)
+#undef SPD_F32_CASE
+        }
+        if (rc != SPD_OK) return rc;
+    }
+
+    const int seqs = p.B * p.S;
+    if (s.head_dim == 128) merge_kernel<128><<<(seqs + 3) / 4, 128, 0, st>>>(p);
+    else merge_kernel<64><<<(seqs + 3) / 4, 128, 0, st>>>(p);
+    ++g_launches;
+    return cudaGetLastError() == cudaSuccess ? SPD_OK : SPD_ERR_CUDA;
+}
+
+spd_partial ws_partial(const spd_shape &s, void *ws, int sms) {
+    const WsLayout L = ws_layout(s, sms);
+    uint8_t *w = static_cast<uint8_t *>(ws);
+    spd_partial part;
+    part.o = reinterpret_cast<float *>(w + L.partial_o);
+    part.m = reinterpret_cast<float *>(w + L.partial_m);
+    part.l = reinterpret_cast<float *>(w + L.partial_l);
+    return part;
+}
+
+}  // namespace
+
+extern "C" {
+
+spd_status spd_workspace_size(const spd_shape *shape, size_t *bytes) {
+    spd_status rc = check_shape(shape);
+    if (rc != SPD_OK) return rc;
+    if (!bytes) return SPD_ERR_INVALID_ARG;
+    DeviceInfo di;
+    if ((rc = device_info(&di)) != SPD_OK) return rc;
+    *bytes = ws_layout(*shape, di.sms).total;
+    return SPD_OK;
+}
+
+spd_status spd_partial_attn(const spd_shape *shape, const void *q, const spd_paged_kv *priv, spd_partial out,
+                            void *ws, size_t ws_bytes, void *cuda_stream) {
+    spd_status rc = check_shape(shape);
+    if (rc != SPD_OK) return rc;
+    if ((rc = check_kv(shape, priv)) != SPD_OK) return rc;
+    if (!out.o || !out.m || !out.l || misaligned(out.o, 16)) return SPD_ERR_INVALID_ARG;
+    Job job{};
+    job.shape = shape; job.q = q; job.part[0] = priv; job.part[1] = nullptr;
+    job.mode = OUT_PARTIAL; job.pout = out; job.pin = nullptr; job.out = nullptr; job.out_dtype = SPD_F32;
+    return run_job(job, ws, ws_bytes, cuda_stream);
+}
+
+spd_status spd_service_attn_merge(const spd_shape *shape, const void *q, const spd_paged_kv *pub, spd_partial in,
+                                  void *out, spd_dtype out_dtype, void *ws, size_t ws_bytes, void *cuda_stream) {
+    spd_status rc = check_shape(shape);
+    if (rc != SPD_OK) return rc;
+    if ((rc = check_kv(shape, pub)) != SPD_OK) return rc;
+    if (!in.o || !in.m || !in.l || misaligned(in.o, 16)) return SPD_ERR_INVALID_ARG;
+    if (!out || misaligned(out, 16)) return SPD_ERR_INVALID_ARG;
+    if (out_dtype != SPD_F32 && out_dtype != SPD_BF16) return SPD_ERR_UNSUPPORTED;
+    Job job{};
+    job.shape = shape; job.q = q; job.part[0] = nullptr; job.part[1] = pub;
+    job.mode = OUT_FINAL; job.pin = &in; job.out = out; job.out_dtype = out_dtype;
+    return run_job(job, ws, ws_bytes, cuda_stream);
+}
+
+spd_status spd_decode_step(const spd_shape *shape, const void *q, const spd_paged_kv *priv, const spd_paged_kv *pub,
+                           void *out, spd_dtype out_dtype, int32_t fused, void *ws, size_t ws_bytes,
+                           void *cuda_stream) {
+    spd_status rc = check_shape(shape);
+    if (rc != SPD_OK) return rc;
+    if ((rc = check_kv(shape, priv)) != SPD_OK) return rc;
+    if ((rc = check_kv(shape, pub)) != SPD_OK) return rc;
+    if (!out || misaligned(out, 16)) return SPD_ERR_INVALID_ARG;
+    if (out_dtype != SPD_F32 && out_dtype != SPD_BF16) return SPD_ERR_UNSUPPORTED;
+    if (fused) {
+        Job job{};
+        job.shape = shape; job.q = q; job.part[0] = priv; job.part[1] = pub;
+        job.mode = OUT_FINAL; job.pin = nullptr; job.out = out; job.out_dtype = out_dtype;
+        return run_job(job, ws, ws_bytes, cuda_stream);
+    }
+    DeviceInfo di;
+    if ((rc = device_info(&di)) != SPD_OK) return rc;
+    if (!ws || misaligned(ws, 256)) return SPD_ERR_INVALID_ARG;
+    if (ws_bytes < ws_layout(*shape, di.sms).total) return SPD_ERR_WORKSPACE;
+    const spd_partial mid = ws_partial(*shape, ws, di.sms);
+    if ((rc = spd_partial_attn(shape, q, priv, mid, ws, ws_bytes, cuda_stream)) != SPD_OK) return rc;
+    return spd_service_attn_merge(shape, q, pub, mid, out, out_dtype, ws, ws_bytes, cuda_stream);
+}
+
+spd_status spd_host_staging_size(const spd_shape *shape, int64_t priv_pages_listed, int64_t pub_pages_listed,
+                                 spd_dtype out_dtype, size_t *bytes) {
+    spd_status rc = check_shape(shape);
+    if (rc != SPD_OK) return rc;
+    if (!bytes || priv_pages_listed < 0 || pub_pages_listed < 0) return SPD_ERR_INVALID_ARG;
+    const size_t B = shape->batch, rows = B * shape->num_q_heads * shape->head_dim;
+    const size_t es = shape->dtype == SPD_BF16 ? 2 : 4, oes = out_dtype == SPD_BF16 ? 2 : 4;
+    size_t off = align_up(rows * es, 256);
+    off += 2 * (align_up((B + 1) * 4, 256) + align_up(B * 4, 256));
+    off += align_up(static_cast<size_t>(priv_pages_listed) * 4, 256) + align_up(static_cast<size_t>(pub_pages_listed) * 4, 256);
+    off += align_up(rows * oes, 256) + 256;
+    *bytes = off;
+    return SPD_OK;
+}
+
+spd_status spd_decode_step_host(const spd_shape *shape, const void *q_host, const spd_paged_kv *priv,
+                                const spd_paged_kv *pub, void *out_host, spd_dtype out_dtype, void *staging,
+                                size_t staging_bytes, void *ws, size_t ws_bytes, void *cuda_stream) {
+    spd_status rc = check_shape(shape);
+    if (rc != SPD_OK) return rc;
+    if (!q_host || !priv || !pub || !out_host || !staging || misaligned(staging, 256)) return SPD_ERR_INVALID_ARG;
+    if (!priv->page_indptr || !pub->page_indptr || !priv->seq_lens || !pub->seq_lens) return SPD_ERR_INVALID_ARG;
+    const size_t B = shape->batch, rows = B * shape->num_q_heads * shape->head_dim;
+    const size_t es = shape->dtype == SPD_BF16 ? 2 : 4, oes = out_dtype == SPD_BF16 ? 2 : 4;
+    const int64_t n_in = priv->page_indptr[B], n_out = pub->page_indptr[B];   // host reads
+    size_t need = 0;
+    if ((rc = spd_host_staging_size(shape, n_in < 0 ? 0 : n_in, n_out < 0 ? 0 : n_out, out_dtype, &need)) != SPD_OK) return rc;
+    if (n_in < 0 || n_out < 0) return SPD_ERR_INVALID_ARG;
+    if (staging_bytes < need) return SPD_ERR_WORKSPACE;
+    if ((n_in > 0 && !priv->page_indices) || (n_out > 0 && !pub->page_indices)) return SPD_ERR_INVALID_ARG;
+    cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+    uint8_t *base = static_cast<uint8_t *>(staging);
+    size_t off = 0;
+    bool ok = true;
+    auto push = [&](const void *src, size_t bytes) -> void * {
+        void *dst = base + off;
+        if (bytes) ok = ok && cudaMemcpyAsync(dst, src, bytes, cudaMemcpyHostToDevice, st) == cudaSuccess;
+        off = align_up(off + bytes, 256);
+        return dst;
+    };
+    const void *dq = push(q_host, rows * es);
+    spd_paged_kv dpriv = *priv, dpub = *pub;
+    dpriv.page_indptr = static_cast<const int32_t *>(push(priv->page_indptr, (B + 1) * 4));
+    dpriv.seq_lens = static_cast<const int32_t *>(push(priv->seq_lens, B * 4));
+    dpriv.page_indices = static_cast<const int32_t *>(push(priv->page_indices, static_cast<size_t>(n_in) * 4));
+    dpub.page_indptr = static_cast<const int32_t *>(push(pub->page_indptr, (B + 1) * 4));
+    dpub.seq_lens = static_cast<const int32_t *>(push(pub->seq_lens, B * 4));
+    dpub.page_indices = static_cast<const int32_t *>(push(pub->page_indices, static_cast<size_t>(n_out) * 4));
+    void *dout = base + off;
+    if (!ok) return SPD_ERR_CUDA;
+    rc = spd_decode_step(shape, dq, &dpriv, &dpub, dout, out_dtype, 1, ws, ws_bytes, cuda_stream);
+    if (rc != SPD_OK) return rc;
+    if (cudaMemcpyAsync(out_host, dout, rows * oes, cudaMemcpyDeviceToHost, st) != cudaSuccess) return SPD_ERR_CUDA;
+    return spd_query_device_status(ws, cuda_stream, nullptr);
+}
+
+spd_status spd_query_device_status(void *ws, void *cuda_stream, int32_t *first_bad_user) {
+    if (!ws) return SPD_ERR_INVALID_ARG;
+    cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+    int32_t hdr[8];
+    if (cudaMemcpyAsync(hdr, ws, sizeof hdr, cudaMemcpyDeviceToHost, st) != cudaSuccess) return SPD_ERR_CUDA;
+    if (cudaStreamSynchronize(st) != cudaSuccess) return SPD_ERR_CUDA;
+    if (first_bad_user) *first_bad_user = hdr[HDR_BAD_ENC] ? 0x7fffffff - hdr[HDR_BAD_ENC] : -1;
+    if (hdr[HDR_STATUS] == 0) return SPD_OK;
+    // clear the sticky words and the per-user flags (they sit right behind the header)
+    const size_t nbad = hdr[HDR_BATCH] > 0 ? static_cast<size_t>(hdr[HDR_BATCH]) * 4 : 0;
+    if (cudaMemsetAsync(ws, 0, 8, st) != cudaSuccess) return SPD_ERR_CUDA;
+    if (nbad && cudaMemsetAsync(static_cast<uint8_t *>(ws) + align_up(HDR_WORDS * 4, 256), 0, nbad, st) != cudaSuccess)
+        return SPD_ERR_CUDA;
+    if (cudaStreamSynchronize(st) != cudaSuccess) return SPD_ERR_CUDA;
+    return static_cast<spd_status>(hdr[HDR_STATUS]);
+}
+
+int64_t spd_kernel_launch_count(void) { return g_launches.load(); }
+
+const char *spd_status_string(spd_status status) {
+    switch (status) {
+        case SPD_OK: return "ok";
+        case SPD_ERR_INVALID_ARG: return "invalid argument";
+        case SPD_ERR_UNSUPPORTED: return "unsupported shape, dtype or device";
+        case SPD_ERR_WORKSPACE: return "workspace or staging buffer too small";
+        case SPD_ERR_BAD_PAGE: return "page index or sequence length out of range (seen on the device)";
+        case SPD_ERR_CUDA: return "CUDA call failed";
+        case SPD_ERR_TIMEOUT: return "a bounded wait inside a kernel ran out";
+    }
+    return "unknown status";
+}
+
+}  // extern "C"

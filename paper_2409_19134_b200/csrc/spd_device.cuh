@@ -1,0 +1,137 @@
+// Device-side building blocks for the partitioned decode-attention kernels (sm_100a):
+// mbarrier + TMA tile loads, ldmatrix / mma.sync wrappers, and the parameter blocks that the
+// host fills.  Everything here is specific to this library; nothing is shared with the CPU oracle.
+#pragma once
+
+#include <cuda.h>
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+namespace spd {
+
+constexpr int kPage = 16;             // tokens per KV page
+constexpr int kHeadsPerItem = 8;      // query heads one warp carries for one KV head
+constexpr int kMinTilesPerWarp = 4;   // do not spread tiny batches thinner than this
+constexpr uint32_t kWaitLimit = 1u << 22;  // bounded mbarrier polling (each poll may block ~us)
+
+// Words of the workspace header (int32 each).
+enum HdrWord {
+    HDR_STATUS = 0,        // 0 or an spd_status code, sticky
+    HDR_BAD_ENC = 1,       // 0 = none, else 0x7fffffff - lowest flagged user (atomicMax)
+    HDR_TOTAL_TILES = 2,   // T: page tiles over all (user, kv head, head group) sequences
+    HDR_TILES_PER_WARP = 3,
+    HDR_BATCH = 4,         // batch size of the last plan (size of the bad-user array)
+    HDR_WORDS = 64
+};
+
+// One KV partition as the kernels see it.
+struct PartDev {
+    const int32_t *indptr;
+    const int32_t *indices;
+    const int32_t *lens;
+    int32_t num_pages;
+    int32_t present;
+};
+
+enum OutMode { OUT_PARTIAL = 0, OUT_FINAL = 1 };
+
+struct Params {
+    int32_t B, Hq, Hkv, g;
+    int32_t hgroups;        // head groups per KV head: max(1, g / 8)
+    int32_t geff;           // query heads per item: min(g, 8)
+    int32_t S;              // sequences per user = Hkv * hgroups
+    int32_t num_warps;      // warps in the attention grid
+    float sm_scale;
+    const void *q;
+    PartDev part[2];        // 0 = private, 1 = public
+    // workspace
+    int32_t *hdr;
+    int32_t *pfx;           // [B+1] exclusive prefix of pages per sequence (np0 + np1)
+    int32_t *np0, *np1;     // [B] validated page counts
+    int32_t *bad;           // [B] sticky per-user flags
+    float *scratch;         // [2 * num_warps][8 * D + 16]
+    // outputs
+    int32_t mode;           // OutMode
+    float *po, *pm, *pl;    // OUT_PARTIAL destination
+    const float *in_o, *in_m, *in_l;  // OUT_FINAL: optional partial to merge in (may be null)
+    void *out;              // OUT_FINAL destination
+    int32_t out_bf16;
+};
+
+// ---------------------------------------------------------------------------------------------
+__device__ __forceinline__ uint32_t smem_u32(const void *p) {
+    return static_cast<uint32_t>(__cvta_generic_to_shared(p));
+}
+
+__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count));
+}
+__device__ __forceinline__ void fence_mbar_init() {
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+}
+__device__ __forceinline__ void fence_proxy_async() {
+    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+}
+__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive(uint32_t bar) {
+    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
+    uint32_t ok;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
+    return ok != 0;
+}
+// Bounded wait: false if the phase did not complete within the polling limit.
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity) {
+    for (uint32_t i = 0; i < kWaitLimit; ++i)
+        if (mbar_try_wait(bar, parity)) return true;
+    return false;
+}
+
+// One 2-D TMA tile load (no multicast): box at (x, y) of the tensor map into shared memory.
+__device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap *map, int x, int y, uint32_t bar) {
+    asm volatile(
+        "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
+        ::"r"(dst), "l"(reinterpret_cast<uint64_t>(map)), "r"(x), "r"(y), "r"(bar) : "memory");
+}
+
+__device__ __forceinline__ void ldsm_x4(uint32_t addr, uint32_t &r0, uint32_t &r1, uint32_t &r2, uint32_t &r3) {
+    asm volatile("ldmatrix.sync.aligned.m8n8.x4.shared.b16 {%0,%1,%2,%3}, [%4];"
+                 : "=r"(r0), "=r"(r1), "=r"(r2), "=r"(r3) : "r"(addr));
+}
+__device__ __forceinline__ void ldsm_x4_t(uint32_t addr, uint32_t &r0, uint32_t &r1, uint32_t &r2, uint32_t &r3) {
+    asm volatile("ldmatrix.sync.aligned.m8n8.x4.trans.shared.b16 {%0,%1,%2,%3}, [%4];"
+                 : "=r"(r0), "=r"(r1), "=r"(r2), "=r"(r3) : "r"(addr));
+}
+// D += A(16x16, row) * B(16x8, col), bf16 inputs, fp32 accumulate.
+__device__ __forceinline__ void mma_bf16(float (&d)[4], uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3,
+                                         uint32_t b0, uint32_t b1) {
+    asm volatile(
+        "mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
+        : "+f"(d[0]), "+f"(d[1]), "+f"(d[2]), "+f"(d[3])
+        : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
+}
+__device__ __forceinline__ float ex2_approx(float x) {
+    float y;
+    asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+    return y;
+}
+__device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
+    __nv_bfloat162 v = __floats2bfloat162_rn(lo, hi);
+    return *reinterpret_cast<uint32_t *>(&v);
+}
+
+// Raise the sticky status and remember the lowest flagged user.
+__device__ __forceinline__ void flag_error(int32_t *hdr, int code, int user) {
+    atomicCAS(&hdr[HDR_STATUS], 0, code);
+    if (user >= 0) atomicMax(&hdr[HDR_BAD_ENC], 0x7fffffff - user);
+}
+
+}  // namespace spd

@@ -1,0 +1,639 @@
+// Kernels of the partitioned decode-attention path.
+//
+//   plan_kernel   : validates lengths, counts the page tiles of every user and scans them, so
+//                   that the attention grid can cut the flattened tile stream into equal shares.
+//   attn_kernel   : persistent warps; each streams its share of (user, kv head) page tiles from
+//                   HBM through a warp-private TMA ring in shared memory and keeps a running
+//                   (O, m, l) per query head (Sec. 4.2: m = max score, l = sum exp(s - m)).
+//                   A share that ends inside a sequence leaves its (O, m, l) in scratch.
+//   merge_kernel  : second-level log-sum-exp merge of those pieces (Theorem 1 applied n-ways),
+//                   plus the sequences that own no tile at all (empty partitions).
+//
+// A "sequence" is the KV of one (user, kv head, group of <= 8 query heads): the private pages
+// followed by the public pages (either part may be absent in a given call).
+#pragma once
+
+#include "spd_device.cuh"
+
+namespace spd {
+
+constexpr float kLog2e = 1.4426950408889634f;
+
+// ------------------------------------------------------------------------------------------------
+// plan: one CTA.  pfx[u] = pages of users < u (private + public, per sequence); T = S * pfx[B].
+__global__ void __launch_bounds__(1024) plan_kernel(Params p) {
+    __shared__ int32_t warp_tot[32];
+    __shared__ int32_t carry;
+    const int tid = threadIdx.x, lane = tid & 31, wid = tid >> 5;
+    if (tid == 0) carry = 0;
+    __syncthreads();
+    for (int base = 0; base < p.B; base += 1024) {
+        const int u = base + tid;
+        int n0 = 0, n1 = 0;
+        if (u < p.B) {
+            bool bad = false;
+            for (int s = 0; s < 2; ++s) {
+                const PartDev &pt = p.part[s];
+                if (!pt.present) continue;
+                const int64_t lo = pt.indptr[u], hi = pt.indptr[u + 1], end = pt.indptr[p.B];
+                const int64_t len = pt.lens[u];
+                if (lo < 0 || hi < lo || hi > end || len < 0 || len > (hi - lo) * kPage) {
+                    bad = true;
+                } else {
+                    const int n = static_cast<int>((len + kPage - 1) / kPage);
+                    if (s == 0) n0 = n; else n1 = n;
+                }
+            }
+            if (bad) {
+                p.bad[u] = 1;
+                flag_error(p.hdr, 4 /* SPD_ERR_BAD_PAGE */, u);
+            }
+            if (bad || p.bad[u]) n0 = n1 = 0;   // flagged users stay silent until the flag is read
+            p.np0[u] = n0;
+            p.np1[u] = n1;
+        }
+        int v = n0 + n1;
+        int inc = v;
+#pragma unroll
+        for (int d = 1; d < 32; d <<= 1) {
+            int t = __shfl_up_sync(0xffffffffu, inc, d);
+            if (lane >= d) inc += t;
+        }
+        if (lane == 31) warp_tot[wid] = inc;
+        __syncthreads();
+        if (wid == 0) {
+            int w = warp_tot[lane];
+            int winc = w;
+#pragma unroll
+            for (int d = 1; d < 32; d <<= 1) {
+                int t = __shfl_up_sync(0xffffffffu, winc, d);
+                if (lane >= d) winc += t;
+            }
+            warp_tot[lane] = winc - w;   // exclusive
+        }
+        __syncthreads();
+        const int excl = carry + warp_tot[wid] + inc - v;
+        if (u < p.B) p.pfx[u] = excl;
+        __syncthreads();
+        if (tid == 1023) carry = excl + v;
+        __syncthreads();
+    }
+    if (tid == 0) {
+        const int64_t total = carry;
+        int64_t T = total * p.S;
+        if (T >= (1ll << 31)) {   // tile counter is 32-bit
+            flag_error(p.hdr, 2 /* SPD_ERR_UNSUPPORTED */, -1);
+            T = 0;
+        }
+        p.pfx[p.B] = carry;
+        int64_t per = (T + p.num_warps - 1) / p.num_warps;
+        if (per < kMinTilesPerWarp) per = kMinTilesPerWarp;
+        p.hdr[HDR_TOTAL_TILES] = static_cast<int32_t>(T);
+        p.hdr[HDR_TILES_PER_WARP] = static_cast<int32_t>(per);
+        p.hdr[HDR_BATCH] = p.B;
+    }
+}
+
+// ------------------------------------------------------------------------------------------------
+// Last step for one (user, query head): either hand out the partial, or merge with the partial
+// that came in (Theorem 1, both sides brought to the common maximum) and normalise.
+// Each lane holds V = D/32 consecutive channels of O; m and l are warp-uniform.
+template <int D>
+__device__ __forceinline__ void finalize_store(const Params &p, int u, int h, float (&o)[D / 32], float m, float l,
+                                               int lane, bool bad) {
+    constexpr int V = D / 32;
+    const int64_t idx = static_cast<int64_t>(u) * p.Hq + h;
+    if (p.mode == OUT_PARTIAL) {
+        if (bad) {
+#pragma unroll
+            for (int i = 0; i < V; ++i) o[i] = 0.f;
+            m = -INFINITY;
+            l = 0.f;
+        }
+        float *dst = p.po + idx * D + lane * V;
+        if constexpr (V == 4) *reinterpret_cast<float4 *>(dst) = make_float4(o[0], o[1], o[2], o[3]);
+        else *reinterpret_cast<float2 *>(dst) = make_float2(o[0], o[1]);
+        if (lane == 0) { p.pm[idx] = m; p.pl[idx] = l; }
+        return;
+    }
+    float L = l;
+    if (p.in_o != nullptr) {
+        const float mi = p.in_m[idx], li = p.in_l[idx];
+        const float M = fmaxf(m, mi);
+        const float w = (m == -INFINITY) ? 0.f : expf(m - M);
+        const float wi = (mi == -INFINITY) ? 0.f : expf(mi - M);
+        const float *src = p.in_o + idx * D + lane * V;
+        float oi[V];
+        if constexpr (V == 4) { float4 t = *reinterpret_cast<const float4 *>(src); oi[0] = t.x; oi[1] = t.y; oi[2] = t.z; oi[3] = t.w; }
+        else { float2 t = *reinterpret_cast<const float2 *>(src); oi[0] = t.x; oi[1] = t.y; }
+        L = w * l + wi * li;
+#pragma unroll
+        for (int i = 0; i < V; ++i) o[i] = w * o[i] + wi * oi[i];
+    }
+    const float inv = (L > 0.f && !bad) ? 1.f / L : 0.f;
+#pragma unroll
+    for (int i = 0; i < V; ++i) o[i] = (inv == 0.f) ? 0.f : o[i] * inv;
+    if (p.out_bf16) {
+        __nv_bfloat16 *dst = reinterpret_cast<__nv_bfloat16 *>(p.out) + idx * D + lane * V;
+#pragma unroll
+        for (int i = 0; i < V; i += 2)
+            *reinterpret_cast<__nv_bfloat162 *>(dst + i) = __floats2bfloat162_rn(o[i], o[i + 1]);
+    } else {
+        float *dst = reinterpret_cast<float *>(p.out) + idx * D + lane * V;
+        if constexpr (V == 4) *reinterpret_cast<float4 *>(dst) = make_float4(o[0], o[1], o[2], o[3]);
+        else *reinterpret_cast<float2 *>(dst) = make_float2(o[0], o[1]);
+    }
+}
+
+__host__ __device__ constexpr int slot_floats(int D) { return kHeadsPerItem * D + 16; }   // O[8][D], m[8], l[8]
+
+// A finished segment sits in shared memory as So[8][D+4], Sm[8], Sl[8].  kind 0: the segment is
+// a whole sequence -> finalize; kind 1/2: a piece -> scratch slot 2w / 2w+1 for the merge kernel.
+template <int D>
+__device__ __forceinline__ void segment_epilogue(const Params &p, const float *So, const float *Sm, const float *Sl,
+                                                 int u, int sq, int kind, int gwarp, int lane, bool bad) {
+    constexpr int V = D / 32, PITCH = D + 4;
+    if (kind != 0) {
+        float *dst = p.scratch + static_cast<int64_t>(2 * gwarp + (kind - 1)) * slot_floats(D);
+#pragma unroll
+        for (int hh = 0; hh < kHeadsPerItem; ++hh)
+#pragma unroll
+            for (int i = 0; i < V; ++i) dst[hh * D + lane * V + i] = So[hh * PITCH + lane * V + i];
+        if (lane < 8) {
+            dst[kHeadsPerItem * D + lane] = Sm[lane];
+            dst[kHeadsPerItem * D + 8 + lane] = Sl[lane];
+        }
+        return;
+    }
+    const int kvh = sq / p.hgroups, hg = sq - kvh * p.hgroups;
+    const int hbase = kvh * p.g + hg * kHeadsPerItem;
+    for (int hh = 0; hh < p.geff; ++hh) {
+        float o[V];
+#pragma unroll
+        for (int i = 0; i < V; ++i) o[i] = So[hh * PITCH + lane * V + i];
+        finalize_store<D>(p, u, hbase + hh, o, Sm[hh], Sl[hh], lane, bad);
+    }
+}
+
+// ------------------------------------------------------------------------------------------------
+// bf16 tile math on the tensor cores (mma.sync m16n8k16, fp32 accumulate).
+//   S  = Q K^T   : M = 16 query-head rows (8 used), N = 8 tokens (x2), K = head_dim
+//   O^T = V^T P^T : M = 16 channels (x D/16), N = 8 query heads, K = 16 tokens
+// The accumulator fragment of S (row = head, columns = two consecutive tokens) is exactly the B
+// fragment that the second product wants for P^T, so P never leaves registers.  P is split into a
+// bf16 head and a bf16 remainder (two MMAs) so that rounding P to 8 bits of mantissa does not show
+// in the output.  K and V tiles sit in shared memory as 128-byte-swizzled [half][16 tokens][64].
+template <int D_>
+struct MathBF16 {
+    static constexpr int D = D_;
+    static constexpr int kTileBytes = kPage * D * 2;
+    static constexpr int kBoxes = D / 64;          // TMA boxes per tile (64 bf16 = 128 B wide)
+    static constexpr int kBoxBytes = kPage * 128;
+    static constexpr int kBoxCols = 64;
+    static constexpr int kWarps = 8;
+    static constexpr int kStages = 3;
+    static constexpr int kExtraBytes = 0;
+    static constexpr int KS = D / 16;
+
+    struct State {
+        uint32_t qf[KS][2];
+        float o[KS][4];
+        float m, l;
+    };
+
+    __device__ static __forceinline__ void begin(State &st, const Params &p, int u, int sq, int lane, uint8_t *) {
+        const int kvh = sq / p.hgroups, hg = sq - kvh * p.hgroups;
+        const int row = lane >> 2;
+        const bool live = row < p.geff;
+        const int h = kvh * p.g + hg * kHeadsPerItem + row;
+        const __nv_bfloat16 *qrow =
+            reinterpret_cast<const __nv_bfloat16 *>(p.q) + (static_cast<int64_t>(u) * p.Hq + (live ? h : 0)) * D;
+#pragma unroll
+        for (int ks = 0; ks < KS; ++ks) {
+            const int d0 = ks * 16 + 2 * (lane & 3);
+            st.qf[ks][0] = live ? *reinterpret_cast<const uint32_t *>(qrow + d0) : 0u;
+            st.qf[ks][1] = live ? *reinterpret_cast<const uint32_t *>(qrow + d0 + 8) : 0u;
+        }
+#pragma unroll
+        for (int mt = 0; mt < KS; ++mt)
+#pragma unroll
+            for (int i = 0; i < 4; ++i) st.o[mt][i] = 0.f;
+        st.m = -INFINITY;
+        st.l = 0.f;
+    }
+
+    __device__ static __forceinline__ void tile(State &st, const Params &p, uint8_t *Ks, uint8_t *Vs, int valid,
+                                                int lane, uint8_t *) {
+        const int mat = lane >> 3, r = lane & 7;
+        const int tok = ((mat >> 1) << 3) + r;
+        const uint32_t lane_off = tok * 128;
+        const int csel = mat & 1;
+        if (valid < kPage) {
+            // V rows past the partition's end may hold anything (even NaN): zero them, since
+            // 0 * NaN would poison the product.  Rows stay rows under the 128-byte swizzle.
+            for (int i = lane; i < (kPage - valid) * 8 * kBoxes; i += 32) {
+                const int rr = valid + (i >> 3) % (kPage - valid), rest = (i >> 3) / (kPage - valid);
+                *reinterpret_cast<uint4 *>(Vs + rest * kBoxBytes + rr * 128 + (i & 7) * 16) = make_uint4(0, 0, 0, 0);
+            }
+            fence_proxy_async();
+            __syncwarp();
+        }
+        const uint32_t kbase = smem_u32(Ks), vbase = smem_u32(Vs);
+        float s[2][4];
+#pragma unroll
+        for (int i = 0; i < 4; ++i) s[0][i] = s[1][i] = 0.f;
+#pragma unroll
+        for (int ks = 0; ks < KS; ++ks) {
+            const int c = 2 * (ks & 3) + csel;
+            uint32_t b00, b01, b10, b11;
+            ldsm_x4(kbase + (ks >> 2) * kBoxBytes + lane_off + ((c ^ r) << 4), b00, b10, b01, b11);
+            // matrices: 0 = tokens 0-7 / chunk c, 1 = tokens 0-7 / chunk c+1, 2,3 = tokens 8-15
+            mma_bf16(s[0], st.qf[ks][0], 0u, st.qf[ks][1], 0u, b00, b10);
+            mma_bf16(s[1], st.qf[ks][0], 0u, st.qf[ks][1], 0u, b01, b11);
+        }
+        const int tk = 2 * (lane & 3);
+        float v0 = s[0][0] * p.sm_scale, v1 = s[0][1] * p.sm_scale;
+        float v2 = s[1][0] * p.sm_scale, v3 = s[1][1] * p.sm_scale;
+        if (tk >= valid) v0 = -INFINITY;
+        if (tk + 1 >= valid) v1 = -INFINITY;
+        if (tk + 8 >= valid) v2 = -INFINITY;
+        if (tk + 9 >= valid) v3 = -INFINITY;
+        float tmax = fmaxf(fmaxf(v0, v1), fmaxf(v2, v3));
+        tmax = fmaxf(tmax, __shfl_xor_sync(0xffffffffu, tmax, 1));
+        tmax = fmaxf(tmax, __shfl_xor_sync(0xffffffffu, tmax, 2));
+        const float m_new = fmaxf(st.m, tmax);
+        const float alpha = ex2_approx((st.m - m_new) * kLog2e);
+        const float p0 = ex2_approx((v0 - m_new) * kLog2e), p1 = ex2_approx((v1 - m_new) * kLog2e);
+        const float p2 = ex2_approx((v2 - m_new) * kLog2e), p3 = ex2_approx((v3 - m_new) * kLog2e);
+        st.l = st.l * alpha + ((p0 + p1) + (p2 + p3));
+        st.m = m_new;
+        const uint32_t bh0 = pack_bf16(p0, p1), bh1 = pack_bf16(p2, p3);
+        const __nv_bfloat162 h0 = *reinterpret_cast<const __nv_bfloat162 *>(&bh0);
+        const __nv_bfloat162 h1 = *reinterpret_cast<const __nv_bfloat162 *>(&bh1);
+        const uint32_t bl0 = pack_bf16(p0 - __low2float(h0), p1 - __high2float(h0));
+        const uint32_t bl1 = pack_bf16(p2 - __low2float(h1), p3 - __high2float(h1));
+        // the accumulator columns are heads 2*(lane%4) and +1; their rescale factors live in the
+        // quads that own those heads as rows
+        const float ae = __shfl_sync(0xffffffffu, alpha, (lane & 3) * 8);
+        const float ao = __shfl_sync(0xffffffffu, alpha, (lane & 3) * 8 + 4);
+#pragma unroll
+        for (int mt = 0; mt < KS; ++mt) {
+            const int c = 2 * (mt & 3) + csel;
+            uint32_t a0, a1, a2, a3;
+            ldsm_x4_t(vbase + (mt >> 2) * kBoxBytes + lane_off + ((c ^ r) << 4), a0, a1, a2, a3);
+            st.o[mt][0] *= ae; st.o[mt][2] *= ae;
+            st.o[mt][1] *= ao; st.o[mt][3] *= ao;
+            mma_bf16(st.o[mt], a0, a1, a2, a3, bh0, bh1);
+            mma_bf16(st.o[mt], a0, a1, a2, a3, bl0, bl1);
+        }
+    }
+
+    // Spill the running state into shared memory as So[8][D+4], Sm[8], Sl[8].
+    __device__ static __forceinline__ void finish(State &st, float *So, float *Sm, float *Sl, int lane) {
+        constexpr int PITCH = D + 4;
+        const int hd = 2 * (lane & 3), dr = lane >> 2;
+#pragma unroll
+        for (int mt = 0; mt < KS; ++mt) {
+            So[hd * PITCH + mt * 16 + dr] = st.o[mt][0];
+            So[(hd + 1) * PITCH + mt * 16 + dr] = st.o[mt][1];
+            So[hd * PITCH + mt * 16 + dr + 8] = st.o[mt][2];
+            So[(hd + 1) * PITCH + mt * 16 + dr + 8] = st.o[mt][3];
+        }
+        float l = st.l;
+        l += __shfl_xor_sync(0xffffffffu, l, 1);
+        l += __shfl_xor_sync(0xffffffffu, l, 2);
+        if ((lane & 3) == 0) { Sm[lane >> 2] = st.m; Sl[lane >> 2] = l; }
+    }
+};
+
+// ------------------------------------------------------------------------------------------------
+// fp32 tile math on the FMA pipes (no reduced precision anywhere).
+//   scores : lane = (token t = lane & 15, half of head_dim = lane >> 4); each lane walks its half
+//            row of K in float4 steps, starting at a chunk rotated by t so that the 8 lanes of a
+//            shared-memory phase hit 8 different bank groups; halves are added with one shuffle.
+//   P V    : probabilities go through a small shared array; each lane owns D/32 channels of O.
+template <int D_, int GE_>
+struct MathF32 {
+    static constexpr int D = D_, GE = GE_;
+    static constexpr int kTileBytes = kPage * D * 4;
+    static constexpr int kBoxes = 1;
+    static constexpr int kBoxBytes = kTileBytes;
+    static constexpr int kBoxCols = D;
+    static constexpr int kWarps = 4;
+    static constexpr int kStages = 3;
+    static constexpr int kExtraBytes = (kHeadsPerItem * D + kHeadsPerItem * kPage) * 4;  // q, P
+    static constexpr int V = D / 32;
+
+    struct State {
+        float o[GE][V];
+        float m[GE], l[GE];
+    };
+
+    __device__ static __forceinline__ void begin(State &st, const Params &p, int u, int sq, int lane, uint8_t *extra) {
+        float *qs = reinterpret_cast<float *>(extra);
+        const int kvh = sq / p.hgroups, hg = sq - kvh * p.hgroups;
+        const int hbase = kvh * p.g + hg * kHeadsPerItem;
+        const float *qg = reinterpret_cast<const float *>(p.q) + (static_cast<int64_t>(u) * p.Hq + hbase) * D;
+        __syncwarp();
+        for (int i = lane; i < GE * D; i += 32) qs[i] = qg[i];
+        __syncwarp();
+#pragma unroll
+        for (int hh = 0; hh < GE; ++hh) {
+#pragma unroll
+            for (int i = 0; i < V; ++i) st.o[hh][i] = 0.f;
+            st.m[hh] = -INFINITY;
+            st.l[hh] = 0.f;
+        }
+    }
+
+    __device__ static __forceinline__ void tile(State &st, const Params &p, uint8_t *Ks, uint8_t *Vs, int valid,
+                                                int lane, uint8_t *extra) {
+        const float *qs = reinterpret_cast<const float *>(extra);
+        float *Ps = reinterpret_cast<float *>(extra) + kHeadsPerItem * D;
+        const int t = lane & 15, hf = lane >> 4;
+        constexpr int HALF = D / 2, NCH = HALF / 4;
+        const float *krow = reinterpret_cast<const float *>(Ks) + t * D + hf * HALF;
+        float s[GE];
+#pragma unroll
+        for (int hh = 0; hh < GE; ++hh) s[hh] = 0.f;
+#pragma unroll
+        for (int j = 0; j < NCH; ++j) {
+            const int c = (j + t) & (NCH - 1);
+            const float4 k4 = *reinterpret_cast<const float4 *>(krow + 4 * c);
+#pragma unroll
+            for (int hh = 0; hh < GE; ++hh) {
+                const float4 q4 = *reinterpret_cast<const float4 *>(qs + hh * D + hf * HALF + 4 * c);
+                s[hh] = fmaf(k4.x, q4.x, s[hh]);
+                s[hh] = fmaf(k4.y, q4.y, s[hh]);
+                s[hh] = fmaf(k4.z, q4.z, s[hh]);
+                s[hh] = fmaf(k4.w, q4.w, s[hh]);
+            }
+        }
+        __syncwarp();   // the previous tile's readers of Ps are done
+#pragma unroll
+        for (int hh = 0; hh < GE; ++hh) {
+            float v = s[hh] + __shfl_xor_sync(0xffffffffu, s[hh], 16);
+            v = (t < valid) ? v * p.sm_scale : -INFINITY;
+            float tmax = v;
+#pragma unroll
+            for (int d = 8; d >= 1; d >>= 1) tmax = fmaxf(tmax, __shfl_xor_sync(0xffffffffu, tmax, d));
+            const float m_new = fmaxf(st.m[hh], tmax);
+            const float alpha = exp2f((st.m[hh] - m_new) * kLog2e);
+            const float pr = exp2f((v - m_new) * kLog2e);
+            st.l[hh] = st.l[hh] * alpha + (hf == 0 ? pr : 0.f);
+            st.m[hh] = m_new;
+#pragma unroll
+            for (int i = 0; i < V; ++i) st.o[hh][i] *= alpha;
+            if (hf == 0) Ps[hh * kPage + t] = pr;
+        }
+        __syncwarp();
+        const float *vcol = reinterpret_cast<const float *>(Vs) + lane * V;
+        for (int tt = 0; tt < valid; ++tt) {   // rows past `valid` are never touched
+            float vv[V];
+            if constexpr (V == 4) { float4 x = *reinterpret_cast<const float4 *>(vcol + tt * D); vv[0] = x.x; vv[1] = x.y; vv[2] = x.z; vv[3] = x.w; }
+            else { float2 x = *reinterpret_cast<const float2 *>(vcol + tt * D); vv[0] = x.x; vv[1] = x.y; }
+#pragma unroll
+            for (int hh = 0; hh < GE; ++hh) {
+                const float pr = Ps[hh * kPage + tt];
+#pragma unroll
+                for (int i = 0; i < V; ++i) st.o[hh][i] = fmaf(pr, vv[i], st.o[hh][i]);
+            }
+        }
+    }
+
+    __device__ static __forceinline__ void finish(State &st, float *So, float *Sm, float *Sl, int lane) {
+        constexpr int PITCH = D + 4;
+#pragma unroll
+        for (int hh = 0; hh < GE; ++hh) {
+#pragma unroll
+            for (int i = 0; i < V; ++i) So[hh * PITCH + lane * V + i] = st.o[hh][i];
+            float l = st.l[hh];
+#pragma unroll
+            for (int d = 8; d >= 1; d >>= 1) l += __shfl_xor_sync(0xffffffffu, l, d);
+            if (lane == 0) { Sm[hh] = st.m[hh]; Sl[hh] = l; }
+        }
+        // rows beyond GE are never read by a complete segment, but a piece copies all 8 rows
+        for (int hh = GE; hh < kHeadsPerItem; ++hh) {
+#pragma unroll
+            for (int i = 0; i < V; ++i) So[hh * PITCH + lane * V + i] = 0.f;
+            if (lane == 0) { Sm[hh] = -INFINITY; Sl[hh] = 0.f; }
+        }
+    }
+};
+
+// ------------------------------------------------------------------------------------------------
+// Where a warp stands in the flattened tile stream.  Tiles are ordered by user, then sequence
+// (kv head x head group), then page; tile index = S * pfx[u] + sq * np + j.
+struct Cursor {
+    int u, sq, j;          // user, sequence of the user, page tile of the sequence
+    int np, npp;           // tiles per sequence of this user; of which private
+    int base0, base1;      // page-table offsets of the user
+    int len0, len1;        // token counts of the user
+    int idx_cur, idx_next; // this lane's page index of the current / next batch of 32 tiles
+    int key;               // (partition << 24 | batch) that idx_cur holds, -1 = nothing
+};
+
+__device__ __forceinline__ void cursor_load_user(Cursor &c, const Params &p) {
+    c.npp = p.np0[c.u];
+    c.np = c.npp + p.np1[c.u];
+    c.base0 = p.part[0].present ? p.part[0].indptr[c.u] : 0;
+    c.base1 = p.part[1].present ? p.part[1].indptr[c.u] : 0;
+    c.len0 = p.part[0].present ? p.part[0].lens[c.u] : 0;
+    c.len1 = p.part[1].present ? p.part[1].lens[c.u] : 0;
+    c.key = -1;
+}
+
+__device__ __forceinline__ int cursor_fetch_batch(const Cursor &c, const Params &p, int part, int batch, int lane) {
+    const int i = batch * 32 + lane;
+    const int n = part ? c.np - c.npp : c.npp;
+    if (i >= n) return -1;
+    return part ? p.part[1].indices[c.base1 + i] : p.part[0].indices[c.base0 + i];
+}
+
+template <class Math>
+__global__ void __launch_bounds__(Math::kWarps * 32, 1)
+attn_kernel(const __grid_constant__ Params p, const __grid_constant__ CUtensorMap mk0,
+            const __grid_constant__ CUtensorMap mv0, const __grid_constant__ CUtensorMap mk1,
+            const __grid_constant__ CUtensorMap mv1) {
+    constexpr int D = Math::D, NS = Math::kStages, TB = Math::kTileBytes;
+    extern __shared__ uint8_t smem_raw[];
+    uint8_t *base = reinterpret_cast<uint8_t *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+    const int wid = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int gwarp = blockIdx.x * Math::kWarps + wid;
+    uint8_t *ring = base + static_cast<size_t>(wid) * NS * 2 * TB;
+    uint8_t *tail = base + static_cast<size_t>(Math::kWarps) * NS * 2 * TB;
+    uint64_t *bars = reinterpret_cast<uint64_t *>(tail) + wid * NS;
+    int4 *descs = reinterpret_cast<int4 *>(tail + Math::kWarps * NS * 8) + wid * NS;
+    uint8_t *extra = tail + Math::kWarps * NS * (8 + 16) + static_cast<size_t>(wid) * Math::kExtraBytes;
+
+    const int T = p.hdr[HDR_TOTAL_TILES], per = p.hdr[HDR_TILES_PER_WARP];
+    const int64_t t0l = static_cast<int64_t>(gwarp) * per;
+    if (t0l >= T) return;
+    const int t0 = static_cast<int>(t0l);
+    const int t1 = static_cast<int>(t0l + per < T ? t0l + per : T);
+    const int n = t1 - t0;
+
+    if (lane == 0) {
+        for (int s = 0; s < NS; ++s) mbar_init(smem_u32(&bars[s]), 1);
+        fence_mbar_init();
+    }
+    __syncwarp();
+
+    // locate the first tile: last user whose first tile is <= t0
+    Cursor c;
+    {
+        int lo = 0, hi = p.B;   // invariant: S*pfx[lo] <= t0 < S*pfx[hi]
+        while (hi - lo > 1) {
+            const int mid = (lo + hi) >> 1;
+            if (static_cast<int64_t>(p.pfx[mid]) * p.S <= t0) lo = mid; else hi = mid;
+        }
+        c.u = lo;
+        cursor_load_user(c, p);
+        const int r = t0 - p.pfx[lo] * p.S;
+        c.sq = r / c.np;
+        c.j = r - c.sq * c.np;
+    }
+
+    int issued = 0;            // tiles handed to the TMA so far
+    bool seg_from0 = false;    // the segment being issued began at the start of its sequence
+    int seg_no = 0;            // segments begun so far by this warp
+
+    auto issue = [&](int stage) {
+        // page of tile (c.u, c.sq, c.j)
+        const int part = c.j >= c.npp ? 1 : 0;
+        const int jj = part ? c.j - c.npp : c.j;
+        const int key = (part << 24) | (jj >> 5);
+        if (key != c.key) {
+            c.idx_cur = (c.key >= 0 && key == c.key + 1) ? c.idx_next : cursor_fetch_batch(c, p, part, jj >> 5, lane);
+            c.idx_next = cursor_fetch_batch(c, p, part, (jj >> 5) + 1, lane);
+            c.key = key;
+        }
+        const int page = __shfl_sync(0xffffffffu, c.idx_cur, jj & 31);
+        const int npart = part ? c.np - c.npp : c.npp;
+        int valid = kPage;
+        if (jj == npart - 1) valid = (part ? c.len1 : c.len0) - jj * kPage;
+        const bool first = (c.j == 0) || (issued == 0);
+        const bool last = (c.j == c.np - 1) || (issued == n - 1);
+        if (first) { seg_from0 = (c.j == 0); ++seg_no; }
+        int kind = 0;
+        if (last && !(seg_from0 && c.j == c.np - 1)) kind = (seg_no == 1) ? 1 : 2;
+        if (page < 0 || page >= p.part[part].num_pages) {
+            valid = 0;
+            if (lane == 0) { p.bad[c.u] = 1; flag_error(p.hdr, 4 /* SPD_ERR_BAD_PAGE */, c.u); }
+        }
+        if (lane == 0) {
+            descs[stage] = make_int4(valid, (first ? 1 : 0) | (last ? 2 : 0) | (kind << 8), c.u, c.sq);
+            const uint32_t bar = smem_u32(&bars[stage]);
+            if (valid == 0) {
+                mbar_arrive(bar);
+            } else {
+                const int kvh = c.sq / p.hgroups;
+                const int row = (page * p.Hkv + kvh) * kPage;
+                const uint32_t kdst = smem_u32(ring + static_cast<size_t>(stage) * 2 * TB), vdst = kdst + TB;
+                const CUtensorMap *mk = part ? &mk1 : &mk0, *mv = part ? &mv1 : &mv0;
+                mbar_expect_tx(bar, 2 * TB);
+#pragma unroll
+                for (int b = 0; b < Math::kBoxes; ++b) {
+                    tma_load_2d(kdst + b * Math::kBoxBytes, mk, b * Math::kBoxCols, row, bar);
+                    tma_load_2d(vdst + b * Math::kBoxBytes, mv, b * Math::kBoxCols, row, bar);
+                }
+            }
+        }
+        ++issued;
+        // advance to the next tile (skipping users that own no tile)
+        if (++c.j == c.np) {
+            c.j = 0;
+            if (++c.sq == p.S) {
+                c.sq = 0;
+                if (issued < n) {
+                    do { ++c.u; } while (c.u < p.B - 1 && p.pfx[c.u + 1] == p.pfx[c.u]);
+                    cursor_load_user(c, p);
+                }
+            } else {
+                c.key = -1;   // same user, page table starts over
+            }
+        }
+    };
+
+    for (int s = 0; s < NS && s < n; ++s) issue(s);
+
+    typename Math::State st;
+    bool seg_bad = false, dead = false;
+    int i = 0;
+    for (; i < n; ++i) {
+        const int stage = i % NS;
+        if (!mbar_wait(smem_u32(&bars[stage]), (i / NS) & 1)) { dead = true; break; }
+        const int4 d = descs[stage];
+        uint8_t *Ks = ring + static_cast<size_t>(stage) * 2 * TB, *Vs = Ks + TB;
+        if (d.y & 1) { Math::begin(st, p, d.z, d.w, lane, extra); seg_bad = false; }
+        if (d.x > 0) Math::tile(st, p, Ks, Vs, d.x, lane, extra);
+        else seg_bad = true;
+        if (d.y & 2) {
+            // the stage just consumed doubles as the staging area of the epilogue
+            __syncwarp();
+            float *So = reinterpret_cast<float *>(Ks);
+            float *Sm = So + kHeadsPerItem * (D + 4), *Sl = Sm + kHeadsPerItem;
+            Math::finish(st, So, Sm, Sl, lane);
+            __syncwarp();
+            const bool bad = seg_bad || (p.bad[d.z] != 0);
+            segment_epilogue<D>(p, So, Sm, Sl, d.z, d.w, d.y >> 8, gwarp, lane, bad);
+            fence_proxy_async();
+        }
+        __syncwarp();
+        if (issued < n) issue(stage);
+    }
+    if (dead) {
+        if (lane == 0) flag_error(p.hdr, 6 /* SPD_ERR_TIMEOUT */, -1);
+        // give the copies still in flight a bounded chance to land before the warp leaves
+        for (int k = i + 1; k < issued; ++k) mbar_wait(smem_u32(&bars[k % NS]), (k / NS) & 1);
+    }
+}
+
+// ------------------------------------------------------------------------------------------------
+// Second-level merge: one warp per sequence.  A sequence that one warp covered completely was
+// already finalised by the attention kernel; one cut across several warps is recombined here from
+// its pieces (M = max m_c; l = sum l_c e^{m_c - M}; O = sum O_c e^{m_c - M}); one that owns no tile
+// is an empty partition (O = 0, m = -inf, l = 0).
+template <int D>
+__global__ void __launch_bounds__(128) merge_kernel(Params p) {
+    constexpr int V = D / 32;
+    const int lane = threadIdx.x & 31;
+    const int seq = blockIdx.x * 4 + (threadIdx.x >> 5);
+    if (seq >= p.B * p.S) return;
+    const int u = seq / p.S, sq = seq - u * p.S;
+    const int np = p.np0[u] + p.np1[u];
+    const int per = p.hdr[HDR_TILES_PER_WARP];
+    const bool bad = p.bad[u] != 0;
+    const int kvh = sq / p.hgroups, hg = sq - kvh * p.hgroups;
+    const int hbase = kvh * p.g + hg * kHeadsPerItem;
+    int w_first = 0, w_last = -1;
+    int64_t s0 = 0;
+    if (np > 0) {
+        s0 = static_cast<int64_t>(p.pfx[u]) * p.S + static_cast<int64_t>(sq) * np;
+        w_first = static_cast<int>(s0 / per);
+        w_last = static_cast<int>((s0 + np - 1) / per);
+        if (w_first == w_last && !bad) return;   // complete: already written
+    }
+    for (int hh = 0; hh < p.geff; ++hh) {
+        float M = -INFINITY;
+        for (int w = w_first; w <= w_last; ++w) {
+            const int slot = 2 * w + ((static_cast<int64_t>(w) * per >= s0) ? 0 : 1);
+            M = fmaxf(M, p.scratch[static_cast<int64_t>(slot) * slot_floats(D) + kHeadsPerItem * D + hh]);
+        }
+        float o[V], l = 0.f;
+#pragma unroll
+        for (int i = 0; i < V; ++i) o[i] = 0.f;
+        for (int w = w_first; w <= w_last; ++w) {
+            const int slot = 2 * w + ((static_cast<int64_t>(w) * per >= s0) ? 0 : 1);
+            const float *src = p.scratch + static_cast<int64_t>(slot) * slot_floats(D);
+            const float mc = src[kHeadsPerItem * D + hh];
+            const float wgt = (mc == -INFINITY) ? 0.f : expf(mc - M);
+            l = fmaf(wgt, src[kHeadsPerItem * D + 8 + hh], l);
+#pragma unroll
+            for (int i = 0; i < V; ++i) o[i] = fmaf(wgt, src[hh * D + lane * V + i], o[i]);
+        }
+        finalize_store<D>(p, u, hbase + hh, o, M, l, lane, bad);
+    }
+}
+
+}  // namespace spd
