@@ -1,0 +1,362 @@
+#!/usr/bin/env python
+"""Benchmark of the partitioned decode-attention step (one layer, one decode step per "step").
+
+  python bench.py [--gpus N] [--steps K] [--warmup W] [--config NAME] [--impl cuda|reference]
+
+Prints ONE JSON line.  `value` is decode-attention KV GB/s (bytes of cached K and V rows divided by
+time) of spd_decode_step (fused) with every input resident in HBM; `e2e` is the same metric through
+spd_decode_step_host, whose per-step inputs (q, page tables, lengths) start in pinned host memory and
+whose output is read back inside the timed region.  The KV pools are the resident cache in both.
+
+With N > 1 (torchrun) every rank runs an independent replica on its own GPU (the path has no exchange
+step) and `value` sums the replicas over the slowest rank's time.
+
+`--impl reference` times the float64 CPU oracle on a bounded sample of the same workload.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import sys
+import threading
+import time
+
+import numpy as np
+import torch
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+sys.path.insert(0, ROOT)
+
+from paper_2409_19134_b200 import workloads as wl  # noqa: E402
+
+METRIC = "decode-attention KV GB/s"
+NOMINAL_HBM_GBS = 8000.0
+OTHER_CONFIGS = ["c3_llama3_8b_gqa", "c4_long_prompt", "c5_many_user"]
+
+
+def measured_peak():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    try:
+        with open(path) as f:
+            return float(json.load(f)["hbm_gbs"]), "measured (MEASURED_PEAKS.json hbm_gbs)"
+    except Exception:
+        return 6650.0, "fallback (6.65 TB/s, earlier measurement on this pool)"
+
+
+class ClockSampler:
+    """Samples SM clock and throttle reasons through NVML while the timed region runs."""
+
+    def __init__(self, index: int, period_s: float = 0.02):
+        self.index, self.period = index, period_s
+        self.samples, self.reasons = [], set()
+        self.max_mhz = None
+        self._stop = threading.Event()
+        self._thread = None
+        try:
+            import pynvml
+            pynvml.nvmlInit()
+            self.nv = pynvml
+            self.h = pynvml.nvmlDeviceGetHandleByIndex(index)
+            self.max_mhz = pynvml.nvmlDeviceGetMaxClockInfo(self.h, pynvml.NVML_CLOCK_SM)
+        except Exception:
+            self.nv = None
+
+    def _run(self):
+        nv = self.nv
+        names = {"hw_slowdown": 0x8, "sw_power_cap": 0x4, "hw_thermal_slowdown": 0x40,
+                 "sw_thermal_slowdown": 0x20, "hw_power_brake_slowdown": 0x80}
+        while not self._stop.is_set():
+            try:
+                self.samples.append(nv.nvmlDeviceGetClockInfo(self.h, nv.NVML_CLOCK_SM))
+                r = nv.nvmlDeviceGetCurrentClocksEventReasons(self.h) if hasattr(
+                    nv, "nvmlDeviceGetCurrentClocksEventReasons") else nv.nvmlDeviceGetCurrentClocksThrottleReasons(self.h)
+                for k, bit in names.items():
+                    if r & bit:
+                        self.reasons.add(k)
+            except Exception:
+                pass
+            time.sleep(self.period)
+
+    def __enter__(self):
+        if self.nv is not None:
+            self._thread = threading.Thread(target=self._run, daemon=True)
+            self._thread.start()
+        return self
+
+    def __exit__(self, *a):
+        self._stop.set()
+        if self._thread:
+            self._thread.join()
+
+    def summary(self):
+        if not self.samples:
+            return {"sm_mhz": None, "sm_max_mhz": self.max_mhz, "reasons": [], "samples": 0}
+        return {"sm_mhz": float(np.median(self.samples)), "sm_max_mhz": self.max_mhz,
+                "reasons": sorted(self.reasons), "samples": len(self.samples)}
+
+
+def max_over_ranks(x: float, device) -> float:
+    """Slowest rank's time (every rank gets it).  Single process: x itself."""
+    import torch.distributed as dist
+    if not (dist.is_available() and dist.is_initialized()) or dist.get_world_size() == 1:
+        return float(x)
+    t = torch.tensor([x], dtype=torch.float64, device=device)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return float(t.item())
+
+
+def replica_throughput(bytes_per_replica: int, ms_slowest: float, world: int) -> float:
+    """GB/s of `world` independent replicas that all finish within the slowest rank's time."""
+    return world * bytes_per_replica / ms_slowest / 1e6
+
+
+def dist_env():
+    return int(os.environ.get("RANK", 0)), int(os.environ.get("LOCAL_RANK", 0)), int(os.environ.get("WORLD_SIZE", 1))
+
+
+# ------------------------------------------------------------------------------------------------ oracle legs
+def _slice_heads(w, n_users, n_kvh):
+    """First n_users users and first n_kvh KV heads (with their query heads): pure slicing."""
+    from oracle import spd_oracle as orc
+    g = w.num_q_heads // w.num_kv_heads
+
+    def part(p):
+        lo = int(p.page_indptr[n_users])
+        kv = orc.kv_from_torch(wl.PagedKV(p.k_pool[:, :n_kvh].contiguous(), p.v_pool[:, :n_kvh].contiguous(),
+                                          p.page_indptr[:n_users + 1].contiguous(), p.page_indices[:lo].contiguous(),
+                                          p.seq_lens[:n_users].contiguous()))
+        return kv
+    q = orc.q_from_torch(w.q[:n_users, :n_kvh * g].contiguous())
+    toks = int(w.priv.seq_lens[:n_users].sum()) + int(w.pub.seq_lens[:n_users].sum())
+    nbytes = toks * 2 * n_kvh * w.head_dim * w.elem_size
+    return q, part(w.priv), part(w.pub), nbytes
+
+
+def oracle_sample(w_cpu, budget_s):
+    """Pick (users, kv heads) so that one oracle pass takes about budget_s; returns a timed closure."""
+    from oracle import spd_oracle as orc
+    q, a, b, nb = _slice_heads(w_cpu, 1, 1)
+    t0 = time.perf_counter()
+    orc.full(q, a, b, w_cpu.sm_scale)
+    t1 = max(time.perf_counter() - t0, 1e-4)        # one user, one KV head (few threads busy)
+    cores = orc.num_threads()
+    g = w_cpu.num_q_heads // w_cpu.num_kv_heads
+    unit = t1 * min(cores, g) / cores               # wall time of one (user, KV head) with all cores busy
+    units = max(1.0, budget_s / unit)
+    n_kvh = int(min(w_cpu.num_kv_heads, max(1, units)))
+    n_users = int(min(w_cpu.batch, max(1, units // n_kvh)))
+    q, a, b, nb = _slice_heads(w_cpu, n_users, n_kvh)
+
+    def run():
+        t = time.perf_counter()
+        orc.full(q, a, b, w_cpu.sm_scale)
+        return time.perf_counter() - t
+    return run, nb, n_users, n_kvh, cores
+
+
+def cpu_baseline(w_cpu, budget_s=12.0):
+    run, nb, n_users, n_kvh, cores = oracle_sample(w_cpu, budget_s)
+    ts = [run()]
+    while sum(ts) < 3.0 and len(ts) < 20:     # a short pass is repeated so that the clock has something to hold
+        ts.append(run())
+    dt = float(np.mean(ts))
+    return {"value": nb / dt / 1e9, "unit": "GB/s", "cores": cores, "kind": "oracle",
+            "sample": f"first {n_users} of {w_cpu.batch} users x first {n_kvh} of {w_cpu.num_kv_heads} KV heads, "
+                      f"mean of {len(ts)} passes of {dt:.2f} s", "user_tokens_per_s": n_users * n_kvh / w_cpu.num_kv_heads / dt}
+
+
+def run_reference(args):
+    rank, _, world = dist_env()
+    if rank != 0:
+        return
+    cfg = args.config
+    w = wl.make_workload(cfg, device="cpu")
+    steps, warmup = args.steps or 5, args.warmup if args.warmup is not None else 1
+    budget = min(15.0, 150.0 / (steps + warmup))
+    run, nb, n_users, n_kvh, cores = oracle_sample(w, budget)
+    for _ in range(warmup):
+        run()
+    ts = [run() for _ in range(steps)]
+    dt = float(np.mean(ts))
+    val = nb / dt / 1e9
+    sample = (f"each step: first {n_users} of {w.batch} users x first {n_kvh} of {w.num_kv_heads} KV heads "
+              f"({nb / 1e6:.1f} MB of KV)")
+    line = {"impl": "reference", "metric": METRIC, "value": val, "unit": "GB/s", "n_gpus": args.gpus, "steps": steps,
+            "warmup": warmup, "ms_per_step": dt * 1e3, "higher_is_better": True, "scaling": "weak",
+            "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+            "config": {"workload": cfg, "sample": sample},
+            "cpu_baseline": {"value": val, "unit": "GB/s", "cores": cores, "kind": "oracle", "sample": sample},
+            "e2e": {"value": val, "unit": "GB/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+            "gpu_launches": 0}
+    print(json.dumps(line), flush=True)
+
+
+# ------------------------------------------------------------------------------------------------ CUDA arm
+def time_config(spd, w, steps, warmup, fused=True):
+    """Device time of `steps` back-to-back decode steps, by CUDA events on the launching stream."""
+    shape = spd.make_shape(w.batch, w.num_q_heads, w.num_kv_heads, w.head_dim, w.dtype, w.sm_scale)
+    ws = spd.alloc_workspace(shape)
+    out = torch.empty((w.batch, w.num_q_heads, w.head_dim), dtype=torch.float32, device=w.q.device)
+    for _ in range(warmup):
+        spd.spd_decode_step(shape, w.q, w.priv, w.pub, out, ws, fused=fused)
+    torch.cuda.synchronize()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    n0 = spd.spd_kernel_launch_count()
+    e0.record()
+    for _ in range(steps):
+        spd.spd_decode_step(shape, w.q, w.priv, w.pub, out, ws, fused=fused)
+    e1.record()
+    torch.cuda.synchronize()
+    launches = spd.spd_kernel_launch_count() - n0
+    code, bad = spd.spd_query_device_status(ws)
+    if code != spd.SPD_OK or not bool(torch.isfinite(out).all()):
+        raise RuntimeError(f"decode step failed: status {code}, first bad user {bad}")
+    return e0.elapsed_time(e1) / steps, launches, shape, ws, out
+
+
+def kernel_split(spd, w, shape, ws, out, steps):
+    """Average device time of each of the three kernels, events recorded inside the library."""
+    steps = min(steps, 2000)
+    spd.spd_profile_begin(steps)
+    for _ in range(steps):
+        spd.spd_decode_step(shape, w.q, w.priv, w.pub, out, ws, fused=True)
+    r = spd.spd_profile_end()
+    n = max(r["calls"], 1)
+    return {k: r[k] / n for k in ("plan_ms", "attn_ms", "merge_ms")}
+
+
+def time_e2e(spd, w, shape, ws, steps, warmup):
+    """Per step: q, page tables and lengths from pinned host memory in, output back out."""
+    dev = w.q.device
+    pin = lambda t: t.cpu().pin_memory()
+    qh = pin(w.q)
+    tabs = [(pin(p.page_indptr), pin(p.page_indices), pin(p.seq_lens)) for p in (w.priv, w.pub)]
+    outh = torch.empty((w.batch, w.num_q_heads, w.head_dim), dtype=torch.float32).pin_memory()
+    n_in, n_out = int(tabs[0][1].numel()), int(tabs[1][1].numel())
+    staging = torch.empty(spd.spd_host_staging_size(shape, n_in, n_out, torch.float32), dtype=torch.uint8, device=dev)
+    pools = [(w.priv.k_pool, w.priv.v_pool), (w.pub.k_pool, w.pub.v_pool)]
+    call = lambda: spd.spd_decode_step_host(shape, qh, pools[0], tabs[0], pools[1], tabs[1], outh, staging, ws)
+    for _ in range(warmup):
+        call()
+    torch.cuda.synchronize()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for _ in range(steps):
+        call()
+    e1.record()
+    torch.cuda.synchronize()
+    h2d = qh.numel() * qh.element_size() + sum(t.numel() * 4 for tab in tabs for t in tab)
+    d2h = outh.numel() * 4 + 32
+    return e0.elapsed_time(e1) / steps, h2d, d2h, outh
+
+
+def run_cuda(args):
+    from paper_2409_19134_b200 import binding as spd
+    rank, local_rank, world = dist_env()
+    torch.cuda.set_device(local_rank)
+    dev = torch.device("cuda", local_rank)
+    if world > 1:
+        import torch.distributed as dist
+        dist.init_process_group("nccl", device_id=dev)
+    steps = args.steps or 2000
+    warmup = args.warmup if args.warmup is not None else 20
+    if warmup < 3:
+        warmup = 3
+    cfg = args.config
+    w = wl.make_workload(cfg, device=dev)     # every rank: its own replica of the same seeded workload
+    kvb = w.kv_bytes()
+    spd.lib()
+
+    def barrier():
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    barrier()
+    with ClockSampler(local_rank) as clocks:
+        ms, launches, shape, ws, out = time_config(spd, w, steps, warmup)
+    barrier()
+    ms_max = max_over_ranks(ms, dev)
+    value = replica_throughput(kvb, ms_max, world)
+
+    split = kernel_split(spd, w, shape, ws, out, steps)
+    e2e_ms, h2d, d2h, outh = time_e2e(spd, w, shape, ws, min(steps, 500), warmup)
+    if not torch.equal(outh, out.cpu()):
+        raise RuntimeError("host-buffer path and device path disagree")
+    e2e_ms = max_over_ranks(e2e_ms, dev)
+    e2e_val = replica_throughput(kvb, e2e_ms, world)
+
+    if rank != 0:
+        if world > 1:
+            dist.destroy_process_group()
+        return
+    peak, peak_src = measured_peak()
+    achieved = kvb / split["attn_ms"] / 1e6
+    line = {
+        "metric": METRIC, "value": value, "unit": "GB/s", "n_gpus": world, "steps": steps, "warmup": warmup,
+        "ms_per_step": ms_max, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+        "dtype": "bf16" if w.dtype == torch.bfloat16 else "f32", "data": "synthetic",
+        "config": {"workload": cfg, "users": w.batch, "q_heads": w.num_q_heads, "kv_heads": w.num_kv_heads,
+                   "head_dim": w.head_dim, "page_size": w.page_size, "kv_bytes_per_step": kvb,
+                   "parallelism": "replicas only" if world > 1 else "single GPU", "call": "spd_decode_step(fused=1)",
+                   "l2": "inputs larger than L2 (KV bytes per step >> 126 MB); no flush"},
+        "user_tokens_per_s": world * w.batch / ms_max * 1e3,
+        "pct_of_nominal_hbm_8000": 100.0 * value / world / NOMINAL_HBM_GBS,
+        "pct_of_measured_hbm": 100.0 * value / world / peak,
+        "e2e": {"value": e2e_val, "unit": "GB/s", "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
+                "ms_per_step": e2e_ms, "call": "spd_decode_step_host"},
+        "gpu_launches": launches,
+        "roofline": {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
+                     "traffic": TRAFFIC_BYTES.get(cfg), "kernel": "attn_kernel", "peak_source": peak_src,
+                     "kernel_ms": split, "timing": "separate pass, CUDA events around each kernel on the launch stream"},
+        "clocks": clocks.summary(),
+    }
+    if world == 1 and not args.no_extras:
+        others = {}
+        for name in OTHER_CONFIGS:
+            if name == cfg:
+                continue
+            del w
+            torch.cuda.empty_cache()
+            w = wl.make_workload(name, device=dev)
+            n = max(50, min(steps, int(300.0 / 1.0)))
+            o = {}
+            for fused in (True, False):
+                m, _, sh, wsx, ox = time_config(spd, w, n, 5, fused=fused)
+                o["fused" if fused else "chained"] = {"ms_per_step": m, "gbs": w.kv_bytes() / m / 1e6}
+            sp = kernel_split(spd, w, sh, wsx, ox, n)
+            o["attn_kernel_gbs"] = w.kv_bytes() / sp["attn_ms"] / 1e6
+            o["pct_of_nominal_hbm_8000"] = 100.0 * o["fused"]["gbs"] / NOMINAL_HBM_GBS
+            o["kv_bytes_per_step"] = w.kv_bytes()
+            others[name] = o
+        line["other_configs"] = others
+        w = wl.make_workload(cfg, device="cpu")
+        line["cpu_baseline"] = cpu_baseline(w)
+    print(json.dumps(line), flush=True)
+    if world > 1:
+        dist.destroy_process_group()
+
+
+# DRAM traffic (dram__bytes_read.sum + dram__bytes_write.sum) of one attn_kernel launch from an ncu
+# capture; None until a capture of the current kernel exists.
+TRAFFIC_BYTES = {}
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=None)
+    ap.add_argument("--warmup", type=int, default=None)
+    ap.add_argument("--config", default="c2_llama2_7b", choices=list(wl.CONFIGS))
+    ap.add_argument("--impl", default="cuda", choices=["cuda", "reference"])
+    ap.add_argument("--no-extras", action="store_true", help="skip the other configs and the CPU baseline")
+    args = ap.parse_args()
+    if args.impl == "reference":
+        run_reference(args)
+    else:
+        run_cuda(args)
+
+
+if __name__ == "__main__":
+    main()

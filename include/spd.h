@@ -138,6 +138,17 @@ spd_status spd_query_device_status(void *ws, void *cuda_stream, int32_t *first_b
 /* Number of kernels the library has launched in this process (for accounting in benchmarks). */
 int64_t spd_kernel_launch_count(void);
 
+/*
+ * Timing aid (no counterpart in the paper): between spd_profile_begin() and spd_profile_end()
+ * every library call (at most `max_calls` of them; a chained decode step counts as two) has its
+ * three kernels -- plan, attention, second-level merge -- bracketed by CUDA events on the
+ * caller's stream.  spd_profile_end() waits for the last recorded call and returns the number
+ * of calls recorded and the summed device time of each kernel in milliseconds.  The events add a
+ * little latency between kernels, so time whole steps with profiling off.
+ */
+spd_status spd_profile_begin(int32_t max_calls);
+spd_status spd_profile_end(int32_t *calls, double *plan_ms, double *attn_ms, double *merge_ms);
+
 /* Static text for a status code. */
 const char *spd_status_string(spd_status status);
 

@@ -20,7 +20,7 @@ _STATUS_NAMES = {0: "SPD_OK", 1: "SPD_ERR_INVALID_ARG", 2: "SPD_ERR_UNSUPPORTED"
 
 EXPORTS = ["spd_workspace_size", "spd_partial_attn", "spd_service_attn_merge", "spd_decode_step",
            "spd_host_staging_size", "spd_decode_step_host", "spd_query_device_status",
-           "spd_kernel_launch_count", "spd_status_string"]
+           "spd_kernel_launch_count", "spd_status_string", "spd_profile_begin", "spd_profile_end"]
 
 
 class SpdError(RuntimeError):
@@ -66,7 +66,10 @@ def lib() -> C.CDLL:
         L.spd_kernel_launch_count.restype = C.c_int64
         L.spd_status_string.restype = C.c_char_p
         L.spd_status_string.argtypes = [C.c_int]
-        for name in EXPORTS[:7]:
+        L.spd_profile_begin.argtypes = [C.c_int32]
+        L.spd_profile_end.argtypes = [C.POINTER(C.c_int32), C.POINTER(C.c_double), C.POINTER(C.c_double),
+                                      C.POINTER(C.c_double)]
+        for name in EXPORTS[:7] + EXPORTS[9:]:
             getattr(L, name).restype = C.c_int
         _lib = L
     return _lib
@@ -183,3 +186,14 @@ def spd_query_device_status(ws, stream=None) -> Tuple[int, int]:
 
 def spd_kernel_launch_count() -> int:
     return int(lib().spd_kernel_launch_count())
+
+
+def spd_profile_begin(max_calls: int) -> None:
+    _check(lib().spd_profile_begin(int(max_calls)), "spd_profile_begin")
+
+
+def spd_profile_end() -> dict:
+    """Returns {'calls', 'plan_ms', 'attn_ms', 'merge_ms'}: summed device time per kernel."""
+    n, a, b, c = C.c_int32(0), C.c_double(0), C.c_double(0), C.c_double(0)
+    _check(lib().spd_profile_end(C.byref(n), C.byref(a), C.byref(b), C.byref(c)), "spd_profile_end")
+    return dict(calls=int(n.value), plan_ms=a.value, attn_ms=b.value, merge_ms=c.value)

@@ -6,6 +6,7 @@
 #include <cstdio>
 #include <cstring>
 #include <mutex>
+#include <vector>
 
 #include "spd_kernels.cuh"
 
@@ -14,6 +15,18 @@ namespace {
 using namespace spd;
 
 std::atomic<int64_t> g_launches{0};
+
+// Optional timing of the three kernels of a call with CUDA events on the caller's stream.
+struct Profiler {
+    std::mutex mu;
+    bool on = false;
+    int jobs = 0, cap = 0;
+    std::vector<cudaEvent_t> ev;   // 4 per job: before plan, after plan, after attention, after merge
+} g_prof;
+
+void prof_mark(int job, int k, cudaStream_t st) {
+    if (job >= 0) cudaEventRecord(g_prof.ev[4 * job + k], st);
+}
 
 struct DeviceInfo {
     int sms = 0;
@@ -221,9 +234,16 @@ spd_status run_job(const Job &job, void *ws, size_t ws_bytes, void *stream) {
             maps[2 * i + 1] = maps[2 * have + 1];
         }
 
+    int pj = -1;
+    {
+        std::lock_guard<std::mutex> lock(g_prof.mu);
+        if (g_prof.on && g_prof.jobs < g_prof.cap) pj = g_prof.jobs++;
+    }
+    prof_mark(pj, 0, st);
     plan_kernel<<<1, 1024, 0, st>>>(p);
     ++g_launches;
     if (cudaGetLastError() != cudaSuccess) return SPD_ERR_CUDA;
+    prof_mark(pj, 1, st);
 
     if (have >= 0) {
         const int D = s.head_dim;
@@ -237,11 +257,13 @@ spd_status run_job(const Job &job, void *ws, size_t ws_bytes, void *stream) {
         }
         if (rc != SPD_OK) return rc;
     }
+    prof_mark(pj, 2, st);
 
     const int seqs = p.B * p.S;
     if (s.head_dim == 128) merge_kernel<128><<<(seqs + 3) / 4, 128, 0, st>>>(p);
     else merge_kernel<64><<<(seqs + 3) / 4, 128, 0, st>>>(p);
     ++g_launches;
+    prof_mark(pj, 3, st);
     return cudaGetLastError() == cudaSuccess ? SPD_OK : SPD_ERR_CUDA;
 }
 
@@ -393,6 +415,40 @@ spd_status spd_query_device_status(void *ws, void *cuda_stream, int32_t *first_b
 }
 
 int64_t spd_kernel_launch_count(void) { return g_launches.load(); }
+
+spd_status spd_profile_begin(int32_t max_calls) {
+    if (max_calls <= 0 || max_calls > (1 << 16)) return SPD_ERR_INVALID_ARG;
+    std::lock_guard<std::mutex> lock(g_prof.mu);
+    while (static_cast<int>(g_prof.ev.size()) < 4 * max_calls) {
+        cudaEvent_t e;
+        if (cudaEventCreate(&e) != cudaSuccess) return SPD_ERR_CUDA;
+        g_prof.ev.push_back(e);
+    }
+    g_prof.cap = max_calls;
+    g_prof.jobs = 0;
+    g_prof.on = true;
+    return SPD_OK;
+}
+
+spd_status spd_profile_end(int32_t *calls, double *plan_ms, double *attn_ms, double *merge_ms) {
+    std::lock_guard<std::mutex> lock(g_prof.mu);
+    if (!g_prof.on) return SPD_ERR_INVALID_ARG;
+    g_prof.on = false;
+    double t[3] = {0, 0, 0};
+    for (int j = 0; j < g_prof.jobs; ++j) {
+        if (cudaEventSynchronize(g_prof.ev[4 * j + 3]) != cudaSuccess) return SPD_ERR_CUDA;
+        for (int k = 0; k < 3; ++k) {
+            float ms = 0.f;
+            if (cudaEventElapsedTime(&ms, g_prof.ev[4 * j + k], g_prof.ev[4 * j + k + 1]) != cudaSuccess) return SPD_ERR_CUDA;
+            t[k] += ms;
+        }
+    }
+    if (calls) *calls = g_prof.jobs;
+    if (plan_ms) *plan_ms = t[0];
+    if (attn_ms) *attn_ms = t[1];
+    if (merge_ms) *merge_ms = t[2];
+    return SPD_OK;
+}
 
 const char *spd_status_string(spd_status status) {
     switch (status) {

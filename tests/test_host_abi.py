@@ -1,0 +1,74 @@
+"""CPU-side checks: the library loads, exports what include/spd.h declares, and rejects bad arguments
+before touching a device.  No kernel runs here."""
+import ctypes as C
+import os
+import re
+
+import pytest
+import torch
+
+from paper_2409_19134_b200 import binding as spd
+from paper_2409_19134_b200 import build as spd_build
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+
+
+@pytest.fixture(scope="module")
+def lib():
+    spd_build.build()
+    return spd.lib()
+
+
+def declared_functions():
+    text = open(os.path.join(ROOT, "include", "spd.h")).read()
+    text = re.sub(r"/\*.*?\*/", "", text, flags=re.S)
+    return sorted(set(re.findall(r"\b(spd_[a-z_]+)\s*\(", text)))
+
+
+def test_every_declared_symbol_is_exported(lib):
+    names = declared_functions()
+    assert len(names) >= 9
+    for n in names:
+        assert hasattr(lib, n), n
+    assert sorted(spd.EXPORTS) == names
+
+
+def test_status_strings(lib):
+    seen = {spd.status_string(c) for c in range(7)}
+    assert len(seen) == 7 and "unknown status" not in seen
+    assert spd.status_string(99) == "unknown status"
+
+
+def test_struct_layouts_match_header(lib):
+    assert C.sizeof(spd.Shape) == 28
+    assert C.sizeof(spd.PagedKV) == 48 and spd.PagedKV.page_indptr.offset == 24
+    assert C.sizeof(spd.Partial) == 24
+
+
+def test_bad_arguments_are_rejected_on_the_host(lib):
+    n = C.c_size_t(0)
+    ok = spd.make_shape(4, 8, 8, 64, torch.float32, 0.125)
+    assert lib.spd_workspace_size(None, C.byref(n)) == 1
+    for bad, code in ((spd.make_shape(4, 8, 8, 96, torch.float32, 1.0), 2),          # head_dim
+                      (spd.make_shape(4, 8, 3, 64, torch.float32, 1.0), 2),          # heads not divisible
+                      (spd.make_shape(4, 24, 8, 64, torch.float32, 1.0), 2),         # group of 3
+                      (spd.make_shape(4, 8, 8, 64, torch.float32, 1.0, page_size=32), 2),
+                      (spd.make_shape(0, 8, 8, 64, torch.float32, 1.0), 1),
+                      (spd.make_shape(4, 8, 8, 64, torch.float32, float("nan")), 1)):
+        assert lib.spd_workspace_size(C.byref(bad), C.byref(n)) == code
+    part = spd.Partial(None, None, None)
+    kv = spd.PagedKV(None, None, 0, None, None, None)
+    assert lib.spd_partial_attn(C.byref(ok), None, None, part, None, 0, None) == 1
+    assert lib.spd_partial_attn(C.byref(ok), None, C.byref(kv), part, None, 0, None) == 1   # null tables
+    assert lib.spd_decode_step(C.byref(ok), None, None, None, None, 0, 1, None, 0, None) == 1
+    assert lib.spd_query_device_status(None, None, None) == 1
+    assert lib.spd_profile_begin(0) == 1
+    assert lib.spd_host_staging_size(C.byref(ok), -1, 0, 0, C.byref(n)) == 1
+    assert lib.spd_host_staging_size(C.byref(ok), 10, 10, 0, C.byref(n)) == 0 and n.value > 4 * 8 * 64 * 4
+
+
+def test_binding_fails_loudly_without_the_library(monkeypatch):
+    monkeypatch.setattr(spd, "_lib", None)
+    monkeypatch.setattr(spd, "LIB_PATH", "/nonexistent/libspd.so")
+    with pytest.raises(FileNotFoundError):
+        spd.lib()
