@@ -197,3 +197,4 @@ def spd_profile_end() -> dict:
     n, a, b, c = C.c_int32(0), C.c_double(0), C.c_double(0), C.c_double(0)
     _check(lib().spd_profile_end(C.byref(n), C.byref(a), C.byref(b), C.byref(c)), "spd_profile_end")
     return dict(calls=int(n.value), plan_ms=a.value, attn_ms=b.value, merge_ms=c.value)
+

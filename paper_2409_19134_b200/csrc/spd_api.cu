@@ -115,7 +115,8 @@ spd_status check_kv(const spd_shape *s, const spd_paged_kv *kv) {
     if (!kv) return SPD_ERR_INVALID_ARG;
     if (kv->num_pages < 0) return SPD_ERR_INVALID_ARG;
     if (!kv->page_indptr || !kv->seq_lens) return SPD_ERR_INVALID_ARG;
-    if (kv->num_pages > 0 && (!kv->k_pool || !kv->v_pool || !kv->page_indices)) return SPD_ERR_INVALID_ARG;
+    // page_indices may be null when no user lists a page (the device checks that before any read)
+    if (kv->num_pages > 0 && (!kv->k_pool || !kv->v_pool)) return SPD_ERR_INVALID_ARG;
     if (misaligned(kv->k_pool, 128) || misaligned(kv->v_pool, 128)) return SPD_ERR_INVALID_ARG;
     // TMA row coordinates are 32-bit
     if (static_cast<int64_t>(kv->num_pages) * s->num_kv_heads * kPage >= (1ll << 31)) return SPD_ERR_UNSUPPORTED;

@@ -37,7 +37,8 @@ __global__ void __launch_bounds__(1024) plan_kernel(Params p) {
                 if (!pt.present) continue;
                 const int64_t lo = pt.indptr[u], hi = pt.indptr[u + 1], end = pt.indptr[p.B];
                 const int64_t len = pt.lens[u];
-                if (lo < 0 || hi < lo || hi > end || len < 0 || len > (hi - lo) * kPage) {
+                if (lo < 0 || hi < lo || hi > end || len < 0 || len > (hi - lo) * kPage ||
+                    (len > 0 && pt.indices == nullptr)) {
                     bad = true;
                 } else {
                     const int n = static_cast<int>((len + kPage - 1) / kPage);

@@ -1,0 +1,143 @@
+"""Edge cases and full-size checks of the CUDA path through the C ABI.
+
+  - bit-exact page-table / length handling (indexing probe with integer-coded values)
+  - empty partitions, users with nothing cached, slack pages, NaN-poisoned unused slots
+  - device-detected mistakes (page index outside the pool, length beyond the pages listed): no
+    fault, zeros for that user, sticky status, everyone else untouched
+  - the benchmark's full-size workloads, on sampled (user, head) outputs the oracle computes one by one
+"""
+import numpy as np
+import pytest
+import torch
+
+from oracle import spd_oracle as orc
+from paper_2409_19134_b200 import binding as spd
+from paper_2409_19134_b200 import workloads as wl
+from tests.test_gpu_parity import SMALL, TOL, assert_close, oracle_inputs, run_decode
+
+pytestmark = pytest.mark.gpu
+
+
+def _decode(w, fused=True):
+    shape = spd.make_shape(w.batch, w.num_q_heads, w.num_kv_heads, w.head_dim, w.dtype, w.sm_scale)
+    ws = spd.alloc_workspace(shape)
+    out = torch.full((w.batch, w.num_q_heads, w.head_dim), float("nan"), dtype=torch.float32, device="cuda")
+    spd.spd_decode_step(shape, w.q, w.priv, w.pub, out, ws, fused=fused)
+    status = spd.spd_query_device_status(ws)
+    return out, status, (shape, ws)
+
+
+@pytest.mark.parametrize("dtype", ["f32", "bf16"])
+@pytest.mark.parametrize("fused", [True, False])
+def test_indexing_probe_is_bit_exact(dtype, fused):
+    """V rows carry (user, kv head, token // 64, token % 64, ...) as small integers; each query head
+    puts an overwhelming score on one token, so the output must be that token's V exactly."""
+    cfg = dict(batch=6, hq=8, hkv=4, d=64, dtype=dtype, lin=("uniform", 1, 900), lout=("uniform", 0, 200), seed=41)
+    w = wl.make_workload(cfg, slack=True)
+    rng = np.random.default_rng(42)
+    g, D, P = 2, 64, 16
+    expect = np.zeros((w.batch, w.num_q_heads, D), np.float64)
+    w.q.zero_()
+    for part in (w.priv, w.pub):
+        valid = ~torch.isnan(part.k_pool.float())
+        part.k_pool[valid] = 0      # scores come only from the planted components
+    for u in range(w.batch):
+        lin, lout = int(w.priv.seq_lens[u]), int(w.pub.seq_lens[u])
+        for part, n, tag in ((w.priv, lin, 1), (w.pub, lout, 2)):
+            lo = int(part.page_indptr[u])
+            for t in range(n):
+                pg = int(part.page_indices[lo + t // P])
+                for kvh in range(w.num_kv_heads):
+                    code = torch.tensor([u, kvh, t // 64, t % 64, tag] + [3] * (D - 5), dtype=torch.float32)
+                    part.v_pool[pg, kvh, t % P] = code.to(part.v_pool.dtype)
+        for h in range(w.num_q_heads):
+            t = int(rng.integers(0, lin + lout))
+            part, tt, tag = (w.priv, t, 1) if t < lin else (w.pub, t - lin, 2)
+            pg = int(part.page_indices[int(part.page_indptr[u]) + tt // P])
+            axis = h            # 8 heads, 64 channels: every head has its own axis
+            w.q[u, h, axis] = 16.0
+            part.k_pool[pg, h // g, tt % P, axis] = 64.0     # score 1024 * scale vs 0 elsewhere
+            expect[u, h] = [u, h // g, tt // 64, tt % 64, tag] + [3] * (D - 5)
+    out, status, _ = _decode(w.to("cuda"), fused)
+    assert status == (spd.SPD_OK, -1)
+    assert np.array_equal(out.cpu().numpy().astype(np.float64), expect)
+
+
+@pytest.mark.parametrize("dtype", ["f32", "bf16"])
+def test_empty_partitions_and_idle_users(dtype):
+    lin = np.array([0, 40, 0, 17, 16, 0, 300])
+    lout = np.array([0, 0, 25, 0, 16, 1, 0])
+    cfg = dict(batch=7, hq=8, hkv=2, d=128, dtype=dtype, lin=("const", 0), lout=("const", 0), seed=43)
+    w = wl.make_workload(cfg, lengths=(lin, lout), slack=True)
+    q, kin, kout = oracle_inputs(w)
+    ref = orc.full(q, kin, kout, w.sm_scale)
+    assert np.all(ref[0] == 0)
+    for fused in (True, False):
+        out, status, _ = _decode(w.to("cuda"), fused)
+        assert status == (spd.SPD_OK, -1)
+        assert bool((out[0] == 0).all())                      # nothing cached at all: zeros, not NaN
+        assert_close(out.cpu().numpy(), ref, w.dtype, f"empty partitions fused={fused}")
+    # a batch whose public partition is empty for everyone (no public pages exist)
+    w2 = wl.make_workload(dict(cfg, batch=3), lengths=(np.array([5, 64, 33]), np.zeros(3, dtype=np.int64)))
+    q, kin, kout = oracle_inputs(w2)
+    out, status, _ = _decode(w2.to("cuda"))
+    assert status == (spd.SPD_OK, -1)
+    assert_close(out.cpu().numpy(), orc.full(q, kin, kout, w2.sm_scale), w2.dtype, "no public tokens")
+
+
+def test_bad_page_index_and_bad_length_are_contained():
+    name = "bf16_gqa4_d128"
+    w = wl.make_workload(dict(SMALL[name], name=name), slack=False)
+    q, kin, kout = oracle_inputs(w)
+    ref = orc.full(q, kin, kout, w.sm_scale)
+    wg = w.to("cuda")
+    others = [u for u in range(w.batch) if u not in (3, 5)]
+    # user 3: a private page index beyond the pool; user 5: a public length beyond its listed pages
+    wg.priv.page_indices[int(wg.priv.page_indptr[3]) + 1] = wg.priv.num_pages
+    wg.pub.seq_lens[5] = 16 * int(wg.pub.page_indptr[6] - wg.pub.page_indptr[5]) + 1
+    for fused in (True, False):
+        out, status, (shape, ws) = _decode(wg, fused)
+        assert status == (4, 3)                               # SPD_ERR_BAD_PAGE, lowest flagged user
+        assert bool((out[3] == 0).all()) and bool((out[5] == 0).all())
+        assert_close(out[others].cpu().numpy(), ref[others], w.dtype, f"bystanders fused={fused}")
+        assert spd.spd_query_device_status(ws) == (spd.SPD_OK, -1)   # the query cleared the flag
+    # negative index, negative length
+    wg = w.to("cuda")
+    wg.priv.page_indices[int(wg.priv.page_indptr[0])] = -1
+    wg.priv.seq_lens[1] = -4
+    out, status, _ = _decode(wg)
+    assert status == (4, 0) and bool((out[:2] == 0).all())
+    assert_close(out[2:].cpu().numpy(), ref[2:], w.dtype, "bystanders of negative inputs")
+
+
+FULL = ["c2_llama2_7b", "c3_llama3_8b_gqa", "c4_long_prompt", "c5_many_user"]
+
+
+@pytest.mark.parametrize("name", FULL)
+def test_full_size_sampled_outputs(name):
+    """The benchmark's workloads at full size, in the benchmark's launch configuration; the oracle
+    recomputes sampled (user, head) outputs from that user's rows gathered out of the device pools."""
+    w = wl.make_workload(name, device="cuda")
+    out, status, _ = _decode(w, fused=True)
+    assert status == (spd.SPD_OK, -1)
+    assert bool(torch.isfinite(out).all())
+    rng = np.random.default_rng(7)
+    lens = (w.priv.seq_lens + w.pub.seq_lens).cpu().numpy()
+    users = {int(np.argmax(lens)), int(np.argmin(lens))} | {int(u) for u in rng.integers(0, w.batch, 6)}
+    g = w.num_q_heads // w.num_kv_heads
+    got, ref = [], []
+    for u in sorted(users):
+        for h in {0, w.num_q_heads - 1, int(rng.integers(0, w.num_q_heads))}:
+            parts = []
+            for part in (w.priv, w.pub):
+                k, v = wl.gather_dense(part, u, h // g)
+                n = k.shape[0]
+                npg = max(1, (n + 15) // 16)
+                pad = lambda x: torch.cat([x, torch.zeros(npg * 16 - n, x.shape[1], dtype=x.dtype, device=x.device)])
+                tonp = lambda x: (orc.bf16_bits(x.cpu()) if x.dtype == torch.bfloat16 else x.cpu().numpy())
+                parts.append(orc.KV(tonp(pad(k)).reshape(npg, 1, 16, -1), tonp(pad(v)).reshape(npg, 1, 16, -1),
+                                    np.array([0, npg]), np.arange(npg), np.array([n])))
+            q1 = orc.q_from_torch(w.q[u:u + 1, h:h + 1].cpu())
+            ref.append(orc.full(q1, parts[0], parts[1], w.sm_scale)[0, 0])
+            got.append(out[u, h].cpu().numpy())
+    assert_close(np.stack(got), np.stack(ref), w.dtype, f"{name} sampled")
