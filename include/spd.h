@@ -149,6 +149,36 @@ int64_t spd_kernel_launch_count(void);
 spd_status spd_profile_begin(int32_t max_calls);
 spd_status spd_profile_end(int32_t *calls, double *plan_ms, double *attn_ms, double *merge_ms);
 
+/*
+ * spd_decode_step (fused) for callers that cannot allocate device memory.  (The paper has no
+ * counterpart; this is a packaging of the same kernels.)
+ *
+ * Some hosts of this library may not call cudaMalloc: code that runs while a CUDA graph is being
+ * captured, plug-ins of a serving engine that owns the whole memory pool and hands none out, and
+ * sandboxed per-user workers that are given buffers but no right to grow their footprint.  For them
+ * the workspace lives inside the library, in one statically declared device array of
+ * SPD_STATIC_WS_BYTES bytes that every GPU loading the library holds until the process exits.  The
+ * caller passes only inputs and the output buffer.
+ *
+ *   - Limit: the shape must need no more than SPD_STATIC_WS_BYTES of workspace (what
+ *     spd_workspace_size() reports); otherwise the call launches nothing, prints one line to stderr
+ *     and returns SPD_ERR_WORKSPACE.  On a 148-SM B200 that admits roughly
+ *     batch * num_q_heads <= 13000 at head_dim 128.
+ *   - The first call on each device looks up the array's device address (with that device current).
+ *     Make that first call outside any stream capture.
+ *   - All calls share the one array, and it keeps what the previous call left.  The call itself
+ *     clears the words that must start at zero (the sticky status and the per-user flags), so a
+ *     flag raised by an earlier call never leaks into this one.  Two calls that overlap on the GPU
+ *     (different streams, or different host threads without ordering) race on the array: order them.
+ *   - The call allocates and frees nothing, on the device or through any library.
+ *   - wait_and_check = 0: returns once the work is enqueued.  Non-zero: waits for the stream and
+ *     returns the device status as spd_query_device_status() would (*first_bad_user as there).
+ */
+#define SPD_STATIC_WS_BYTES (16u << 20)
+spd_status spd_decode_step_static(const spd_shape *shape, const void *q, const spd_paged_kv *priv,
+                                  const spd_paged_kv *pub, void *out, spd_dtype out_dtype,
+                                  int32_t wait_and_check, int32_t *first_bad_user, void *cuda_stream);
+
 /* Static text for a status code. */
 const char *spd_status_string(spd_status status);
 

@@ -20,7 +20,8 @@ _STATUS_NAMES = {0: "SPD_OK", 1: "SPD_ERR_INVALID_ARG", 2: "SPD_ERR_UNSUPPORTED"
 
 EXPORTS = ["spd_workspace_size", "spd_partial_attn", "spd_service_attn_merge", "spd_decode_step",
            "spd_host_staging_size", "spd_decode_step_host", "spd_query_device_status",
-           "spd_kernel_launch_count", "spd_status_string", "spd_profile_begin", "spd_profile_end"]
+           "spd_kernel_launch_count", "spd_status_string", "spd_profile_begin", "spd_profile_end",
+           "spd_decode_step_static"]
 
 
 class SpdError(RuntimeError):
@@ -69,6 +70,8 @@ def lib() -> C.CDLL:
         L.spd_profile_begin.argtypes = [C.c_int32]
         L.spd_profile_end.argtypes = [C.POINTER(C.c_int32), C.POINTER(C.c_double), C.POINTER(C.c_double),
                                       C.POINTER(C.c_double)]
+        L.spd_decode_step_static.argtypes = [C.POINTER(Shape), vp, C.POINTER(PagedKV), C.POINTER(PagedKV), vp, C.c_int,
+                                             C.c_int32, C.POINTER(C.c_int32), vp]
         for name in EXPORTS[:7] + EXPORTS[9:]:
             getattr(L, name).restype = C.c_int
         _lib = L
@@ -198,3 +201,21 @@ def spd_profile_end() -> dict:
     _check(lib().spd_profile_end(C.byref(n), C.byref(a), C.byref(b), C.byref(c)), "spd_profile_end")
     return dict(calls=int(n.value), plan_ms=a.value, attn_ms=b.value, merge_ms=c.value)
 
+
+STATIC_WS_BYTES = 16 << 20
+
+
+def spd_decode_step_static(shape, q, priv, pub, out, wait_and_check=True, stream=None) -> Tuple[int, int]:
+    """The fused decode step with the workspace held inside the library (nothing is allocated).
+
+    For callers that cannot allocate device memory; the shape must need at most STATIC_WS_BYTES of
+    workspace.  Returns (status, first flagged user or -1); status is SPD_OK when not waiting.
+    Raises SpdError for host-side rejections such as a shape beyond the limit."""
+    a, b = paged_kv(priv), paged_kv(pub)
+    bad = C.c_int32(-1)
+    code = lib().spd_decode_step_static(C.byref(shape), q.data_ptr(), C.byref(a), C.byref(b), out.data_ptr(),
+                                        _dtype_code(out.dtype), 1 if wait_and_check else 0, C.byref(bad),
+                                        _stream_ptr(stream))
+    if code not in (SPD_OK, 4, 6):
+        raise SpdError(code, "spd_decode_step_static")
+    return int(code), int(bad.value)

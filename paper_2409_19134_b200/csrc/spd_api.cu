@@ -465,3 +465,55 @@ const char *spd_status_string(spd_status status) {
 }
 
 }  // extern "C"
+
+// ------------------------------------------------------------------------------------------------
+// Allocation-free variant: the workspace is a device array that lives in this library.
+namespace {
+
+// The name below is a host-side handle in host code, not a device address: only
+// cudaGetSymbolAddress() turns it into a pointer that kernels and cudaMemset may use.
+static __device__ __align__(256) unsigned char g_static_ws[SPD_STATIC_WS_BYTES];
+
+// Device address of g_static_ws on the current device, looked up once per device.
+spd_status static_ws_address(void **out) {
+    static std::mutex mu;
+    static void *addr[64] = {nullptr};
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return SPD_ERR_CUDA;
+    std::lock_guard<std::mutex> lock(mu);
+    if (!addr[dev]) {
+        void *p = nullptr;
+        if (cudaGetSymbolAddress(&p, g_static_ws) != cudaSuccess || p == nullptr) return SPD_ERR_CUDA;
+        addr[dev] = p;
+    }
+    *out = addr[dev];
+    return SPD_OK;
+}
+
+}  // namespace
+
+extern "C" spd_status spd_decode_step_static(const spd_shape *shape, const void *q, const spd_paged_kv *priv,
+                                             const spd_paged_kv *pub, void *out, spd_dtype out_dtype,
+                                             int32_t wait_and_check, int32_t *first_bad_user, void *cuda_stream) {
+    spd_status rc = check_shape(shape);
+    if (rc != SPD_OK) return rc;
+    DeviceInfo di;
+    if ((rc = device_info(&di)) != SPD_OK) return rc;
+    const WsLayout L = ws_layout(*shape, di.sms);
+    if (L.total > SPD_STATIC_WS_BYTES) {
+        fprintf(stderr, "spd_decode_step_static: this shape needs %zu bytes of workspace, the built-in array holds %u; "
+                        "use spd_decode_step with a caller-provided workspace\n", L.total, SPD_STATIC_WS_BYTES);
+        return SPD_ERR_WORKSPACE;
+    }
+    void *ws = nullptr;
+    if ((rc = static_ws_address(&ws)) != SPD_OK) return rc;
+    cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+    // The array still holds the previous call's contents.  Everything in it is rewritten before it is
+    // read, except the sticky status words and the per-user flags: those must start at zero.
+    if (cudaMemsetAsync(ws, 0, 8, st) != cudaSuccess) return SPD_ERR_CUDA;
+    if (cudaMemsetAsync(static_cast<uint8_t *>(ws) + L.bad, 0, static_cast<size_t>(shape->batch) * 4, st) != cudaSuccess)
+        return SPD_ERR_CUDA;
+    rc = spd_decode_step(shape, q, priv, pub, out, out_dtype, 1, ws, SPD_STATIC_WS_BYTES, cuda_stream);
+    if (rc != SPD_OK || !wait_and_check) return rc;
+    return spd_query_device_status(ws, cuda_stream, first_bad_user);
+}
