@@ -78,15 +78,17 @@ typedef struct {
 
 /*
  * Bytes of device workspace the calls below need for `shape` on the current device.
- * The workspace holds the per-call plan, split-K scratch and the sticky status words; zero it
- * once (cudaMemset) before first use.  One workspace serves one stream at a time.
+ * The workspace holds the sticky status words, per-user flags, merge tickets, split-K scratch and
+ * the partial of a chained step; zero it once (cudaMemset) before first use, and again after an
+ * SPD_ERR_CUDA.  One workspace serves one stream at a time.
  */
 spd_status spd_workspace_size(const spd_shape *shape, size_t *bytes);
 
 /*
  * Private partial attention (protocol step 3b; Fig. 3 step 4; Sec. 4.2): for every user and
  * query head, (O, m, l) over the user's private partition.  Long partitions are split across
- * warps and recombined by a second-level log-sum-exp merge.  `out` is fully overwritten.
+ * warps and recombined by a second-level log-sum-exp merge.  `out` is fully overwritten; a user
+ * flagged by the device gets the empty partial.  One kernel launch.
  */
 spd_status spd_partial_attn(const spd_shape *shape, const void *q, const spd_paged_kv *priv,
                             spd_partial out, void *ws, size_t ws_bytes, void *cuda_stream);
@@ -141,13 +143,12 @@ int64_t spd_kernel_launch_count(void);
 /*
  * Timing aid (no counterpart in the paper): between spd_profile_begin() and spd_profile_end()
  * every library call (at most `max_calls` of them; a chained decode step counts as two) has its
- * three kernels -- plan, attention, second-level merge -- bracketed by CUDA events on the
- * caller's stream.  spd_profile_end() waits for the last recorded call and returns the number
- * of calls recorded and the summed device time of each kernel in milliseconds.  The events add a
- * little latency between kernels, so time whole steps with profiling off.
+ * kernel bracketed by CUDA events on the caller's stream.  spd_profile_end() waits for the last
+ * recorded call and returns the number of calls recorded and their summed kernel time in
+ * milliseconds.
  */
 spd_status spd_profile_begin(int32_t max_calls);
-spd_status spd_profile_end(int32_t *calls, double *plan_ms, double *attn_ms, double *merge_ms);
+spd_status spd_profile_end(int32_t *calls, double *kernel_ms);
 
 /*
  * spd_decode_step (fused) for callers that cannot allocate device memory.  (The paper has no

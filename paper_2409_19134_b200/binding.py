@@ -68,8 +68,7 @@ def lib() -> C.CDLL:
         L.spd_status_string.restype = C.c_char_p
         L.spd_status_string.argtypes = [C.c_int]
         L.spd_profile_begin.argtypes = [C.c_int32]
-        L.spd_profile_end.argtypes = [C.POINTER(C.c_int32), C.POINTER(C.c_double), C.POINTER(C.c_double),
-                                      C.POINTER(C.c_double)]
+        L.spd_profile_end.argtypes = [C.POINTER(C.c_int32), C.POINTER(C.c_double)]
         L.spd_decode_step_static.argtypes = [C.POINTER(Shape), vp, C.POINTER(PagedKV), C.POINTER(PagedKV), vp, C.c_int,
                                              C.c_int32, C.POINTER(C.c_int32), vp]
         for name in EXPORTS[:7] + EXPORTS[9:]:
@@ -196,10 +195,10 @@ def spd_profile_begin(max_calls: int) -> None:
 
 
 def spd_profile_end() -> dict:
-    """Returns {'calls', 'plan_ms', 'attn_ms', 'merge_ms'}: summed device time per kernel."""
-    n, a, b, c = C.c_int32(0), C.c_double(0), C.c_double(0), C.c_double(0)
-    _check(lib().spd_profile_end(C.byref(n), C.byref(a), C.byref(b), C.byref(c)), "spd_profile_end")
-    return dict(calls=int(n.value), plan_ms=a.value, attn_ms=b.value, merge_ms=c.value)
+    """Returns {'calls', 'kernel_ms'}: calls recorded and their summed kernel time."""
+    n, a = C.c_int32(0), C.c_double(0)
+    _check(lib().spd_profile_end(C.byref(n), C.byref(a)), "spd_profile_end")
+    return dict(calls=int(n.value), kernel_ms=a.value)
 
 
 STATIC_WS_BYTES = 16 << 20

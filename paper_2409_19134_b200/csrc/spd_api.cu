@@ -21,11 +21,20 @@ struct Profiler {
     std::mutex mu;
     bool on = false;
     int jobs = 0, cap = 0;
-    std::vector<cudaEvent_t> ev;   // 4 per job: before plan, after plan, after attention, after merge
+    std::vector<cudaEvent_t> ev;   // 2 per call: before and after the kernel
 } g_prof;
 
 void prof_mark(int job, int k, cudaStream_t st) {
-    if (job >= 0) cudaEventRecord(g_prof.ev[4 * job + k], st);
+    if (job >= 0) cudaEventRecord(g_prof.ev[2 * job + k], st);
+}
+
+std::atomic<uint32_t> g_epoch{0};
+
+// Ids of calls: non-zero, so that a zeroed workspace matches none.
+int32_t next_epoch() {
+    uint32_t e = ++g_epoch;
+    if ((e & 0x7fffffffu) == 0) e = ++g_epoch;
+    return static_cast<int32_t>(e & 0x7fffffffu);
 }
 
 struct DeviceInfo {
@@ -52,6 +61,10 @@ spd_status device_info(DeviceInfo *out) {
     return SPD_OK;
 }
 
+#ifndef SPD_TMA_L2_PROMOTION
+#define SPD_TMA_L2_PROMOTION CU_TENSOR_MAP_L2_PROMOTION_L2_256B
+#endif
+
 typedef CUresult (*EncodeTiledFn)(CUtensorMap *, CUtensorMapDataType, cuuint32_t, void *, const cuuint64_t *,
                                   const cuuint64_t *, const cuuint32_t *, const cuuint32_t *, CUtensorMapInterleave,
                                   CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
@@ -71,10 +84,10 @@ EncodeTiledFn encode_fn() {
 
 constexpr size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
 
-// Workspace layout.  The header and the bad-user array come first so that the status query can
-// find them without knowing the shape.
+// Workspace layout.  The header, the per-user flags and the tickets come first so that the status
+// query can find them without knowing the shape.
 struct WsLayout {
-    size_t hdr, bad, pfx, np0, np1, scratch, partial_o, partial_m, partial_l, total;
+    size_t hdr, bad, tickets, scratch, partial_o, partial_m, partial_l, total;
 };
 
 WsLayout ws_layout(const spd_shape &s, int sms) {
@@ -83,10 +96,11 @@ WsLayout ws_layout(const spd_shape &s, int sms) {
     const size_t B = s.batch;
     L.hdr = off;       off = align_up(off + HDR_WORDS * 4, 256);
     L.bad = off;       off = align_up(off + B * 4, 256);
-    L.pfx = off;       off = align_up(off + (B + 1) * 4, 256);
-    L.np0 = off;       off = align_up(off + B * 4, 256);
-    L.np1 = off;       off = align_up(off + B * 4, 256);
-    const size_t max_warps = static_cast<size_t>(sms) * 8;
+    const int g = s.num_q_heads / s.num_kv_heads;
+    const size_t seqs = B * s.num_kv_heads * (g > kHeadsPerItem ? g / kHeadsPerItem : 1);
+    L.tickets = off;   off = align_up(off + seqs * 4, 256);
+    constexpr int wmax = MathBF16<128>::kWarps > MathF32<128, 1>::kWarps ? MathBF16<128>::kWarps : MathF32<128, 1>::kWarps;
+    const size_t max_warps = static_cast<size_t>(sms) * wmax;
     L.scratch = off;   off = align_up(off + 2 * max_warps * slot_floats(s.head_dim) * 4, 256);
     const size_t rows = B * s.num_q_heads;
     L.partial_o = off; off = align_up(off + rows * s.head_dim * 4, 256);
@@ -135,15 +149,9 @@ spd_status make_map(CUtensorMap *map, const spd_shape &s, const void *pool, int6
     cuuint32_t estr[2] = {1, 1};
     CUresult r = fn(map, bf ? CU_TENSOR_MAP_DATA_TYPE_BFLOAT16 : CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 2,
                     const_cast<void *>(pool), dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
-                    bf ? CU_TENSOR_MAP_SWIZZLE_128B : CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                    bf ? CU_TENSOR_MAP_SWIZZLE_128B : CU_TENSOR_MAP_SWIZZLE_NONE, SPD_TMA_L2_PROMOTION,
                     CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
     return r == CUDA_SUCCESS ? SPD_OK : SPD_ERR_CUDA;
-}
-
-template <class Math>
-constexpr size_t attn_smem_bytes() {
-    return 1024 + static_cast<size_t>(Math::kWarps) * Math::kStages * (2 * Math::kTileBytes + 8 + 16) +
-           static_cast<size_t>(Math::kWarps) * Math::kExtraBytes;
 }
 
 template <class Math>
@@ -163,10 +171,7 @@ spd_status launch_attn(const Params &p, const CUtensorMap *maps, int sms, cudaSt
     return cudaGetLastError() == cudaSuccess ? SPD_OK : SPD_ERR_CUDA;
 }
 
-template <class Math>
-int warps_of() { return Math::kWarps; }
-
-// What one library call boils down to: plan -> attention -> second-level merge.
+// What one library call boils down to: one launch of the attention kernel.
 struct Job {
     const spd_shape *shape;
     const void *q;
@@ -176,6 +181,7 @@ struct Job {
     const spd_partial *pin;        // OUT_FINAL, optional
     void *out;
     spd_dtype out_dtype;
+    int32_t epoch;                 // id of the call (both halves of a chained step share one)
 };
 
 spd_status run_job(const Job &job, void *ws, size_t ws_bytes, void *stream) {
@@ -203,9 +209,8 @@ spd_status run_job(const Job &job, void *ws, size_t ws_bytes, void *stream) {
     p.num_warps = di.sms * warps_per_cta;
     p.hdr = reinterpret_cast<int32_t *>(w + L.hdr);
     p.bad = reinterpret_cast<int32_t *>(w + L.bad);
-    p.pfx = reinterpret_cast<int32_t *>(w + L.pfx);
-    p.np0 = reinterpret_cast<int32_t *>(w + L.np0);
-    p.np1 = reinterpret_cast<int32_t *>(w + L.np1);
+    p.tickets = reinterpret_cast<int32_t *>(w + L.tickets);
+    p.epoch = job.epoch;
     p.scratch = reinterpret_cast<float *>(w + L.scratch);
     p.mode = job.mode;
     p.po = job.pout.o; p.pm = job.pout.m; p.pl = job.pout.l;
@@ -235,37 +240,28 @@ spd_status run_job(const Job &job, void *ws, size_t ws_bytes, void *stream) {
             maps[2 * i + 1] = maps[2 * have + 1];
         }
 
+    if (have < 0) {
+        // no partition owns a page: the kernel still runs (it writes the empty results), with
+        // descriptors it never uses
+        memset(maps, 0, sizeof maps);
+    }
     int pj = -1;
     {
         std::lock_guard<std::mutex> lock(g_prof.mu);
         if (g_prof.on && g_prof.jobs < g_prof.cap) pj = g_prof.jobs++;
     }
     prof_mark(pj, 0, st);
-    plan_kernel<<<1, 1024, 0, st>>>(p);
-    ++g_launches;
-    if (cudaGetLastError() != cudaSuccess) return SPD_ERR_CUDA;
-    prof_mark(pj, 1, st);
-
-    if (have >= 0) {
-        const int D = s.head_dim;
-        if (bf) {
-            rc = D == 128 ? launch_attn<MathBF16<128>>(p, maps, di.sms, st) : launch_attn<MathBF16<64>>(p, maps, di.sms, st);
-        } else {
+    const int D = s.head_dim;
+    if (bf) {
+        rc = D == 128 ? launch_attn<MathBF16<128>>(p, maps, di.sms, st) : launch_attn<MathBF16<64>>(p, maps, di.sms, st);
+    } else {
 #define SPD_F32_CASE(DD, GG) if (D == DD && p.geff == GG) rc = launch_attn<MathF32<DD, GG>>(p, maps, di.sms, st);
-            SPD_F32_CASE(64, 1) SPD_F32_CASE(64, 2) SPD_F32_CASE(64, 4) SPD_F32_CASE(64, 8)
-            SPD_F32_CASE(128, 1) SPD_F32_CASE(128, 2) SPD_F32_CASE(128, 4) SPD_F32_CASE(128, 8)
+        SPD_F32_CASE(64, 1) SPD_F32_CASE(64, 2) SPD_F32_CASE(64, 4) SPD_F32_CASE(64, 8)
+        SPD_F32_CASE(128, 1) SPD_F32_CASE(128, 2) SPD_F32_CASE(128, 4) SPD_F32_CASE(128, 8)
 #undef SPD_F32_CASE
-        }
-        if (rc != SPD_OK) return rc;
     }
-    prof_mark(pj, 2, st);
-
-    const int seqs = p.B * p.S;
-    if (s.head_dim == 128) merge_kernel<128><<<(seqs + 3) / 4, 128, 0, st>>>(p);
-    else merge_kernel<64><<<(seqs + 3) / 4, 128, 0, st>>>(p);
-    ++g_launches;
-    prof_mark(pj, 3, st);
-    return cudaGetLastError() == cudaSuccess ? SPD_OK : SPD_ERR_CUDA;
+    prof_mark(pj, 1, st);
+    return rc;
 }
 
 spd_partial ws_partial(const spd_shape &s, void *ws, int sms) {
@@ -301,6 +297,7 @@ spd_status spd_partial_attn(const spd_shape *shape, const void *q, const spd_pag
     Job job{};
     job.shape = shape; job.q = q; job.part[0] = priv; job.part[1] = nullptr;
     job.mode = OUT_PARTIAL; job.pout = out; job.pin = nullptr; job.out = nullptr; job.out_dtype = SPD_F32;
+    job.epoch = next_epoch();
     return run_job(job, ws, ws_bytes, cuda_stream);
 }
 
@@ -315,6 +312,7 @@ spd_status spd_service_attn_merge(const spd_shape *shape, const void *q, const s
     Job job{};
     job.shape = shape; job.q = q; job.part[0] = nullptr; job.part[1] = pub;
     job.mode = OUT_FINAL; job.pin = &in; job.out = out; job.out_dtype = out_dtype;
+    job.epoch = next_epoch();
     return run_job(job, ws, ws_bytes, cuda_stream);
 }
 
@@ -331,15 +329,22 @@ spd_status spd_decode_step(const spd_shape *shape, const void *q, const spd_page
         Job job{};
         job.shape = shape; job.q = q; job.part[0] = priv; job.part[1] = pub;
         job.mode = OUT_FINAL; job.pin = nullptr; job.out = out; job.out_dtype = out_dtype;
+        job.epoch = next_epoch();
         return run_job(job, ws, ws_bytes, cuda_stream);
     }
     DeviceInfo di;
     if ((rc = device_info(&di)) != SPD_OK) return rc;
     if (!ws || misaligned(ws, 256)) return SPD_ERR_INVALID_ARG;
     if (ws_bytes < ws_layout(*shape, di.sms).total) return SPD_ERR_WORKSPACE;
+    // Both halves carry one call id, so a user flagged in the first half stays zeroed in the second.
     const spd_partial mid = ws_partial(*shape, ws, di.sms);
-    if ((rc = spd_partial_attn(shape, q, priv, mid, ws, ws_bytes, cuda_stream)) != SPD_OK) return rc;
-    return spd_service_attn_merge(shape, q, pub, mid, out, out_dtype, ws, ws_bytes, cuda_stream);
+    Job a{}, b{};
+    a.shape = b.shape = shape; a.q = b.q = q;
+    a.part[0] = priv; a.mode = OUT_PARTIAL; a.pout = mid; a.out_dtype = SPD_F32;
+    b.part[1] = pub; b.mode = OUT_FINAL; b.pin = &mid; b.out = out; b.out_dtype = out_dtype;
+    a.epoch = b.epoch = next_epoch();
+    if ((rc = run_job(a, ws, ws_bytes, cuda_stream)) != SPD_OK) return rc;
+    return run_job(b, ws, ws_bytes, cuda_stream);
 }
 
 spd_status spd_host_staging_size(const spd_shape *shape, int64_t priv_pages_listed, int64_t pub_pages_listed,
@@ -406,10 +411,12 @@ spd_status spd_query_device_status(void *ws, void *cuda_stream, int32_t *first_b
     if (cudaStreamSynchronize(st) != cudaSuccess) return SPD_ERR_CUDA;
     if (first_bad_user) *first_bad_user = hdr[HDR_BAD_ENC] ? 0x7fffffff - hdr[HDR_BAD_ENC] : -1;
     if (hdr[HDR_STATUS] == 0) return SPD_OK;
-    // clear the sticky words and the per-user flags (they sit right behind the header)
-    const size_t nbad = hdr[HDR_BATCH] > 0 ? static_cast<size_t>(hdr[HDR_BATCH]) * 4 : 0;
+    // clear the sticky words, the per-user flags and the tickets (a kernel that gave up on a wait may
+    // have left tickets drawn); they sit right behind the header
+    const size_t nbad = hdr[HDR_BATCH] > 0 ? align_up(static_cast<size_t>(hdr[HDR_BATCH]) * 4, 256) : 0;
+    const size_t ntic = hdr[HDR_NSEQ] > 0 ? align_up(static_cast<size_t>(hdr[HDR_NSEQ]) * 4, 256) : 0;
     if (cudaMemsetAsync(ws, 0, 8, st) != cudaSuccess) return SPD_ERR_CUDA;
-    if (nbad && cudaMemsetAsync(static_cast<uint8_t *>(ws) + align_up(HDR_WORDS * 4, 256), 0, nbad, st) != cudaSuccess)
+    if (nbad + ntic && cudaMemsetAsync(static_cast<uint8_t *>(ws) + align_up(HDR_WORDS * 4, 256), 0, nbad + ntic, st) != cudaSuccess)
         return SPD_ERR_CUDA;
     if (cudaStreamSynchronize(st) != cudaSuccess) return SPD_ERR_CUDA;
     return static_cast<spd_status>(hdr[HDR_STATUS]);
@@ -420,7 +427,7 @@ int64_t spd_kernel_launch_count(void) { return g_launches.load(); }
 spd_status spd_profile_begin(int32_t max_calls) {
     if (max_calls <= 0 || max_calls > (1 << 16)) return SPD_ERR_INVALID_ARG;
     std::lock_guard<std::mutex> lock(g_prof.mu);
-    while (static_cast<int>(g_prof.ev.size()) < 4 * max_calls) {
+    while (static_cast<int>(g_prof.ev.size()) < 2 * max_calls) {
         cudaEvent_t e;
         if (cudaEventCreate(&e) != cudaSuccess) return SPD_ERR_CUDA;
         g_prof.ev.push_back(e);
@@ -431,23 +438,19 @@ spd_status spd_profile_begin(int32_t max_calls) {
     return SPD_OK;
 }
 
-spd_status spd_profile_end(int32_t *calls, double *plan_ms, double *attn_ms, double *merge_ms) {
+spd_status spd_profile_end(int32_t *calls, double *kernel_ms) {
     std::lock_guard<std::mutex> lock(g_prof.mu);
     if (!g_prof.on) return SPD_ERR_INVALID_ARG;
     g_prof.on = false;
-    double t[3] = {0, 0, 0};
+    double t = 0;
     for (int j = 0; j < g_prof.jobs; ++j) {
-        if (cudaEventSynchronize(g_prof.ev[4 * j + 3]) != cudaSuccess) return SPD_ERR_CUDA;
-        for (int k = 0; k < 3; ++k) {
-            float ms = 0.f;
-            if (cudaEventElapsedTime(&ms, g_prof.ev[4 * j + k], g_prof.ev[4 * j + k + 1]) != cudaSuccess) return SPD_ERR_CUDA;
-            t[k] += ms;
-        }
+        float ms = 0.f;
+        if (cudaEventSynchronize(g_prof.ev[2 * j + 1]) != cudaSuccess) return SPD_ERR_CUDA;
+        if (cudaEventElapsedTime(&ms, g_prof.ev[2 * j], g_prof.ev[2 * j + 1]) != cudaSuccess) return SPD_ERR_CUDA;
+        t += ms;
     }
     if (calls) *calls = g_prof.jobs;
-    if (plan_ms) *plan_ms = t[0];
-    if (attn_ms) *attn_ms = t[1];
-    if (merge_ms) *merge_ms = t[2];
+    if (kernel_ms) *kernel_ms = t;
     return SPD_OK;
 }
 

@@ -19,9 +19,8 @@ constexpr uint32_t kWaitLimit = 1u << 22;  // bounded mbarrier polling (each pol
 enum HdrWord {
     HDR_STATUS = 0,        // 0 or an spd_status code, sticky
     HDR_BAD_ENC = 1,       // 0 = none, else 0x7fffffff - lowest flagged user (atomicMax)
-    HDR_TOTAL_TILES = 2,   // T: page tiles over all (user, kv head, head group) sequences
-    HDR_TILES_PER_WARP = 3,
-    HDR_BATCH = 4,         // batch size of the last plan (size of the bad-user array)
+    HDR_BATCH = 2,         // batch size of the last call (size of the per-user flag array)
+    HDR_NSEQ = 3,          // sequences of the last call (size of the ticket array)
     HDR_WORDS = 64
 };
 
@@ -47,9 +46,9 @@ struct Params {
     PartDev part[2];        // 0 = private, 1 = public
     // workspace
     int32_t *hdr;
-    int32_t *pfx;           // [B+1] exclusive prefix of pages per sequence (np0 + np1)
-    int32_t *np0, *np1;     // [B] validated page counts
-    int32_t *bad;           // [B] sticky per-user flags
+    int32_t *bad;           // [B] per-user flags: holds `epoch` if the user was flagged by this call
+    int32_t *tickets;       // [B * S] pieces delivered so far per sequence; zero between calls
+    int32_t epoch;          // non-zero id of this call
     float *scratch;         // [2 * num_warps][8 * D + 16]
     // outputs
     int32_t mode;           // OutMode

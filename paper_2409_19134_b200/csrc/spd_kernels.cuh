@@ -1,13 +1,16 @@
-// Kernels of the partitioned decode-attention path.
+// The kernel of the partitioned decode-attention path.
 //
-//   plan_kernel   : validates lengths, counts the page tiles of every user and scans them, so
-//                   that the attention grid can cut the flattened tile stream into equal shares.
-//   attn_kernel   : persistent warps; each streams its share of (user, kv head) page tiles from
-//                   HBM through a warp-private TMA ring in shared memory and keeps a running
-//                   (O, m, l) per query head (Sec. 4.2: m = max score, l = sum exp(s - m)).
-//                   A share that ends inside a sequence leaves its (O, m, l) in scratch.
-//   merge_kernel  : second-level log-sum-exp merge of those pieces (Theorem 1 applied n-ways),
-//                   plus the sequences that own no tile at all (empty partitions).
+// One persistent launch does a whole call:
+//   plan    : every CTA derives the same plan from the inputs alone -- validated page-tile counts
+//             per user, their prefix sums, and the equal share of the flattened tile stream that
+//             each warp of the grid owns.
+//   stream  : each warp streams its share of (user, kv head) page tiles from HBM through a
+//             warp-private TMA ring in shared memory and keeps a running (O, m, l) per query head
+//             (Sec. 4.2: m = max score, l = sum exp(s - m)).
+//   merge   : a share that ends inside a sequence leaves its (O, m, l) in scratch and takes a
+//             ticket; whoever delivers the last piece of a sequence recombines all of them
+//             (Theorem 1 applied n-ways: M = max m_c, l = sum l_c e^{m_c-M}, O = sum O_c e^{m_c-M}).
+//             Nobody waits for anybody.
 //
 // A "sequence" is the KV of one (user, kv head, group of <= 8 query heads): the private pages
 // followed by the public pages (either part may be absent in a given call).
@@ -19,79 +22,40 @@ namespace spd {
 
 constexpr float kLog2e = 1.4426950408889634f;
 
+// Shape of the bf16 attention CTA: warps per CTA and TMA ring depth per warp (8 KB per stage at
+// head_dim 128).  warps * stages * 8 KB must fit the 227 KB of shared memory; at most 16 warps.
+#ifndef SPD_BF16_WARPS
+#define SPD_BF16_WARPS 8
+#endif
+#ifndef SPD_BF16_STAGES
+#define SPD_BF16_STAGES 3
+#endif
+
 // ------------------------------------------------------------------------------------------------
-// plan: one CTA.  pfx[u] = pages of users < u (private + public, per sequence); T = S * pfx[B].
-__global__ void __launch_bounds__(1024) plan_kernel(Params p) {
-    __shared__ int32_t warp_tot[32];
-    __shared__ int32_t carry;
-    const int tid = threadIdx.x, lane = tid & 31, wid = tid >> 5;
-    if (tid == 0) carry = 0;
-    __syncthreads();
-    for (int base = 0; base < p.B; base += 1024) {
-        const int u = base + tid;
-        int n0 = 0, n1 = 0;
-        if (u < p.B) {
-            bool bad = false;
-            for (int s = 0; s < 2; ++s) {
-                const PartDev &pt = p.part[s];
-                if (!pt.present) continue;
-                const int64_t lo = pt.indptr[u], hi = pt.indptr[u + 1], end = pt.indptr[p.B];
-                const int64_t len = pt.lens[u];
-                if (lo < 0 || hi < lo || hi > end || len < 0 || len > (hi - lo) * kPage ||
-                    (len > 0 && pt.indices == nullptr)) {
-                    bad = true;
-                } else {
-                    const int n = static_cast<int>((len + kPage - 1) / kPage);
-                    if (s == 0) n0 = n; else n1 = n;
-                }
-            }
-            if (bad) {
-                p.bad[u] = 1;
-                flag_error(p.hdr, 4 /* SPD_ERR_BAD_PAGE */, u);
-            }
-            if (bad || p.bad[u]) n0 = n1 = 0;   // flagged users stay silent until the flag is read
-            p.np0[u] = n0;
-            p.np1[u] = n1;
-        }
-        int v = n0 + n1;
-        int inc = v;
+// Validated page-tile counts of one user (private, public).  A pure function of the call's inputs,
+// so every CTA that evaluates it agrees.  A user whose tables are inconsistent owns no tile, is
+// flagged for this call, and gets zeros.
+__device__ __forceinline__ void user_tiles(const Params &p, int u, int &n0, int &n1) {
+    n0 = n1 = 0;
+    bool bad = false;
 #pragma unroll
-        for (int d = 1; d < 32; d <<= 1) {
-            int t = __shfl_up_sync(0xffffffffu, inc, d);
-            if (lane >= d) inc += t;
+    for (int s = 0; s < 2; ++s) {
+        const PartDev &pt = p.part[s];
+        if (!pt.present) continue;
+        const int64_t lo = pt.indptr[u], hi = pt.indptr[u + 1], end = pt.indptr[p.B];
+        const int64_t len = pt.lens[u];
+        if (lo < 0 || hi < lo || hi > end || len < 0 || len > (hi - lo) * kPage ||
+            (len > 0 && pt.indices == nullptr)) {
+            bad = true;
+        } else {
+            const int n = static_cast<int>((len + kPage - 1) / kPage);
+            if (s == 0) n0 = n; else n1 = n;
         }
-        if (lane == 31) warp_tot[wid] = inc;
-        __syncthreads();
-        if (wid == 0) {
-            int w = warp_tot[lane];
-            int winc = w;
-#pragma unroll
-            for (int d = 1; d < 32; d <<= 1) {
-                int t = __shfl_up_sync(0xffffffffu, winc, d);
-                if (lane >= d) winc += t;
-            }
-            warp_tot[lane] = winc - w;   // exclusive
-        }
-        __syncthreads();
-        const int excl = carry + warp_tot[wid] + inc - v;
-        if (u < p.B) p.pfx[u] = excl;
-        __syncthreads();
-        if (tid == 1023) carry = excl + v;
-        __syncthreads();
     }
-    if (tid == 0) {
-        const int64_t total = carry;
-        int64_t T = total * p.S;
-        if (T >= (1ll << 31)) {   // tile counter is 32-bit
-            flag_error(p.hdr, 2 /* SPD_ERR_UNSUPPORTED */, -1);
-            T = 0;
-        }
-        p.pfx[p.B] = carry;
-        int64_t per = (T + p.num_warps - 1) / p.num_warps;
-        if (per < kMinTilesPerWarp) per = kMinTilesPerWarp;
-        p.hdr[HDR_TOTAL_TILES] = static_cast<int32_t>(T);
-        p.hdr[HDR_TILES_PER_WARP] = static_cast<int32_t>(per);
-        p.hdr[HDR_BATCH] = p.B;
+    if (bad) {
+        n0 = n1 = 0;
+        p.bad[u] = p.epoch;
+        flag_error(p.hdr, 4 /* SPD_ERR_BAD_PAGE */, u);
     }
 }
 
@@ -148,32 +112,126 @@ __device__ __forceinline__ void finalize_store(const Params &p, int u, int h, fl
 
 __host__ __device__ constexpr int slot_floats(int D) { return kHeadsPerItem * D + 16; }   // O[8][D], m[8], l[8]
 
-// A finished segment sits in shared memory as So[8][D+4], Sm[8], Sl[8].  kind 0: the segment is
-// a whole sequence -> finalize; kind 1/2: a piece -> scratch slot 2w / 2w+1 for the merge kernel.
+__device__ __forceinline__ int first_head(const Params &p, int sq) {
+    const int kvh = sq / p.hgroups, hg = sq - kvh * p.hgroups;
+    return kvh * p.g + hg * kHeadsPerItem;
+}
+
+// Scratch slot that warp w used for its piece of the sequence starting at tile s0: the first slot
+// if the sequence contains the warp's first tile, else the second.
+__device__ __forceinline__ const float *piece_slot(const Params &p, int D, int w, int per, int64_t s0) {
+    const int which = (static_cast<int64_t>(w) * per >= s0) ? 0 : 1;
+    return p.scratch + static_cast<int64_t>(2 * w + which) * slot_floats(D);
+}
+
+// Recombine the pieces that warps w_first..w_last left for one sequence (Theorem 1 applied n-ways,
+// every piece brought to the common maximum) and finalise it.  Run by the warp that delivered the
+// last piece.  Pieces are read past L1 (other SMs wrote them).  Lane c of a batch looks after piece c.
+template <int D>
+__device__ __noinline__ void merge_pieces(const Params &p, int u, int sq, int w_first, int w_last, int per,
+                                             int64_t s0, int lane, bool bad) {
+    constexpr int V = D / 32, H = kHeadsPerItem;
+    float M[H], L[H], o[H][V];
+#pragma unroll
+    for (int hh = 0; hh < H; ++hh) {
+        M[hh] = -INFINITY;
+        L[hh] = 0.f;
+#pragma unroll
+        for (int i = 0; i < V; ++i) o[hh][i] = 0.f;
+    }
+    for (int b0 = w_first; b0 <= w_last; b0 += 32) {
+        const int nb = min(32, w_last - b0 + 1);
+        const bool mine = lane < nb;
+        const float *ms = piece_slot(p, D, mine ? b0 + lane : b0, per, s0) + H * D;
+        float wgt[H];
+#pragma unroll
+        for (int hh = 0; hh < H; ++hh) {
+            if (hh >= p.geff) break;
+            const float mc = mine ? __ldcg(ms + hh) : -INFINITY;
+            const float lc = mine ? __ldcg(ms + H + hh) : 0.f;
+            float mb = mc;
+#pragma unroll
+            for (int d = 16; d >= 1; d >>= 1) mb = fmaxf(mb, __shfl_xor_sync(0xffffffffu, mb, d));
+            const float Mn = fmaxf(M[hh], mb);
+            const float resc = (M[hh] == -INFINITY) ? 0.f : expf(M[hh] - Mn);
+            wgt[hh] = (mc == -INFINITY) ? 0.f : expf(mc - Mn);
+            float ls = wgt[hh] * lc;
+#pragma unroll
+            for (int d = 16; d >= 1; d >>= 1) ls += __shfl_xor_sync(0xffffffffu, ls, d);
+            L[hh] = L[hh] * resc + ls;
+            M[hh] = Mn;
+#pragma unroll
+            for (int i = 0; i < V; ++i) o[hh][i] *= resc;
+        }
+        for (int c = 0; c < nb; ++c) {
+            const float *src = piece_slot(p, D, b0 + c, per, s0) + lane * V;
+#pragma unroll
+            for (int hh = 0; hh < H; ++hh) {
+                if (hh >= p.geff) break;
+                const float wc = __shfl_sync(0xffffffffu, wgt[hh], c);
+                if constexpr (V == 4) {
+                    const float4 x = __ldcg(reinterpret_cast<const float4 *>(src + hh * D));
+                    o[hh][0] = fmaf(wc, x.x, o[hh][0]); o[hh][1] = fmaf(wc, x.y, o[hh][1]);
+                    o[hh][2] = fmaf(wc, x.z, o[hh][2]); o[hh][3] = fmaf(wc, x.w, o[hh][3]);
+                } else {
+                    const float2 x = __ldcg(reinterpret_cast<const float2 *>(src + hh * D));
+                    o[hh][0] = fmaf(wc, x.x, o[hh][0]); o[hh][1] = fmaf(wc, x.y, o[hh][1]);
+                }
+            }
+        }
+    }
+    const int hbase = first_head(p, sq);
+#pragma unroll
+    for (int hh = 0; hh < H; ++hh)
+        if (hh < p.geff) finalize_store<D>(p, u, hbase + hh, o[hh], M[hh], L[hh], lane, bad);
+}
+
+// A finished segment sits in shared memory as So[8][D+4], Sm[8], Sl[8].
+//   kind 0  : the segment is a whole sequence -> finalise it here.
+//   kind 1/2: a piece -> scratch slot 2w / 2w+1, then a ticket on the sequence; the warp that draws
+//             the last ticket merges all pieces (and puts the ticket counter back to zero).
+// j_last is the tile of the sequence this segment ended on, t_last its index in the tile stream.
 template <int D>
 __device__ __forceinline__ void segment_epilogue(const Params &p, const float *So, const float *Sm, const float *Sl,
-                                                 int u, int sq, int kind, int gwarp, int lane, bool bad) {
+                                                 int u, int sq, int kind, int gwarp, int lane, bool bad, int per,
+                                                 int np, int j_last, int64_t t_last) {
     constexpr int V = D / 32, PITCH = D + 4;
-    if (kind != 0) {
-        float *dst = p.scratch + static_cast<int64_t>(2 * gwarp + (kind - 1)) * slot_floats(D);
+    if (kind == 0) {
+        const int hbase = first_head(p, sq);
+        for (int hh = 0; hh < p.geff; ++hh) {
+            float o[V];
 #pragma unroll
-        for (int hh = 0; hh < kHeadsPerItem; ++hh)
-#pragma unroll
-            for (int i = 0; i < V; ++i) dst[hh * D + lane * V + i] = So[hh * PITCH + lane * V + i];
-        if (lane < 8) {
-            dst[kHeadsPerItem * D + lane] = Sm[lane];
-            dst[kHeadsPerItem * D + 8 + lane] = Sl[lane];
+            for (int i = 0; i < V; ++i) o[i] = So[hh * PITCH + lane * V + i];
+            finalize_store<D>(p, u, hbase + hh, o, Sm[hh], Sl[hh], lane, bad);
         }
         return;
     }
-    const int kvh = sq / p.hgroups, hg = sq - kvh * p.hgroups;
-    const int hbase = kvh * p.g + hg * kHeadsPerItem;
-    for (int hh = 0; hh < p.geff; ++hh) {
-        float o[V];
+    float *dst = p.scratch + static_cast<int64_t>(2 * gwarp + (kind - 1)) * slot_floats(D);
 #pragma unroll
-        for (int i = 0; i < V; ++i) o[i] = So[hh * PITCH + lane * V + i];
-        finalize_store<D>(p, u, hbase + hh, o, Sm[hh], Sl[hh], lane, bad);
+    for (int hh = 0; hh < kHeadsPerItem; ++hh) {
+        if (hh >= p.geff) break;     // rows past the group are never read back
+        if constexpr (V == 4)
+            __stcg(reinterpret_cast<float4 *>(dst + hh * D + lane * V), *reinterpret_cast<const float4 *>(So + hh * PITCH + lane * V));
+        else
+            __stcg(reinterpret_cast<float2 *>(dst + hh * D + lane * V), *reinterpret_cast<const float2 *>(So + hh * PITCH + lane * V));
     }
+    if (lane < 8) {
+        __stcg(dst + kHeadsPerItem * D + lane, Sm[lane]);
+        __stcg(dst + kHeadsPerItem * D + 8 + lane, Sl[lane]);
+    }
+    const int64_t s0 = t_last - j_last;
+    const int w_first = static_cast<int>(s0 / per), w_last = static_cast<int>((s0 + np - 1) / per);
+    __threadfence();     // this lane's part of the piece is visible before the ticket is drawn
+    __syncwarp();
+    int ticket = 0;
+    int32_t *counter = p.tickets + static_cast<int64_t>(u) * p.S + sq;
+    if (lane == 0) ticket = atomicAdd(counter, 1);
+    ticket = __shfl_sync(0xffffffffu, ticket, 0);
+    if (ticket != w_last - w_first) return;   // other pieces are still to come
+    __threadfence();
+    if (lane == 0) *counter = 0;              // everybody has drawn: ready for the next call
+    const bool any_bad = bad || (__ldcg(p.bad + u) == p.epoch);
+    merge_pieces<D>(p, u, sq, w_first, w_last, per, s0, lane, any_bad);
 }
 
 // ------------------------------------------------------------------------------------------------
@@ -191,8 +249,8 @@ struct MathBF16 {
     static constexpr int kBoxes = D / 64;          // TMA boxes per tile (64 bf16 = 128 B wide)
     static constexpr int kBoxBytes = kPage * 128;
     static constexpr int kBoxCols = 64;
-    static constexpr int kWarps = 8;
-    static constexpr int kStages = 3;
+    static constexpr int kWarps = SPD_BF16_WARPS;
+    static constexpr int kStages = SPD_BF16_STAGES;
     static constexpr int kExtraBytes = 0;
     static constexpr int KS = D / 16;
 
@@ -424,7 +482,7 @@ struct MathF32 {
 
 // ------------------------------------------------------------------------------------------------
 // Where a warp stands in the flattened tile stream.  Tiles are ordered by user, then sequence
-// (kv head x head group), then page; tile index = S * pfx[u] + sq * np + j.
+// (kv head x head group), then page; tile index = S * (tiles of earlier users) + sq * np + j.
 struct Cursor {
     int u, sq, j;          // user, sequence of the user, page tile of the sequence
     int np, npp;           // tiles per sequence of this user; of which private
@@ -435,8 +493,10 @@ struct Cursor {
 };
 
 __device__ __forceinline__ void cursor_load_user(Cursor &c, const Params &p) {
-    c.npp = p.np0[c.u];
-    c.np = c.npp + p.np1[c.u];
+    int n0, n1;
+    user_tiles(p, c.u, n0, n1);
+    c.npp = n0;
+    c.np = n0 + n1;
     c.base0 = p.part[0].present ? p.part[0].indptr[c.u] : 0;
     c.base1 = p.part[1].present ? p.part[1].indptr[c.u] : 0;
     c.len0 = p.part[0].present ? p.part[0].lens[c.u] : 0;
@@ -451,23 +511,97 @@ __device__ __forceinline__ int cursor_fetch_batch(const Cursor &c, const Params 
     return part ? p.part[1].indices[c.base1 + i] : p.part[0].indices[c.base0 + i];
 }
 
+// Shared-memory carve-up behind the rings: mbarriers (8 B each), then the per-stage descriptors
+// (two int4 each, so 16-byte aligned), then each warp's private extra area (16-byte aligned).
+template <class Math>
+__host__ __device__ constexpr size_t attn_desc_offset() {
+    return (static_cast<size_t>(Math::kWarps) * Math::kStages * 8 + 15) / 16 * 16;
+}
+template <class Math>
+__host__ __device__ constexpr size_t attn_extra_offset() {
+    return attn_desc_offset<Math>() + static_cast<size_t>(Math::kWarps) * Math::kStages * 32;
+}
+template <class Math>
+__host__ __device__ constexpr size_t attn_smem_bytes() {
+    return 1024 + static_cast<size_t>(Math::kWarps) * Math::kStages * 2 * Math::kTileBytes + attn_extra_offset<Math>() +
+           static_cast<size_t>(Math::kWarps) * Math::kExtraBytes;
+}
+
 template <class Math>
 __global__ void __launch_bounds__(Math::kWarps * 32, 1)
 attn_kernel(const __grid_constant__ Params p, const __grid_constant__ CUtensorMap mk0,
             const __grid_constant__ CUtensorMap mv0, const __grid_constant__ CUtensorMap mk1,
             const __grid_constant__ CUtensorMap mv1) {
-    constexpr int D = Math::D, NS = Math::kStages, TB = Math::kTileBytes;
+    constexpr int D = Math::D, NS = Math::kStages, TB = Math::kTileBytes, NT = Math::kWarps * 32;
+    static_assert(TB % 1024 == 0, "swizzled tiles need 1024-byte aligned bases");
+    static_assert(Math::kExtraBytes % 16 == 0, "per-warp extra area holds float4 data");
+    static_assert(2 * TB >= (kHeadsPerItem * (D + 4) + 2 * kHeadsPerItem) * 4, "a stage must hold the epilogue staging");
+    static_assert(attn_smem_bytes<Math>() + 2048 <= 227 * 1024, "ring does not fit shared memory");
+    static_assert(Math::kWarps <= 16 && Math::kStages >= 2, "CTA shape");
     extern __shared__ uint8_t smem_raw[];
+    __shared__ int32_t chunk_pfx[NT + 1];
+    __shared__ int32_t warp_tot[Math::kWarps];
     uint8_t *base = reinterpret_cast<uint8_t *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
     const int wid = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int gwarp = blockIdx.x * Math::kWarps + wid;
     uint8_t *ring = base + static_cast<size_t>(wid) * NS * 2 * TB;
     uint8_t *tail = base + static_cast<size_t>(Math::kWarps) * NS * 2 * TB;
     uint64_t *bars = reinterpret_cast<uint64_t *>(tail) + wid * NS;
-    int4 *descs = reinterpret_cast<int4 *>(tail + Math::kWarps * NS * 8) + wid * NS;
-    uint8_t *extra = tail + Math::kWarps * NS * (8 + 16) + static_cast<size_t>(wid) * Math::kExtraBytes;
+    int4 *descs = reinterpret_cast<int4 *>(tail + attn_desc_offset<Math>()) + wid * NS * 2;
+    uint8_t *extra = tail + attn_extra_offset<Math>() + static_cast<size_t>(wid) * Math::kExtraBytes;
 
-    const int T = p.hdr[HDR_TOTAL_TILES], per = p.hdr[HDR_TILES_PER_WARP];
+    // ---- plan: every CTA computes the same thing from the inputs alone -------------------------
+    // Thread t sums the tiles of users [t*C, (t+1)*C); a block scan gives chunk prefixes.
+    const int C = (p.B + NT - 1) / NT;
+    {
+        int sum = 0;
+        const int ub = threadIdx.x * C, ue = min(p.B, ub + C);
+        for (int u = ub; u < ue; ++u) {
+            int n0, n1;
+            user_tiles(p, u, n0, n1);
+            sum += n0 + n1;
+        }
+        int inc = sum;
+#pragma unroll
+        for (int d = 1; d < 32; d <<= 1) {
+            const int t = __shfl_up_sync(0xffffffffu, inc, d);
+            if (lane >= d) inc += t;
+        }
+        if (lane == 31) warp_tot[wid] = inc;
+        __syncthreads();
+        int before = 0;
+        for (int w = 0; w < wid; ++w) before += warp_tot[w];
+        chunk_pfx[threadIdx.x] = before + inc - sum;
+        if (threadIdx.x == NT - 1) chunk_pfx[NT] = before + inc;
+        __syncthreads();
+    }
+    const int64_t T64 = static_cast<int64_t>(chunk_pfx[NT]) * p.S;
+    if (blockIdx.x == 0 && threadIdx.x == 0) {
+        p.hdr[HDR_BATCH] = p.B;
+        p.hdr[HDR_NSEQ] = p.B * p.S;
+        if (T64 >= (1ll << 31)) flag_error(p.hdr, 2 /* SPD_ERR_UNSUPPORTED */, -1);   // 32-bit tile counter
+    }
+    const int T = T64 >= (1ll << 31) ? 0 : static_cast<int>(T64);
+    int per = (T + p.num_warps - 1) / p.num_warps;
+    if (per < kMinTilesPerWarp) per = kMinTilesPerWarp;
+
+    // ---- users that own no tile (nothing cached, or flagged): their outputs are written here ----
+    for (int u = gwarp; u < p.B; u += p.num_warps) {
+        int n0, n1;
+        user_tiles(p, u, n0, n1);
+        if (n0 + n1 != 0) continue;
+        const bool bad = __ldcg(p.bad + u) == p.epoch;
+        for (int sq = 0; sq < p.S; ++sq) {
+            const int hbase = first_head(p, sq);
+            for (int hh = 0; hh < p.geff; ++hh) {
+                float o[D / 32];
+#pragma unroll
+                for (int i = 0; i < D / 32; ++i) o[i] = 0.f;
+                finalize_store<D>(p, u, hbase + hh, o, -INFINITY, 0.f, lane, bad);
+            }
+        }
+    }
+
     const int64_t t0l = static_cast<int64_t>(gwarp) * per;
     if (t0l >= T) return;
     const int t0 = static_cast<int>(t0l);
@@ -480,17 +614,24 @@ attn_kernel(const __grid_constant__ Params p, const __grid_constant__ CUtensorMa
     }
     __syncwarp();
 
-    // locate the first tile: last user whose first tile is <= t0
+    // locate the first tile: the user u with S * pfx[u] <= t0 < S * pfx[u + 1]
     Cursor c;
     {
-        int lo = 0, hi = p.B;   // invariant: S*pfx[lo] <= t0 < S*pfx[hi]
+        const int x = t0 / p.S;   // in units of tiles per sequence
+        int lo = 0, hi = NT;      // invariant: chunk_pfx[lo] <= x < chunk_pfx[hi]
         while (hi - lo > 1) {
             const int mid = (lo + hi) >> 1;
-            if (static_cast<int64_t>(p.pfx[mid]) * p.S <= t0) lo = mid; else hi = mid;
+            if (chunk_pfx[mid] <= x) lo = mid; else hi = mid;
         }
-        c.u = lo;
+        int acc = chunk_pfx[lo], u = lo * C, n0 = 0, n1 = 0;
+        for (;; ++u) {            // ends inside the chunk, because the chunk holds tile x
+            user_tiles(p, u, n0, n1);
+            if (acc + n0 + n1 > x) break;
+            acc += n0 + n1;
+        }
+        c.u = u;
         cursor_load_user(c, p);
-        const int r = t0 - p.pfx[lo] * p.S;
+        const int r = t0 - acc * p.S;
         c.sq = r / c.np;
         c.j = r - c.sq * c.np;
     }
@@ -520,10 +661,11 @@ attn_kernel(const __grid_constant__ Params p, const __grid_constant__ CUtensorMa
         if (last && !(seg_from0 && c.j == c.np - 1)) kind = (seg_no == 1) ? 1 : 2;
         if (page < 0 || page >= p.part[part].num_pages) {
             valid = 0;
-            if (lane == 0) { p.bad[c.u] = 1; flag_error(p.hdr, 4 /* SPD_ERR_BAD_PAGE */, c.u); }
+            if (lane == 0) { p.bad[c.u] = p.epoch; flag_error(p.hdr, 4 /* SPD_ERR_BAD_PAGE */, c.u); }
         }
         if (lane == 0) {
-            descs[stage] = make_int4(valid, (first ? 1 : 0) | (last ? 2 : 0) | (kind << 8), c.u, c.sq);
+            descs[2 * stage] = make_int4(valid, (first ? 1 : 0) | (last ? 2 : 0) | (kind << 8), c.u, c.sq);
+            descs[2 * stage + 1] = make_int4(c.np, c.j, t0 + issued, 0);
             const uint32_t bar = smem_u32(&bars[stage]);
             if (valid == 0) {
                 mbar_arrive(bar);
@@ -547,8 +689,7 @@ attn_kernel(const __grid_constant__ Params p, const __grid_constant__ CUtensorMa
             if (++c.sq == p.S) {
                 c.sq = 0;
                 if (issued < n) {
-                    do { ++c.u; } while (c.u < p.B - 1 && p.pfx[c.u + 1] == p.pfx[c.u]);
-                    cursor_load_user(c, p);
+                    do { ++c.u; cursor_load_user(c, p); } while (c.np == 0 && c.u < p.B - 1);
                 }
             } else {
                 c.key = -1;   // same user, page table starts over
@@ -564,20 +705,21 @@ attn_kernel(const __grid_constant__ Params p, const __grid_constant__ CUtensorMa
     for (; i < n; ++i) {
         const int stage = i % NS;
         if (!mbar_wait(smem_u32(&bars[stage]), (i / NS) & 1)) { dead = true; break; }
-        const int4 d = descs[stage];
+        const int4 d = descs[2 * stage];
         uint8_t *Ks = ring + static_cast<size_t>(stage) * 2 * TB, *Vs = Ks + TB;
         if (d.y & 1) { Math::begin(st, p, d.z, d.w, lane, extra); seg_bad = false; }
         if (d.x > 0) Math::tile(st, p, Ks, Vs, d.x, lane, extra);
         else seg_bad = true;
         if (d.y & 2) {
             // the stage just consumed doubles as the staging area of the epilogue
+            const int4 e = descs[2 * stage + 1];
             __syncwarp();
             float *So = reinterpret_cast<float *>(Ks);
             float *Sm = So + kHeadsPerItem * (D + 4), *Sl = Sm + kHeadsPerItem;
             Math::finish(st, So, Sm, Sl, lane);
             __syncwarp();
-            const bool bad = seg_bad || (p.bad[d.z] != 0);
-            segment_epilogue<D>(p, So, Sm, Sl, d.z, d.w, d.y >> 8, gwarp, lane, bad);
+            const bool bad = seg_bad || (__ldcg(p.bad + d.z) == p.epoch);
+            segment_epilogue<D>(p, So, Sm, Sl, d.z, d.w, d.y >> 8, gwarp, lane, bad, per, e.x, e.y, e.z);
             fence_proxy_async();
         }
         __syncwarp();
@@ -587,53 +729,6 @@ attn_kernel(const __grid_constant__ Params p, const __grid_constant__ CUtensorMa
         if (lane == 0) flag_error(p.hdr, 6 /* SPD_ERR_TIMEOUT */, -1);
         // give the copies still in flight a bounded chance to land before the warp leaves
         for (int k = i + 1; k < issued; ++k) mbar_wait(smem_u32(&bars[k % NS]), (k / NS) & 1);
-    }
-}
-
-// ------------------------------------------------------------------------------------------------
-// Second-level merge: one warp per sequence.  A sequence that one warp covered completely was
-// already finalised by the attention kernel; one cut across several warps is recombined here from
-// its pieces (M = max m_c; l = sum l_c e^{m_c - M}; O = sum O_c e^{m_c - M}); one that owns no tile
-// is an empty partition (O = 0, m = -inf, l = 0).
-template <int D>
-__global__ void __launch_bounds__(128) merge_kernel(Params p) {
-    constexpr int V = D / 32;
-    const int lane = threadIdx.x & 31;
-    const int seq = blockIdx.x * 4 + (threadIdx.x >> 5);
-    if (seq >= p.B * p.S) return;
-    const int u = seq / p.S, sq = seq - u * p.S;
-    const int np = p.np0[u] + p.np1[u];
-    const int per = p.hdr[HDR_TILES_PER_WARP];
-    const bool bad = p.bad[u] != 0;
-    const int kvh = sq / p.hgroups, hg = sq - kvh * p.hgroups;
-    const int hbase = kvh * p.g + hg * kHeadsPerItem;
-    int w_first = 0, w_last = -1;
-    int64_t s0 = 0;
-    if (np > 0) {
-        s0 = static_cast<int64_t>(p.pfx[u]) * p.S + static_cast<int64_t>(sq) * np;
-        w_first = static_cast<int>(s0 / per);
-        w_last = static_cast<int>((s0 + np - 1) / per);
-        if (w_first == w_last && !bad) return;   // complete: already written
-    }
-    for (int hh = 0; hh < p.geff; ++hh) {
-        float M = -INFINITY;
-        for (int w = w_first; w <= w_last; ++w) {
-            const int slot = 2 * w + ((static_cast<int64_t>(w) * per >= s0) ? 0 : 1);
-            M = fmaxf(M, p.scratch[static_cast<int64_t>(slot) * slot_floats(D) + kHeadsPerItem * D + hh]);
-        }
-        float o[V], l = 0.f;
-#pragma unroll
-        for (int i = 0; i < V; ++i) o[i] = 0.f;
-        for (int w = w_first; w <= w_last; ++w) {
-            const int slot = 2 * w + ((static_cast<int64_t>(w) * per >= s0) ? 0 : 1);
-            const float *src = p.scratch + static_cast<int64_t>(slot) * slot_floats(D);
-            const float mc = src[kHeadsPerItem * D + hh];
-            const float wgt = (mc == -INFINITY) ? 0.f : expf(mc - M);
-            l = fmaf(wgt, src[kHeadsPerItem * D + 8 + hh], l);
-#pragma unroll
-            for (int i = 0; i < V; ++i) o[i] = fmaf(wgt, src[hh * D + lane * V + i], o[i]);
-        }
-        finalize_store<D>(p, u, hbase + hh, o, M, l, lane, bad);
     }
 }
 
