@@ -281,7 +281,7 @@ def run_cuda(args):
 
     split = kernel_split(spd, w, shape, ws, out, steps)
     e2e_ms, h2d, d2h, outh = time_e2e(spd, w, shape, ws, min(steps, 500), warmup)
-    if not torch.equal(outh, out.cpu()):
+    if not torch.allclose(outh, out.cpu(), atol=2e-3, rtol=0):   # share sizes adapt, so rounding order may differ
         raise RuntimeError("host-buffer path and device path disagree")
     e2e_ms = max_over_ranks(e2e_ms, dev)
     e2e_val = replica_throughput(kvb, e2e_ms, world)

@@ -87,7 +87,7 @@ constexpr size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
 // Workspace layout.  The header, the per-user flags and the tickets come first so that the status
 // query can find them without knowing the shape.
 struct WsLayout {
-    size_t hdr, bad, tickets, scratch, partial_o, partial_m, partial_l, total;
+    size_t hdr, rates, bad, tickets, scratch, partial_o, partial_m, partial_l, total;
 };
 
 WsLayout ws_layout(const spd_shape &s, int sms) {
@@ -95,6 +95,7 @@ WsLayout ws_layout(const spd_shape &s, int sms) {
     size_t off = 0;
     const size_t B = s.batch;
     L.hdr = off;       off = align_up(off + HDR_WORDS * 4, 256);
+    L.rates = off;     off = align_up(off + 2 * kMaxGrid * sizeof(float2), 256);
     L.bad = off;       off = align_up(off + B * 4, 256);
     const int g = s.num_q_heads / s.num_kv_heads;
     const size_t seqs = B * s.num_kv_heads * (g > kHeadsPerItem ? g / kHeadsPerItem : 1);
@@ -156,7 +157,8 @@ spd_status make_map(CUtensorMap *map, const spd_shape &s, const void *pool, int6
 
 template <class Math>
 spd_status launch_attn(const Params &p, const CUtensorMap *maps, int sms, cudaStream_t st) {
-    constexpr size_t smem = attn_smem_bytes<Math>();
+    if (sms > kMaxGrid) return SPD_ERR_UNSUPPORTED;
+    const size_t smem = attn_smem_bytes<Math>(sms);
     static std::once_flag once[64];
     int dev = 0;
     cudaGetDevice(&dev);
@@ -210,6 +212,8 @@ spd_status run_job(const Job &job, void *ws, size_t ws_bytes, void *stream) {
     p.hdr = reinterpret_cast<int32_t *>(w + L.hdr);
     p.bad = reinterpret_cast<int32_t *>(w + L.bad);
     p.tickets = reinterpret_cast<int32_t *>(w + L.tickets);
+    p.rates = reinterpret_cast<float2 *>(w + L.rates);
+    p.rate_sel = static_cast<int32_t>(g_launches.load() & 1);   // launches alternate between the two halves
     p.epoch = job.epoch;
     p.scratch = reinterpret_cast<float *>(w + L.scratch);
     p.mode = job.mode;
@@ -416,7 +420,7 @@ spd_status spd_query_device_status(void *ws, void *cuda_stream, int32_t *first_b
     const size_t nbad = hdr[HDR_BATCH] > 0 ? align_up(static_cast<size_t>(hdr[HDR_BATCH]) * 4, 256) : 0;
     const size_t ntic = hdr[HDR_NSEQ] > 0 ? align_up(static_cast<size_t>(hdr[HDR_NSEQ]) * 4, 256) : 0;
     if (cudaMemsetAsync(ws, 0, 8, st) != cudaSuccess) return SPD_ERR_CUDA;
-    if (nbad + ntic && cudaMemsetAsync(static_cast<uint8_t *>(ws) + align_up(HDR_WORDS * 4, 256), 0, nbad + ntic, st) != cudaSuccess)
+    if (nbad + ntic && cudaMemsetAsync(static_cast<uint8_t *>(ws) + align_up(HDR_WORDS * 4, 256) + align_up(2 * kMaxGrid * sizeof(float2), 256), 0, nbad + ntic, st) != cudaSuccess)
         return SPD_ERR_CUDA;
     if (cudaStreamSynchronize(st) != cudaSuccess) return SPD_ERR_CUDA;
     return static_cast<spd_status>(hdr[HDR_STATUS]);

@@ -49,6 +49,8 @@ struct Params {
     int32_t *bad;           // [B] per-user flags: holds `epoch` if the user was flagged by this call
     int32_t *tickets;       // [B * S] pieces delivered so far per sequence; zero between calls
     int32_t epoch;          // non-zero id of this call
+    float2 *rates;          // [2][kMaxGrid] per-CTA (share weight, cycles) of earlier launches, double-buffered
+    int32_t rate_sel;       // which half this launch reads (it writes the other)
     float *scratch;         // [2 * num_warps][8 * D + 16]
     // outputs
     int32_t mode;           // OutMode

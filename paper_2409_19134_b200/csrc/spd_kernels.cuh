@@ -1,9 +1,10 @@
 // The kernel of the partitioned decode-attention path.
 //
 // One persistent launch does a whole call:
-//   plan    : every CTA derives the same plan from the inputs alone -- validated page-tile counts
-//             per user, their prefix sums, and the equal share of the flattened tile stream that
-//             each warp of the grid owns.
+//   plan    : every CTA derives the same plan from memory nobody writes during the call --
+//             validated page-tile counts per user, their prefix sums, and the share of the
+//             flattened tile stream that each warp of the grid owns (sized by the streaming rate
+//             each CTA showed on the previous call).
 //   stream  : each warp streams its share of (user, kv head) page tiles from HBM through a
 //             warp-private TMA ring in shared memory and keeps a running (O, m, l) per query head
 //             (Sec. 4.2: m = max score, l = sum exp(s - m)).
@@ -118,18 +119,28 @@ __device__ __forceinline__ int first_head(const Params &p, int sq) {
 }
 
 // Scratch slot that warp w used for its piece of the sequence starting at tile s0: the first slot
-// if the sequence contains the warp's first tile, else the second.
-__device__ __forceinline__ const float *piece_slot(const Params &p, int D, int w, int per, int64_t s0) {
-    const int which = (static_cast<int64_t>(w) * per >= s0) ? 0 : 1;
+// if the sequence contains the warp's first tile (bnd[w]), else the second.
+__device__ __forceinline__ const float *piece_slot(const Params &p, int D, int w, const int32_t *bnd, int s0) {
+    const int which = (bnd[w] >= s0) ? 0 : 1;
     return p.scratch + static_cast<int64_t>(2 * w + which) * slot_floats(D);
+}
+
+// The warp whose share [bnd[w], bnd[w+1]) holds tile t (shares may be empty; A = warps with a share).
+__device__ __forceinline__ int warp_of_tile(const int32_t *bnd, int A, int t) {
+    int lo = 0, hi = A;          // invariant: bnd[lo] <= t < bnd[hi]
+    while (hi - lo > 1) {
+        const int mid = (lo + hi) >> 1;
+        if (bnd[mid] <= t) lo = mid; else hi = mid;
+    }
+    return lo;
 }
 
 // Recombine the pieces that warps w_first..w_last left for one sequence (Theorem 1 applied n-ways,
 // every piece brought to the common maximum) and finalise it.  Run by the warp that delivered the
 // last piece.  Pieces are read past L1 (other SMs wrote them).  Lane c of a batch looks after piece c.
 template <int D>
-__device__ __noinline__ void merge_pieces(const Params &p, int u, int sq, int w_first, int w_last, int per,
-                                             int64_t s0, int lane, bool bad) {
+__device__ __noinline__ void merge_pieces(const Params &p, int u, int sq, int w_first, int w_last, const int32_t *bnd,
+                                          int s0, int lane, bool bad) {
     constexpr int V = D / 32, H = kHeadsPerItem;
     float M[H], L[H], o[H][V];
 #pragma unroll
@@ -141,8 +152,8 @@ __device__ __noinline__ void merge_pieces(const Params &p, int u, int sq, int w_
     }
     for (int b0 = w_first; b0 <= w_last; b0 += 32) {
         const int nb = min(32, w_last - b0 + 1);
-        const bool mine = lane < nb;
-        const float *ms = piece_slot(p, D, mine ? b0 + lane : b0, per, s0) + H * D;
+        const bool mine = lane < nb && bnd[b0 + lane + 1] > bnd[b0 + lane];   // warps with an empty share left nothing
+        const float *ms = piece_slot(p, D, mine ? b0 + lane : b0, bnd, s0) + H * D;
         float wgt[H];
 #pragma unroll
         for (int hh = 0; hh < H; ++hh) {
@@ -164,7 +175,8 @@ __device__ __noinline__ void merge_pieces(const Params &p, int u, int sq, int w_
             for (int i = 0; i < V; ++i) o[hh][i] *= resc;
         }
         for (int c = 0; c < nb; ++c) {
-            const float *src = piece_slot(p, D, b0 + c, per, s0) + lane * V;
+            if (bnd[b0 + c + 1] == bnd[b0 + c]) continue;
+            const float *src = piece_slot(p, D, b0 + c, bnd, s0) + lane * V;
 #pragma unroll
             for (int hh = 0; hh < H; ++hh) {
                 if (hh >= p.geff) break;
@@ -193,8 +205,8 @@ __device__ __noinline__ void merge_pieces(const Params &p, int u, int sq, int w_
 // j_last is the tile of the sequence this segment ended on, t_last its index in the tile stream.
 template <int D>
 __device__ __forceinline__ void segment_epilogue(const Params &p, const float *So, const float *Sm, const float *Sl,
-                                                 int u, int sq, int kind, int gwarp, int lane, bool bad, int per,
-                                                 int np, int j_last, int64_t t_last) {
+                                                 int u, int sq, int kind, int gwarp, int lane, bool bad,
+                                                 const int32_t *bnd, int A, int np, int j_last, int t_last) {
     constexpr int V = D / 32, PITCH = D + 4;
     if (kind == 0) {
         const int hbase = first_head(p, sq);
@@ -219,19 +231,23 @@ __device__ __forceinline__ void segment_epilogue(const Params &p, const float *S
         __stcg(dst + kHeadsPerItem * D + lane, Sm[lane]);
         __stcg(dst + kHeadsPerItem * D + 8 + lane, Sl[lane]);
     }
-    const int64_t s0 = t_last - j_last;
-    const int w_first = static_cast<int>(s0 / per), w_last = static_cast<int>((s0 + np - 1) / per);
+    const int s0 = t_last - j_last;
+    const int w_first = warp_of_tile(bnd, A, s0), w_last = warp_of_tile(bnd, A, s0 + np - 1);
+    int pieces = 0;
+    for (int w = w_first + lane; w <= w_last; w += 32) pieces += bnd[w + 1] > bnd[w] ? 1 : 0;
+#pragma unroll
+    for (int d = 16; d >= 1; d >>= 1) pieces += __shfl_xor_sync(0xffffffffu, pieces, d);
     __threadfence();     // this lane's part of the piece is visible before the ticket is drawn
     __syncwarp();
     int ticket = 0;
     int32_t *counter = p.tickets + static_cast<int64_t>(u) * p.S + sq;
     if (lane == 0) ticket = atomicAdd(counter, 1);
     ticket = __shfl_sync(0xffffffffu, ticket, 0);
-    if (ticket != w_last - w_first) return;   // other pieces are still to come
+    if (ticket != pieces - 1) return;         // other pieces are still to come
     __threadfence();
     if (lane == 0) *counter = 0;              // everybody has drawn: ready for the next call
     const bool any_bad = bad || (__ldcg(p.bad + u) == p.epoch);
-    merge_pieces<D>(p, u, sq, w_first, w_last, per, s0, lane, any_bad);
+    merge_pieces<D>(p, u, sq, w_first, w_last, bnd, s0, lane, any_bad);
 }
 
 // ------------------------------------------------------------------------------------------------
@@ -521,10 +537,16 @@ template <class Math>
 __host__ __device__ constexpr size_t attn_extra_offset() {
     return attn_desc_offset<Math>() + static_cast<size_t>(Math::kWarps) * Math::kStages * 32;
 }
+constexpr int kMaxGrid = 256;   // CTAs (one per SM) the share tables are sized for
 template <class Math>
-__host__ __device__ constexpr size_t attn_smem_bytes() {
-    return 1024 + static_cast<size_t>(Math::kWarps) * Math::kStages * 2 * Math::kTileBytes + attn_extra_offset<Math>() +
-           static_cast<size_t>(Math::kWarps) * Math::kExtraBytes;
+__host__ __device__ constexpr size_t attn_bnd_offset() {
+    return attn_extra_offset<Math>() + static_cast<size_t>(Math::kWarps) * Math::kExtraBytes;
+}
+// dynamic shared memory for a grid of `grid` CTAs: rings, barriers, descriptors, extras, share boundaries
+template <class Math>
+__host__ __device__ constexpr size_t attn_smem_bytes(int grid = 148) {
+    return 1024 + static_cast<size_t>(Math::kWarps) * Math::kStages * 2 * Math::kTileBytes + attn_bnd_offset<Math>() +
+           (static_cast<size_t>(grid) * Math::kWarps + 1) * 4 + 16;
 }
 
 template <class Math>
@@ -536,11 +558,15 @@ attn_kernel(const __grid_constant__ Params p, const __grid_constant__ CUtensorMa
     static_assert(TB % 1024 == 0, "swizzled tiles need 1024-byte aligned bases");
     static_assert(Math::kExtraBytes % 16 == 0, "per-warp extra area holds float4 data");
     static_assert(2 * TB >= (kHeadsPerItem * (D + 4) + 2 * kHeadsPerItem) * 4, "a stage must hold the epilogue staging");
-    static_assert(attn_smem_bytes<Math>() + 2048 <= 227 * 1024, "ring does not fit shared memory");
+    static_assert(attn_smem_bytes<Math>(kMaxGrid) + 8192 <= 227 * 1024, "ring does not fit shared memory");
     static_assert(Math::kWarps <= 16 && Math::kStages >= 2, "CTA shape");
     extern __shared__ uint8_t smem_raw[];
     __shared__ int32_t chunk_pfx[NT + 1];
     __shared__ int32_t warp_tot[Math::kWarps];
+    __shared__ float sh_w[kMaxGrid], sh_r[kMaxGrid], sh_norm[2];
+    __shared__ int32_t sh_wq[kMaxGrid], sh_pc[kMaxGrid + 1];
+    __shared__ long long cta_clock0;
+    __shared__ int32_t cta_exits;
     uint8_t *base = reinterpret_cast<uint8_t *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
     const int wid = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int gwarp = blockIdx.x * Math::kWarps + wid;
@@ -582,8 +608,55 @@ attn_kernel(const __grid_constant__ Params p, const __grid_constant__ CUtensorMa
         if (T64 >= (1ll << 31)) flag_error(p.hdr, 2 /* SPD_ERR_UNSUPPORTED */, -1);   // 32-bit tile counter
     }
     const int T = T64 >= (1ll << 31) ? 0 : static_cast<int>(T64);
-    int per = (T + p.num_warps - 1) / p.num_warps;
-    if (per < kMinTilesPerWarp) per = kMinTilesPerWarp;
+
+    // ---- shares: warp w of the grid owns tiles [bnd[w], bnd[w+1]) ------------------------------
+    // CTAs do not all stream at the same rate (some SMs sit behind busier ports), so shares are
+    // sized by the rates measured on the previous call that used this workspace: each CTA left its
+    // (weight, cycles) in one half of a double-buffered table; this call reads that half and writes
+    // the other, so every CTA sees the same numbers however late it starts.
+    const int G = gridDim.x;
+    const float2 *rate_rd = p.rates + (p.rate_sel & 1) * kMaxGrid;
+    float2 *rate_wr = p.rates + ((p.rate_sel + 1) & 1) * kMaxGrid;
+    if (threadIdx.x == 0) { cta_clock0 = clock64(); cta_exits = 0; }
+    for (int i = threadIdx.x; i < G; i += NT) {
+        const float2 v = __ldcg(rate_rd + i);
+        sh_w[i] = v.x;
+        sh_r[i] = (v.x > 0.f && v.y > 0.f) ? v.x / v.y : 0.f;
+    }
+    __syncthreads();
+    if (threadIdx.x == 0) {          // serial, so that every CTA rounds alike
+        float sw = 0.f, sr = 0.f;
+        bool ok = true;
+        for (int i = 0; i < G; ++i) { sw += sh_w[i]; sr += sh_r[i]; ok = ok && sh_r[i] > 0.f; }
+        sh_norm[0] = ok ? G / sw : 0.f;
+        sh_norm[1] = ok ? G / sr : 0.f;
+    }
+    __syncthreads();
+    for (int i = threadIdx.x; i < G; i += NT) {
+        // 1/4 of the weight used last time + 3/4 of the rate it achieved, both relative to the mean
+        const float m = sh_norm[0] > 0.f ? 0.25f * sh_w[i] * sh_norm[0] + 0.75f * sh_r[i] * sh_norm[1] : 1.f;
+        const int q = static_cast<int>(m * 1024.f + 0.5f);
+        sh_wq[i] = q < 512 ? 512 : (q > 2048 ? 2048 : q);
+    }
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        int acc = 0;
+        for (int i = 0; i < G; ++i) { sh_pc[i] = acc; acc += sh_wq[i]; }
+        sh_pc[G] = acc;
+    }
+    __syncthreads();
+    int32_t *bnd = reinterpret_cast<int32_t *>(tail + attn_bnd_offset<Math>());
+    int A = (T + kMinTilesPerWarp - 1) / kMinTilesPerWarp;     // warps that get a share
+    if (A > p.num_warps) A = p.num_warps;
+    {
+        auto wsum = [&](int w) {     // weights of warps < w; a CTA's warps all carry the CTA's weight
+            const int c = w / Math::kWarps;
+            return static_cast<int64_t>(Math::kWarps) * sh_pc[c] + static_cast<int64_t>(w - c * Math::kWarps) * (c < G ? sh_wq[c] : 0);
+        };
+        const int64_t total = A > 0 ? wsum(A) : 1;
+        for (int w = threadIdx.x; w <= A; w += NT) bnd[w] = static_cast<int32_t>(static_cast<int64_t>(T) * wsum(w) / total);
+    }
+    __syncthreads();
 
     // ---- users that own no tile (nothing cached, or flagged): their outputs are written here ----
     for (int u = gwarp; u < p.B; u += p.num_warps) {
@@ -602,11 +675,9 @@ attn_kernel(const __grid_constant__ Params p, const __grid_constant__ CUtensorMa
         }
     }
 
-    const int64_t t0l = static_cast<int64_t>(gwarp) * per;
-    if (t0l >= T) return;
-    const int t0 = static_cast<int>(t0l);
-    const int t1 = static_cast<int>(t0l + per < T ? t0l + per : T);
-    const int n = t1 - t0;
+    const int t0 = gwarp < A ? bnd[gwarp] : 0;
+    const int n = gwarp < A ? bnd[gwarp + 1] - t0 : 0;
+    if (n > 0) {
 
     if (lane == 0) {
         for (int s = 0; s < NS; ++s) mbar_init(smem_u32(&bars[s]), 1);
@@ -719,7 +790,7 @@ attn_kernel(const __grid_constant__ Params p, const __grid_constant__ CUtensorMa
             Math::finish(st, So, Sm, Sl, lane);
             __syncwarp();
             const bool bad = seg_bad || (__ldcg(p.bad + d.z) == p.epoch);
-            segment_epilogue<D>(p, So, Sm, Sl, d.z, d.w, d.y >> 8, gwarp, lane, bad, per, e.x, e.y, e.z);
+            segment_epilogue<D>(p, So, Sm, Sl, d.z, d.w, d.y >> 8, gwarp, lane, bad, bnd, A, e.x, e.y, e.z);
             fence_proxy_async();
         }
         __syncwarp();
@@ -729,6 +800,19 @@ attn_kernel(const __grid_constant__ Params p, const __grid_constant__ CUtensorMa
         if (lane == 0) flag_error(p.hdr, 6 /* SPD_ERR_TIMEOUT */, -1);
         // give the copies still in flight a bounded chance to land before the warp leaves
         for (int k = i + 1; k < issued; ++k) mbar_wait(smem_u32(&bars[k % NS]), (k / NS) & 1);
+    }
+
+    }   // n > 0
+
+    // ---- the CTA's last warp out leaves (weight, cycles) for the next call's shares -------------
+    __syncwarp();
+    if (lane == 0 && atomicAdd(&cta_exits, 1) == Math::kWarps - 1) {
+        const int wa = blockIdx.x * Math::kWarps, wb = wa + Math::kWarps;
+        const int tiles = (wb <= A ? bnd[wb] : T) - (wa <= A ? bnd[wa] : T);
+        float2 v = __ldcg(rate_rd + blockIdx.x);                   // a call too small to tell keeps the old entry
+        if (tiles >= 32 * Math::kWarps)
+            v = make_float2(static_cast<float>(sh_wq[blockIdx.x]), static_cast<float>(clock64() - cta_clock0));
+        __stcg(rate_wr + blockIdx.x, v);
     }
 }
 
