@@ -137,14 +137,15 @@ __device__ __forceinline__ int warp_of_tile(const int32_t *bnd, int A, int t) {
 
 // Recombine the pieces that warps w_first..w_last left for one sequence (Theorem 1 applied n-ways,
 // every piece brought to the common maximum) and finalise it.  Run by the warp that delivered the
-// last piece.  Pieces are read past L1 (other SMs wrote them).  Lane c of a batch looks after piece c.
-template <int D>
+// last piece.  Pieces are read past L1 (other SMs wrote them).  Lane c of a batch looks after the
+// (m, l) of piece c; the O rows are fetched 16 at a time so that the loads overlap.
+template <int D, int GE>
 __device__ __noinline__ void merge_pieces(const Params &p, int u, int sq, int w_first, int w_last, const int32_t *bnd,
                                           int s0, int lane, bool bad) {
-    constexpr int V = D / 32, H = kHeadsPerItem;
-    float M[H], L[H], o[H][V];
+    constexpr int V = D / 32, H = kHeadsPerItem, PB = 16 / GE;   // PB pieces per batch of loads
+    float M[GE], L[GE], o[GE][V];
 #pragma unroll
-    for (int hh = 0; hh < H; ++hh) {
+    for (int hh = 0; hh < GE; ++hh) {
         M[hh] = -INFINITY;
         L[hh] = 0.f;
 #pragma unroll
@@ -154,10 +155,9 @@ __device__ __noinline__ void merge_pieces(const Params &p, int u, int sq, int w_
         const int nb = min(32, w_last - b0 + 1);
         const bool mine = lane < nb && bnd[b0 + lane + 1] > bnd[b0 + lane];   // warps with an empty share left nothing
         const float *ms = piece_slot(p, D, mine ? b0 + lane : b0, bnd, s0) + H * D;
-        float wgt[H];
+        float wgt[GE];
 #pragma unroll
-        for (int hh = 0; hh < H; ++hh) {
-            if (hh >= p.geff) break;
+        for (int hh = 0; hh < GE; ++hh) {
             const float mc = mine ? __ldcg(ms + hh) : -INFINITY;
             const float lc = mine ? __ldcg(ms + H + hh) : 0.f;
             float mb = mc;
@@ -174,50 +174,62 @@ __device__ __noinline__ void merge_pieces(const Params &p, int u, int sq, int w_
 #pragma unroll
             for (int i = 0; i < V; ++i) o[hh][i] *= resc;
         }
-        for (int c = 0; c < nb; ++c) {
-            if (bnd[b0 + c + 1] == bnd[b0 + c]) continue;
-            const float *src = piece_slot(p, D, b0 + c, bnd, s0) + lane * V;
+        for (int c0 = 0; c0 < nb; c0 += PB) {
+            float x[PB][GE][V];
 #pragma unroll
-            for (int hh = 0; hh < H; ++hh) {
-                if (hh >= p.geff) break;
-                const float wc = __shfl_sync(0xffffffffu, wgt[hh], c);
-                if constexpr (V == 4) {
-                    const float4 x = __ldcg(reinterpret_cast<const float4 *>(src + hh * D));
-                    o[hh][0] = fmaf(wc, x.x, o[hh][0]); o[hh][1] = fmaf(wc, x.y, o[hh][1]);
-                    o[hh][2] = fmaf(wc, x.z, o[hh][2]); o[hh][3] = fmaf(wc, x.w, o[hh][3]);
-                } else {
-                    const float2 x = __ldcg(reinterpret_cast<const float2 *>(src + hh * D));
-                    o[hh][0] = fmaf(wc, x.x, o[hh][0]); o[hh][1] = fmaf(wc, x.y, o[hh][1]);
+            for (int k = 0; k < PB; ++k) {
+                const int c = c0 + k;
+                const bool live = c < nb && bnd[b0 + c + 1] > bnd[b0 + c];
+                const float *src = piece_slot(p, D, live ? b0 + c : b0, bnd, s0) + lane * V;
+#pragma unroll
+                for (int hh = 0; hh < GE; ++hh) {
+                    if constexpr (V == 4) {
+                        const float4 t = live ? __ldcg(reinterpret_cast<const float4 *>(src + hh * D)) : make_float4(0.f, 0.f, 0.f, 0.f);
+                        x[k][hh][0] = t.x; x[k][hh][1] = t.y; x[k][hh][2] = t.z; x[k][hh][3] = t.w;
+                    } else {
+                        const float2 t = live ? __ldcg(reinterpret_cast<const float2 *>(src + hh * D)) : make_float2(0.f, 0.f);
+                        x[k][hh][0] = t.x; x[k][hh][1] = t.y;
+                    }
+                }
+            }
+#pragma unroll
+            for (int k = 0; k < PB; ++k) {
+                const int c = (c0 + k) & 31;
+#pragma unroll
+                for (int hh = 0; hh < GE; ++hh) {
+                    const float wc = __shfl_sync(0xffffffffu, wgt[hh], c);   // a piece that is not live has weight 0
+#pragma unroll
+                    for (int i = 0; i < V; ++i) o[hh][i] = fmaf(wc, x[k][hh][i], o[hh][i]);
                 }
             }
         }
     }
     const int hbase = first_head(p, sq);
 #pragma unroll
-    for (int hh = 0; hh < H; ++hh)
-        if (hh < p.geff) finalize_store<D>(p, u, hbase + hh, o[hh], M[hh], L[hh], lane, bad);
+    for (int hh = 0; hh < GE; ++hh) finalize_store<D>(p, u, hbase + hh, o[hh], M[hh], L[hh], lane, bad);
 }
 
-// A finished segment sits in shared memory as So[8][D+4], Sm[8], Sl[8].
-//   kind 0  : the segment is a whole sequence -> finalise it here.
-//   kind 1/2: a piece -> scratch slot 2w / 2w+1, then a ticket on the sequence; the warp that draws
-//             the last ticket merges all pieces (and puts the ticket counter back to zero).
-// j_last is the tile of the sequence this segment ended on, t_last its index in the tile stream.
+// A finished segment sits in shared memory as So[8][D+4], Sm[8], Sl[8].  A segment that is a whole
+// sequence is finalised on the spot (the warp has seen every page of it, so `bad` is complete).
 template <int D>
-__device__ __forceinline__ void segment_epilogue(const Params &p, const float *So, const float *Sm, const float *Sl,
-                                                 int u, int sq, int kind, int gwarp, int lane, bool bad,
-                                                 const int32_t *bnd, int A, int np, int j_last, int t_last) {
+__device__ __forceinline__ void finalize_segment(const Params &p, const float *So, const float *Sm, const float *Sl,
+                                                 int u, int sq, int lane, bool bad) {
     constexpr int V = D / 32, PITCH = D + 4;
-    if (kind == 0) {
-        const int hbase = first_head(p, sq);
-        for (int hh = 0; hh < p.geff; ++hh) {
-            float o[V];
+    const int hbase = first_head(p, sq);
+    for (int hh = 0; hh < p.geff; ++hh) {
+        float o[V];
 #pragma unroll
-            for (int i = 0; i < V; ++i) o[i] = So[hh * PITCH + lane * V + i];
-            finalize_store<D>(p, u, hbase + hh, o, Sm[hh], Sl[hh], lane, bad);
-        }
-        return;
+        for (int i = 0; i < V; ++i) o[i] = So[hh * PITCH + lane * V + i];
+        finalize_store<D>(p, u, hbase + hh, o, Sm[hh], Sl[hh], lane, bad);
     }
+}
+
+// A segment that is only a piece of its sequence goes to scratch slot 2w (kind 1) or 2w+1 (kind 2).
+// The stores are fire-and-forget; piece_ticket fences them before it draws the ticket.
+template <int D>
+__device__ __forceinline__ void piece_store(const Params &p, const float *So, const float *Sm, const float *Sl,
+                                            int kind, int gwarp, int lane) {
+    constexpr int V = D / 32, PITCH = D + 4;
     float *dst = p.scratch + static_cast<int64_t>(2 * gwarp + (kind - 1)) * slot_floats(D);
 #pragma unroll
     for (int hh = 0; hh < kHeadsPerItem; ++hh) {
@@ -231,8 +243,20 @@ __device__ __forceinline__ void segment_epilogue(const Params &p, const float *S
         __stcg(dst + kHeadsPerItem * D + lane, Sm[lane]);
         __stcg(dst + kHeadsPerItem * D + 8 + lane, Sl[lane]);
     }
-    const int s0 = t_last - j_last;
-    const int w_first = warp_of_tile(bnd, A, s0), w_last = warp_of_tile(bnd, A, s0 + np - 1);
+}
+
+// A piece of a sequence: whose it is, the sequence's tile count and first tile, and whether a
+// page of the piece was out of range.
+struct PieceInfo {
+    int u, sq, np, s0;
+    bool bad;
+};
+
+// Draw the ticket of a piece already stored; the warp that draws the last ticket of a sequence
+// merges all its pieces (and puts the counter back to zero for the next call).
+template <int D>
+__device__ __forceinline__ void piece_ticket(const Params &p, const PieceInfo &pp, const int32_t *bnd, int A, int lane) {
+    const int w_first = warp_of_tile(bnd, A, pp.s0), w_last = warp_of_tile(bnd, A, pp.s0 + pp.np - 1);
     int pieces = 0;
     for (int w = w_first + lane; w <= w_last; w += 32) pieces += bnd[w + 1] > bnd[w] ? 1 : 0;
 #pragma unroll
@@ -240,14 +264,19 @@ __device__ __forceinline__ void segment_epilogue(const Params &p, const float *S
     __threadfence();     // this lane's part of the piece is visible before the ticket is drawn
     __syncwarp();
     int ticket = 0;
-    int32_t *counter = p.tickets + static_cast<int64_t>(u) * p.S + sq;
+    int32_t *counter = p.tickets + static_cast<int64_t>(pp.u) * p.S + pp.sq;
     if (lane == 0) ticket = atomicAdd(counter, 1);
     ticket = __shfl_sync(0xffffffffu, ticket, 0);
     if (ticket != pieces - 1) return;         // other pieces are still to come
     __threadfence();
     if (lane == 0) *counter = 0;              // everybody has drawn: ready for the next call
-    const bool any_bad = bad || (__ldcg(p.bad + u) == p.epoch);
-    merge_pieces<D>(p, u, sq, w_first, w_last, bnd, s0, lane, any_bad);
+    const bool bad = pp.bad || (__ldcg(p.bad + pp.u) == p.epoch);
+    switch (p.geff) {
+        case 1: merge_pieces<D, 1>(p, pp.u, pp.sq, w_first, w_last, bnd, pp.s0, lane, bad); break;
+        case 2: merge_pieces<D, 2>(p, pp.u, pp.sq, w_first, w_last, bnd, pp.s0, lane, bad); break;
+        case 4: merge_pieces<D, 4>(p, pp.u, pp.sq, w_first, w_last, bnd, pp.s0, lane, bad); break;
+        default: merge_pieces<D, 8>(p, pp.u, pp.sq, w_first, w_last, bnd, pp.s0, lane, bad); break;
+    }
 }
 
 // ------------------------------------------------------------------------------------------------
@@ -395,7 +424,7 @@ struct MathF32 {
     static constexpr int kBoxBytes = kTileBytes;
     static constexpr int kBoxCols = D;
     static constexpr int kWarps = 4;
-    static constexpr int kStages = 3;
+    static constexpr int kStages = D == 128 ? 2 : 3;   // 16 KB per stage at head_dim 128
     static constexpr int kExtraBytes = (kHeadsPerItem * D + kHeadsPerItem * kPage) * 4;  // q, P
     static constexpr int V = D / 32;
 
@@ -508,9 +537,22 @@ struct Cursor {
     int key;               // (partition << 24 | batch) that idx_cur holds, -1 = nothing
 };
 
-__device__ __forceinline__ void cursor_load_user(Cursor &c, const Params &p) {
+constexpr int kUserCache = 1024;   // users whose validated tile counts a CTA keeps in shared memory
+
+// Tile counts of user u: from the CTA's cache when it holds them, else recomputed from the inputs.
+__device__ __forceinline__ void cached_tiles(const Params &p, const int2 *cache, int u, int &n0, int &n1) {
+    if (u < kUserCache) {
+        const int2 v = cache[u];
+        n0 = v.x;
+        n1 = v.y;
+    } else {
+        user_tiles(p, u, n0, n1);
+    }
+}
+
+__device__ __forceinline__ void cursor_load_user(Cursor &c, const Params &p, const int2 *cache) {
     int n0, n1;
-    user_tiles(p, c.u, n0, n1);
+    cached_tiles(p, cache, c.u, n0, n1);
     c.npp = n0;
     c.np = n0 + n1;
     c.base0 = p.part[0].present ? p.part[0].indptr[c.u] : 0;
@@ -558,13 +600,14 @@ attn_kernel(const __grid_constant__ Params p, const __grid_constant__ CUtensorMa
     static_assert(TB % 1024 == 0, "swizzled tiles need 1024-byte aligned bases");
     static_assert(Math::kExtraBytes % 16 == 0, "per-warp extra area holds float4 data");
     static_assert(2 * TB >= (kHeadsPerItem * (D + 4) + 2 * kHeadsPerItem) * 4, "a stage must hold the epilogue staging");
-    static_assert(attn_smem_bytes<Math>(kMaxGrid) + 8192 <= 227 * 1024, "ring does not fit shared memory");
+    static_assert(attn_smem_bytes<Math>(kMaxGrid) + 16384 <= 227 * 1024, "ring does not fit shared memory");
     static_assert(Math::kWarps <= 16 && Math::kStages >= 2, "CTA shape");
     extern __shared__ uint8_t smem_raw[];
     __shared__ int32_t chunk_pfx[NT + 1];
     __shared__ int32_t warp_tot[Math::kWarps];
-    __shared__ float sh_w[kMaxGrid], sh_r[kMaxGrid], sh_norm[2];
+    __shared__ float sh_w[kMaxGrid], sh_r[kMaxGrid];
     __shared__ int32_t sh_wq[kMaxGrid], sh_pc[kMaxGrid + 1];
+    __shared__ int2 sh_np[kUserCache];
     __shared__ long long cta_clock0;
     __shared__ int32_t cta_exits;
     uint8_t *base = reinterpret_cast<uint8_t *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
@@ -579,12 +622,22 @@ attn_kernel(const __grid_constant__ Params p, const __grid_constant__ CUtensorMa
     // ---- plan: every CTA computes the same thing from the inputs alone -------------------------
     // Thread t sums the tiles of users [t*C, (t+1)*C); a block scan gives chunk prefixes.
     const int C = (p.B + NT - 1) / NT;
+    const int G = gridDim.x;
+    const float2 *rate_rd = p.rates + (p.rate_sel & 1) * kMaxGrid;
+    float2 *rate_wr = p.rates + ((p.rate_sel + 1) & 1) * kMaxGrid;
     {
+        if (threadIdx.x == 0) { cta_clock0 = clock64(); cta_exits = 0; }
+        for (int i = threadIdx.x; i < G; i += NT) {     // the rate table travels together with the lengths
+            const float2 v = __ldcg(rate_rd + i);
+            sh_w[i] = v.x;
+            sh_r[i] = (v.x > 0.f && v.y > 0.f) ? v.x / v.y : 0.f;
+        }
         int sum = 0;
         const int ub = threadIdx.x * C, ue = min(p.B, ub + C);
         for (int u = ub; u < ue; ++u) {
             int n0, n1;
             user_tiles(p, u, n0, n1);
+            if (u < kUserCache) sh_np[u] = make_int2(n0, n1);
             sum += n0 + n1;
         }
         int inc = sum;
@@ -614,35 +667,37 @@ attn_kernel(const __grid_constant__ Params p, const __grid_constant__ CUtensorMa
     // sized by the rates measured on the previous call that used this workspace: each CTA left its
     // (weight, cycles) in one half of a double-buffered table; this call reads that half and writes
     // the other, so every CTA sees the same numbers however late it starts.
-    const int G = gridDim.x;
-    const float2 *rate_rd = p.rates + (p.rate_sel & 1) * kMaxGrid;
-    float2 *rate_wr = p.rates + ((p.rate_sel + 1) & 1) * kMaxGrid;
-    if (threadIdx.x == 0) { cta_clock0 = clock64(); cta_exits = 0; }
-    for (int i = threadIdx.x; i < G; i += NT) {
-        const float2 v = __ldcg(rate_rd + i);
-        sh_w[i] = v.x;
-        sh_r[i] = (v.x > 0.f && v.y > 0.f) ? v.x / v.y : 0.f;
-    }
-    __syncthreads();
-    if (threadIdx.x == 0) {          // serial, so that every CTA rounds alike
+    if (wid == 0) {                  // one fixed reduction tree, so that every CTA rounds alike
         float sw = 0.f, sr = 0.f;
         bool ok = true;
-        for (int i = 0; i < G; ++i) { sw += sh_w[i]; sr += sh_r[i]; ok = ok && sh_r[i] > 0.f; }
-        sh_norm[0] = ok ? G / sw : 0.f;
-        sh_norm[1] = ok ? G / sr : 0.f;
-    }
-    __syncthreads();
-    for (int i = threadIdx.x; i < G; i += NT) {
-        // 1/4 of the weight used last time + 3/4 of the rate it achieved, both relative to the mean
-        const float m = sh_norm[0] > 0.f ? 0.25f * sh_w[i] * sh_norm[0] + 0.75f * sh_r[i] * sh_norm[1] : 1.f;
-        const int q = static_cast<int>(m * 1024.f + 0.5f);
-        sh_wq[i] = q < 512 ? 512 : (q > 2048 ? 2048 : q);
-    }
-    __syncthreads();
-    if (threadIdx.x == 0) {
-        int acc = 0;
-        for (int i = 0; i < G; ++i) { sh_pc[i] = acc; acc += sh_wq[i]; }
-        sh_pc[G] = acc;
+        for (int i = lane; i < G; i += 32) { sw += sh_w[i]; sr += sh_r[i]; ok = ok && sh_r[i] > 0.f; }
+#pragma unroll
+        for (int d = 16; d >= 1; d >>= 1) {
+            sw += __shfl_xor_sync(0xffffffffu, sw, d);
+            sr += __shfl_xor_sync(0xffffffffu, sr, d);
+        }
+        ok = __all_sync(0xffffffffu, ok);
+        const float nw = ok ? G / sw : 0.f, nr = ok ? G / sr : 0.f;
+        // weight of CTA i: 1/4 of the weight it had last time + 3/4 of the rate it achieved, both
+        // relative to the mean; lane l looks after CTAs [l*cpl, (l+1)*cpl)
+        const int cpl = (G + 31) / 32;
+        int mysum = 0;
+        for (int i = lane * cpl; i < min(G, (lane + 1) * cpl); ++i) {
+            const float m = ok ? 0.25f * sh_w[i] * nw + 0.75f * sh_r[i] * nr : 1.f;
+            int q = static_cast<int>(m * 1024.f + 0.5f);
+            q = q < 512 ? 512 : (q > 2048 ? 2048 : q);
+            sh_wq[i] = q;
+            mysum += q;
+        }
+        int inc = mysum;
+#pragma unroll
+        for (int d = 1; d < 32; d <<= 1) {
+            const int t = __shfl_up_sync(0xffffffffu, inc, d);
+            if (lane >= d) inc += t;
+        }
+        int acc = inc - mysum;
+        for (int i = lane * cpl; i < min(G, (lane + 1) * cpl); ++i) { sh_pc[i] = acc; acc += sh_wq[i]; }
+        if (lane == 31) sh_pc[G] = inc;
     }
     __syncthreads();
     int32_t *bnd = reinterpret_cast<int32_t *>(tail + attn_bnd_offset<Math>());
@@ -661,7 +716,7 @@ attn_kernel(const __grid_constant__ Params p, const __grid_constant__ CUtensorMa
     // ---- users that own no tile (nothing cached, or flagged): their outputs are written here ----
     for (int u = gwarp; u < p.B; u += p.num_warps) {
         int n0, n1;
-        user_tiles(p, u, n0, n1);
+        cached_tiles(p, sh_np, u, n0, n1);
         if (n0 + n1 != 0) continue;
         const bool bad = __ldcg(p.bad + u) == p.epoch;
         for (int sq = 0; sq < p.S; ++sq) {
@@ -685,33 +740,54 @@ attn_kernel(const __grid_constant__ Params p, const __grid_constant__ CUtensorMa
     }
     __syncwarp();
 
-    // locate the first tile: the user u with S * pfx[u] <= t0 < S * pfx[u + 1]
-    Cursor c;
-    {
-        const int x = t0 / p.S;   // in units of tiles per sequence
+    // Where tile t sits: its user (the u with S * pfx[u] <= t < S * pfx[u + 1]), the tiles per
+    // sequence of that user, the sequence and the tile within it.
+    auto seq_of_tile = [&](int t, int &u, int &np, int &sq, int &jt) {
+        const int x = t / p.S;    // in units of tiles per sequence
         int lo = 0, hi = NT;      // invariant: chunk_pfx[lo] <= x < chunk_pfx[hi]
         while (hi - lo > 1) {
             const int mid = (lo + hi) >> 1;
             if (chunk_pfx[mid] <= x) lo = mid; else hi = mid;
         }
-        int acc = chunk_pfx[lo], u = lo * C, n0 = 0, n1 = 0;
-        for (;; ++u) {            // ends inside the chunk, because the chunk holds tile x
-            user_tiles(p, u, n0, n1);
+        int acc = chunk_pfx[lo], n0 = 0, n1 = 0;
+        for (u = lo * C;; ++u) {  // ends inside the chunk, because the chunk holds tile x
+            cached_tiles(p, sh_np, u, n0, n1);
             if (acc + n0 + n1 > x) break;
             acc += n0 + n1;
         }
-        c.u = u;
-        cursor_load_user(c, p);
-        const int r = t0 - acc * p.S;
-        c.sq = r / c.np;
-        c.j = r - c.sq * c.np;
+        np = n0 + n1;
+        const int r = t - acc * p.S;
+        sq = r / np;
+        jt = r - sq * np;
+    };
+    Cursor c;
+    auto seek = [&](int t) {
+        int np;
+        seq_of_tile(t, c.u, np, c.sq, c.j);
+        cursor_load_user(c, p, sh_np);
+    };
+
+    // Order of work.  A share usually ends inside a sequence; that trailing piece needs a ticket
+    // (a fence and an atomic, perhaps a merge: round trips to memory).  Done last they would be
+    // exposed at the end of the kernel, done first the other warps cover them.  So the warp
+    // streams [tb, t1) -- its trailing piece -- first and [t0, tb) afterwards.
+    const int t1 = t0 + n;
+    int tb = t0;
+    {
+        int u, np, sq, jt;
+        seq_of_tile(t1 - 1, u, np, sq, jt);
+        if (jt != np - 1 && t1 - 1 - jt > t0) tb = t1 - 1 - jt;
     }
+    const int n2 = tb == t0 ? n : t1 - tb;   // tiles streamed before the jump back to t0
+    seek(tb);
+    int cur_t = tb;            // index in the tile stream of the next tile to issue
 
     int issued = 0;            // tiles handed to the TMA so far
     bool seg_from0 = false;    // the segment being issued began at the start of its sequence
-    int seg_no = 0;            // segments begun so far by this warp
+    bool seg_has_t0 = false;   // ... and holds the share's first tile
 
     auto issue = [&](int stage) {
+        if (issued == n2 && n2 < n) { seek(t0); cur_t = t0; }
         // page of tile (c.u, c.sq, c.j)
         const int part = c.j >= c.npp ? 1 : 0;
         const int jj = part ? c.j - c.npp : c.j;
@@ -725,18 +801,18 @@ attn_kernel(const __grid_constant__ Params p, const __grid_constant__ CUtensorMa
         const int npart = part ? c.np - c.npp : c.npp;
         int valid = kPage;
         if (jj == npart - 1) valid = (part ? c.len1 : c.len0) - jj * kPage;
-        const bool first = (c.j == 0) || (issued == 0);
-        const bool last = (c.j == c.np - 1) || (issued == n - 1);
-        if (first) { seg_from0 = (c.j == 0); ++seg_no; }
+        const bool first = (c.j == 0) || (cur_t == t0);
+        const bool last = (c.j == c.np - 1) || (cur_t == t1 - 1);
+        if (first) { seg_from0 = (c.j == 0); seg_has_t0 = (cur_t == t0); }
         int kind = 0;
-        if (last && !(seg_from0 && c.j == c.np - 1)) kind = (seg_no == 1) ? 1 : 2;
+        if (last && !(seg_from0 && c.j == c.np - 1)) kind = seg_has_t0 ? 1 : 2;
         if (page < 0 || page >= p.part[part].num_pages) {
             valid = 0;
             if (lane == 0) { p.bad[c.u] = p.epoch; flag_error(p.hdr, 4 /* SPD_ERR_BAD_PAGE */, c.u); }
         }
         if (lane == 0) {
             descs[2 * stage] = make_int4(valid, (first ? 1 : 0) | (last ? 2 : 0) | (kind << 8), c.u, c.sq);
-            descs[2 * stage + 1] = make_int4(c.np, c.j, t0 + issued, 0);
+            descs[2 * stage + 1] = make_int4(c.np, c.j, cur_t, 0);
             const uint32_t bar = smem_u32(&bars[stage]);
             if (valid == 0) {
                 mbar_arrive(bar);
@@ -754,14 +830,13 @@ attn_kernel(const __grid_constant__ Params p, const __grid_constant__ CUtensorMa
             }
         }
         ++issued;
-        // advance to the next tile (skipping users that own no tile)
-        if (++c.j == c.np) {
+        ++cur_t;
+        // advance to the next tile (skipping users that own no tile), unless the range ends here
+        if (issued != n && issued != n2 && ++c.j == c.np) {
             c.j = 0;
             if (++c.sq == p.S) {
                 c.sq = 0;
-                if (issued < n) {
-                    do { ++c.u; cursor_load_user(c, p); } while (c.np == 0 && c.u < p.B - 1);
-                }
+                do { ++c.u; cursor_load_user(c, p, sh_np); } while (c.np == 0 && c.u < p.B - 1);
             } else {
                 c.key = -1;   // same user, page table starts over
             }
@@ -789,8 +864,14 @@ attn_kernel(const __grid_constant__ Params p, const __grid_constant__ CUtensorMa
             float *Sm = So + kHeadsPerItem * (D + 4), *Sl = Sm + kHeadsPerItem;
             Math::finish(st, So, Sm, Sl, lane);
             __syncwarp();
-            const bool bad = seg_bad || (__ldcg(p.bad + d.z) == p.epoch);
-            segment_epilogue<D>(p, So, Sm, Sl, d.z, d.w, d.y >> 8, gwarp, lane, bad, bnd, A, e.x, e.y, e.z);
+            const int kind = d.y >> 8;
+            if (kind == 0) {
+                finalize_segment<D>(p, So, Sm, Sl, d.z, d.w, lane, seg_bad);
+            } else {
+                piece_store<D>(p, So, Sm, Sl, kind, gwarp, lane);
+                const PieceInfo pp{d.z, d.w, e.x, e.z - e.y, seg_bad};
+                piece_ticket<D>(p, pp, bnd, A, lane);
+            }
             fence_proxy_async();
         }
         __syncwarp();
