@@ -5,7 +5,7 @@
 
 Prints ONE JSON line.  `value` is decode-attention KV GB/s (bytes of cached K and V rows divided by
 time) of spd_decode_step (fused) with every input resident in HBM; `e2e` is the same metric through
-spd_decode_step_host, whose per-step inputs (q, page tables, lengths) start in pinned host memory and
+spd_decode_step_host, whose per-step inputs (q, page tables, lengths) start in one pinned host buffer and
 whose output is read back inside the timed region.  The KV pools are the resident cache in both.
 
 With N > 1 (torchrun) every rank runs an independent replica on its own GPU (the path has no exchange
@@ -226,16 +226,18 @@ def kernel_split(spd, w, shape, ws, out, steps):
 
 
 def time_e2e(spd, w, shape, ws, steps, warmup):
-    """Per step: q, page tables and lengths from pinned host memory in, output back out."""
+    """Per step: q, page tables and lengths go in from one pinned host blob, the output comes back."""
     dev = w.q.device
-    pin = lambda t: t.cpu().pin_memory()
-    qh = pin(w.q)
-    tabs = [(pin(p.page_indptr), pin(p.page_indices), pin(p.seq_lens)) for p in (w.priv, w.pub)]
-    outh = torch.empty((w.batch, w.num_q_heads, w.head_dim), dtype=torch.float32).pin_memory()
-    n_in, n_out = int(tabs[0][1].numel()), int(tabs[1][1].numel())
-    staging = torch.empty(spd.spd_host_staging_size(shape, n_in, n_out, torch.float32), dtype=torch.uint8, device=dev)
+    lay = spd.spd_step_blob_layout(shape, int(w.priv.page_indices.numel()), int(w.pub.page_indices.numel()), torch.float32)
+    host = torch.zeros(lay.total_bytes, dtype=torch.uint8).pin_memory()
+    spd.fill_step_blob(lay, host, w.q, w.priv, w.pub)
+    devb = torch.empty(lay.total_bytes, dtype=torch.uint8, device=dev)
     pools = [(w.priv.k_pool, w.priv.v_pool), (w.pub.k_pool, w.pub.v_pool)]
-    call = lambda: spd.spd_decode_step_host(shape, qh, pools[0], tabs[0], pools[1], tabs[1], outh, staging, ws)
+
+    def call():
+        code, bad = spd.spd_decode_step_host(shape, lay, host, devb, pools[0], pools[1], torch.float32, ws)
+        if code != spd.SPD_OK:
+            raise RuntimeError(f"host-buffer step failed: status {code}, user {bad}")
     for _ in range(warmup):
         call()
     torch.cuda.synchronize()
@@ -245,9 +247,10 @@ def time_e2e(spd, w, shape, ws, steps, warmup):
         call()
     e1.record()
     torch.cuda.synchronize()
-    h2d = qh.numel() * qh.element_size() + sum(t.numel() * 4 for tab in tabs for t in tab)
-    d2h = outh.numel() * 4 + 32
-    return e0.elapsed_time(e1) / steps, h2d, d2h, outh
+    d2h = lay.total_bytes - lay.out + 32
+    n_out = w.batch * w.num_q_heads * w.head_dim
+    outh = host[lay.out:lay.out + 4 * n_out].view(torch.float32).reshape(w.batch, w.num_q_heads, w.head_dim).clone()
+    return e0.elapsed_time(e1) / steps, lay.in_bytes, d2h, outh
 
 
 def run_cuda(args):

@@ -116,19 +116,35 @@ spd_status spd_decode_step(const spd_shape *shape, const void *q, const spd_page
                            void *ws, size_t ws_bytes, void *cuda_stream);
 
 /*
- * spd_decode_step for a caller whose per-step data lives in HOST memory: q, both partitions'
- * page_indptr / page_indices / seq_lens and `out` are host pointers (pinned memory makes the
- * copies asynchronous); only k_pool / v_pool inside `priv` and `pub` are device pointers (the KV
- * cache stays resident).  The call copies the host inputs into `staging` (device memory of at
- * least spd_host_staging_size() bytes), runs the fused step, copies `out` back and waits for
- * the stream.  Returns the device status as spd_query_device_status() would.
+ * spd_decode_step (fused) for a caller whose per-step data lives in HOST memory (no counterpart in
+ * the paper, whose two processes exchange these arrays through the host on every layer).
+ *
+ * Everything that changes from step to step -- q, both partitions' page_indptr / seq_lens /
+ * page_indices -- sits in ONE host buffer (pinned memory makes the copy asynchronous) at the offsets
+ * that spd_step_blob_layout() reports, so that a step costs one host-to-device copy, one kernel and
+ * two device-to-host copies (the output, the status words).  The KV pools stay resident on the
+ * device: `priv_pools` and `pub_pools` carry k_pool, v_pool and num_pages only (their table pointers
+ * are ignored).  `device_blob` is device memory of layout->total_bytes, 256-byte aligned.
+ *
+ * The call copies host_blob[0, in_bytes) to the device, runs the step, copies the output to
+ * host_blob + layout->out, waits for the stream and returns the device status as
+ * spd_query_device_status() would (*first_bad_user likewise; may be NULL).
  */
-spd_status spd_host_staging_size(const spd_shape *shape, int64_t priv_pages_listed,
-                                 int64_t pub_pages_listed, spd_dtype out_dtype, size_t *bytes);
-spd_status spd_decode_step_host(const spd_shape *shape, const void *q_host, const spd_paged_kv *priv,
-                                const spd_paged_kv *pub, void *out_host, spd_dtype out_dtype,
-                                void *staging, size_t staging_bytes,
-                                void *ws, size_t ws_bytes, void *cuda_stream);
+typedef struct {
+    int64_t priv_pages_listed, pub_pages_listed;   /* entries of the two page_indices arrays */
+    size_t  q;                                      /* [batch][num_q_heads][head_dim], shape dtype */
+    size_t  priv_indptr, priv_lens, priv_indices;   /* int32 [batch+1], [batch], [priv_pages_listed] */
+    size_t  pub_indptr, pub_lens, pub_indices;
+    size_t  in_bytes;                               /* the inputs occupy [0, in_bytes) */
+    size_t  out;                                    /* [batch][num_q_heads][head_dim], out_dtype */
+    size_t  total_bytes;
+} spd_step_blob;
+spd_status spd_step_blob_layout(const spd_shape *shape, int64_t priv_pages_listed, int64_t pub_pages_listed,
+                                spd_dtype out_dtype, spd_step_blob *layout);
+spd_status spd_decode_step_host(const spd_shape *shape, const spd_step_blob *layout, void *host_blob,
+                                void *device_blob, const spd_paged_kv *priv_pools,
+                                const spd_paged_kv *pub_pools, spd_dtype out_dtype,
+                                int32_t *first_bad_user, void *ws, size_t ws_bytes, void *cuda_stream);
 
 /*
  * Waits for `cuda_stream`, then reads and clears the workspace's sticky status.  Returns SPD_OK,

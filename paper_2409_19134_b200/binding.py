@@ -19,7 +19,7 @@ _STATUS_NAMES = {0: "SPD_OK", 1: "SPD_ERR_INVALID_ARG", 2: "SPD_ERR_UNSUPPORTED"
                  4: "SPD_ERR_BAD_PAGE", 5: "SPD_ERR_CUDA", 6: "SPD_ERR_TIMEOUT"}
 
 EXPORTS = ["spd_workspace_size", "spd_partial_attn", "spd_service_attn_merge", "spd_decode_step",
-           "spd_host_staging_size", "spd_decode_step_host", "spd_query_device_status",
+           "spd_step_blob_layout", "spd_decode_step_host", "spd_query_device_status",
            "spd_kernel_launch_count", "spd_status_string", "spd_profile_begin", "spd_profile_end",
            "spd_decode_step_static"]
 
@@ -38,6 +38,13 @@ class Shape(C.Structure):
 class PagedKV(C.Structure):
     _fields_ = [("k_pool", C.c_void_p), ("v_pool", C.c_void_p), ("num_pages", C.c_int32),
                 ("page_indptr", C.c_void_p), ("page_indices", C.c_void_p), ("seq_lens", C.c_void_p)]
+
+
+class StepBlob(C.Structure):
+    _fields_ = [("priv_pages_listed", C.c_int64), ("pub_pages_listed", C.c_int64), ("q", C.c_size_t),
+                ("priv_indptr", C.c_size_t), ("priv_lens", C.c_size_t), ("priv_indices", C.c_size_t),
+                ("pub_indptr", C.c_size_t), ("pub_lens", C.c_size_t), ("pub_indices", C.c_size_t),
+                ("in_bytes", C.c_size_t), ("out", C.c_size_t), ("total_bytes", C.c_size_t)]
 
 
 class Partial(C.Structure):
@@ -60,9 +67,9 @@ def lib() -> C.CDLL:
         L.spd_service_attn_merge.argtypes = [C.POINTER(Shape), vp, C.POINTER(PagedKV), Partial, vp, C.c_int, vp, sz, vp]
         L.spd_decode_step.argtypes = [C.POINTER(Shape), vp, C.POINTER(PagedKV), C.POINTER(PagedKV), vp, C.c_int,
                                       C.c_int32, vp, sz, vp]
-        L.spd_host_staging_size.argtypes = [C.POINTER(Shape), C.c_int64, C.c_int64, C.c_int, C.POINTER(sz)]
-        L.spd_decode_step_host.argtypes = [C.POINTER(Shape), vp, C.POINTER(PagedKV), C.POINTER(PagedKV), vp, C.c_int,
-                                           vp, sz, vp, sz, vp]
+        L.spd_step_blob_layout.argtypes = [C.POINTER(Shape), C.c_int64, C.c_int64, C.c_int, C.POINTER(StepBlob)]
+        L.spd_decode_step_host.argtypes = [C.POINTER(Shape), C.POINTER(StepBlob), vp, vp, C.POINTER(PagedKV),
+                                           C.POINTER(PagedKV), C.c_int, C.POINTER(C.c_int32), vp, sz, vp]
         L.spd_query_device_status.argtypes = [vp, vp, C.POINTER(C.c_int32)]
         L.spd_kernel_launch_count.restype = C.c_int64
         L.spd_status_string.restype = C.c_char_p
@@ -157,26 +164,41 @@ def spd_decode_step(shape, q, priv, pub, out, ws, fused=True, stream=None) -> No
                                  _stream_ptr(stream)), "spd_decode_step")
 
 
-def spd_host_staging_size(shape, priv_pages_listed: int, pub_pages_listed: int, out_dtype) -> int:
-    n = C.c_size_t(0)
-    _check(lib().spd_host_staging_size(C.byref(shape), priv_pages_listed, pub_pages_listed,
-                                       _dtype_code(out_dtype), C.byref(n)), "spd_host_staging_size")
-    return int(n.value)
+def spd_step_blob_layout(shape, priv_pages_listed: int, pub_pages_listed: int, out_dtype) -> StepBlob:
+    lay = StepBlob()
+    _check(lib().spd_step_blob_layout(C.byref(shape), priv_pages_listed, pub_pages_listed,
+                                      _dtype_code(out_dtype), C.byref(lay)), "spd_step_blob_layout")
+    return lay
 
 
-def spd_decode_step_host(shape, q_host, priv_pools, priv_tables, pub_pools, pub_tables, out_host, staging, ws,
-                         stream=None) -> None:
-    """q_host / *_tables (indptr, indices, lens) / out_host are HOST tensors (pinned for async copies);
-    *_pools are (k_pool, v_pool) device tensors."""
-    def kv(pools, tables):
-        indptr, indices, lens = tables
-        return PagedKV(_ptr(pools[0]), _ptr(pools[1]), int(pools[0].shape[0]), indptr.data_ptr(),
-                       _ptr(indices), lens.data_ptr())
-    a, b = kv(priv_pools, priv_tables), kv(pub_pools, pub_tables)
-    _check(lib().spd_decode_step_host(C.byref(shape), q_host.data_ptr(), C.byref(a), C.byref(b),
-                                      out_host.data_ptr(), _dtype_code(out_host.dtype), staging.data_ptr(),
-                                      staging.numel(), ws.data_ptr(), ws.numel(), _stream_ptr(stream)),
-           "spd_decode_step_host")
+def spd_decode_step_host(shape, layout, host_blob, device_blob, priv_pools, pub_pools, out_dtype, ws,
+                         stream=None) -> Tuple[int, int]:
+    """host_blob: pinned uint8 host tensor laid out per `layout`; device_blob: uint8 device tensor of
+    layout.total_bytes; *_pools: (k_pool, v_pool) device tensors.  Waits for the stream; the output is
+    then at host_blob[layout.out:].  Returns (device status, first flagged user or -1)."""
+    def kv(pools):
+        return PagedKV(_ptr(pools[0]), _ptr(pools[1]), int(pools[0].shape[0]), None, None, None)
+    a, b = kv(priv_pools), kv(pub_pools)
+    bad = C.c_int32(-1)
+    code = lib().spd_decode_step_host(C.byref(shape), C.byref(layout), host_blob.data_ptr(), device_blob.data_ptr(),
+                                      C.byref(a), C.byref(b), _dtype_code(out_dtype), C.byref(bad), ws.data_ptr(),
+                                      ws.numel(), _stream_ptr(stream))
+    if code not in (SPD_OK, 4, 6):
+        raise SpdError(code, "spd_decode_step_host")
+    return int(code), int(bad.value)
+
+
+def fill_step_blob(layout, host_blob, q, priv, pub) -> None:
+    """Copy q and the two partitions' tables (any device) into a host blob at the layout's offsets."""
+    def put(off, t):
+        src = t.detach().cpu().contiguous().view(torch.uint8).reshape(-1)
+        host_blob[off:off + src.numel()] = src
+    put(layout.q, q)
+    for part, (a, b, c) in ((priv, (layout.priv_indptr, layout.priv_lens, layout.priv_indices)),
+                            (pub, (layout.pub_indptr, layout.pub_lens, layout.pub_indices))):
+        put(a, part.page_indptr)
+        put(b, part.seq_lens)
+        put(c, part.page_indices)
 
 
 def spd_query_device_status(ws, stream=None) -> Tuple[int, int]:

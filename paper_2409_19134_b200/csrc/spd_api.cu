@@ -351,60 +351,65 @@ spd_status spd_decode_step(const spd_shape *shape, const void *q, const spd_page
     return run_job(b, ws, ws_bytes, cuda_stream);
 }
 
-spd_status spd_host_staging_size(const spd_shape *shape, int64_t priv_pages_listed, int64_t pub_pages_listed,
-                                 spd_dtype out_dtype, size_t *bytes) {
+spd_status spd_step_blob_layout(const spd_shape *shape, int64_t priv_pages_listed, int64_t pub_pages_listed,
+                                spd_dtype out_dtype, spd_step_blob *layout) {
     spd_status rc = check_shape(shape);
     if (rc != SPD_OK) return rc;
-    if (!bytes || priv_pages_listed < 0 || pub_pages_listed < 0) return SPD_ERR_INVALID_ARG;
+    if (!layout || priv_pages_listed < 0 || pub_pages_listed < 0) return SPD_ERR_INVALID_ARG;
+    if (out_dtype != SPD_F32 && out_dtype != SPD_BF16) return SPD_ERR_UNSUPPORTED;
     const size_t B = shape->batch, rows = B * shape->num_q_heads * shape->head_dim;
     const size_t es = shape->dtype == SPD_BF16 ? 2 : 4, oes = out_dtype == SPD_BF16 ? 2 : 4;
-    size_t off = align_up(rows * es, 256);
-    off += 2 * (align_up((B + 1) * 4, 256) + align_up(B * 4, 256));
-    off += align_up(static_cast<size_t>(priv_pages_listed) * 4, 256) + align_up(static_cast<size_t>(pub_pages_listed) * 4, 256);
-    off += align_up(rows * oes, 256) + 256;
-    *bytes = off;
+    size_t off = 0;
+    auto take = [&](size_t bytes) { const size_t at = off; off = align_up(off + bytes, 256); return at; };
+    layout->priv_pages_listed = priv_pages_listed;
+    layout->pub_pages_listed = pub_pages_listed;
+    layout->q = take(rows * es);
+    layout->priv_indptr = take((B + 1) * 4);
+    layout->priv_lens = take(B * 4);
+    layout->priv_indices = take(static_cast<size_t>(priv_pages_listed) * 4);
+    layout->pub_indptr = take((B + 1) * 4);
+    layout->pub_lens = take(B * 4);
+    layout->pub_indices = take(static_cast<size_t>(pub_pages_listed) * 4);
+    layout->in_bytes = off;
+    layout->out = take(rows * oes);
+    layout->total_bytes = off;
     return SPD_OK;
 }
 
-spd_status spd_decode_step_host(const spd_shape *shape, const void *q_host, const spd_paged_kv *priv,
-                                const spd_paged_kv *pub, void *out_host, spd_dtype out_dtype, void *staging,
-                                size_t staging_bytes, void *ws, size_t ws_bytes, void *cuda_stream) {
+spd_status spd_decode_step_host(const spd_shape *shape, const spd_step_blob *layout, void *host_blob,
+                                void *device_blob, const spd_paged_kv *priv_pools, const spd_paged_kv *pub_pools,
+                                spd_dtype out_dtype, int32_t *first_bad_user, void *ws, size_t ws_bytes,
+                                void *cuda_stream) {
     spd_status rc = check_shape(shape);
     if (rc != SPD_OK) return rc;
-    if (!q_host || !priv || !pub || !out_host || !staging || misaligned(staging, 256)) return SPD_ERR_INVALID_ARG;
-    if (!priv->page_indptr || !pub->page_indptr || !priv->seq_lens || !pub->seq_lens) return SPD_ERR_INVALID_ARG;
-    const size_t B = shape->batch, rows = B * shape->num_q_heads * shape->head_dim;
-    const size_t es = shape->dtype == SPD_BF16 ? 2 : 4, oes = out_dtype == SPD_BF16 ? 2 : 4;
-    const int64_t n_in = priv->page_indptr[B], n_out = pub->page_indptr[B];   // host reads
-    size_t need = 0;
-    if ((rc = spd_host_staging_size(shape, n_in < 0 ? 0 : n_in, n_out < 0 ? 0 : n_out, out_dtype, &need)) != SPD_OK) return rc;
-    if (n_in < 0 || n_out < 0) return SPD_ERR_INVALID_ARG;
-    if (staging_bytes < need) return SPD_ERR_WORKSPACE;
-    if ((n_in > 0 && !priv->page_indices) || (n_out > 0 && !pub->page_indices)) return SPD_ERR_INVALID_ARG;
+    if (!layout || !host_blob || !device_blob || !priv_pools || !pub_pools || !ws) return SPD_ERR_INVALID_ARG;
+    if (misaligned(device_blob, 256) || misaligned(host_blob, 16)) return SPD_ERR_INVALID_ARG;
+    spd_step_blob want;
+    if ((rc = spd_step_blob_layout(shape, layout->priv_pages_listed, layout->pub_pages_listed, out_dtype, &want)) != SPD_OK)
+        return rc;
+    if (memcmp(&want, layout, sizeof want) != 0) return SPD_ERR_INVALID_ARG;   // not a layout this library made
+    const size_t B = shape->batch;
+    const uint8_t *hb = static_cast<const uint8_t *>(host_blob);
+    // the tables in the blob must fit the blob: their last prefix entry is the number of pages listed
+    if (reinterpret_cast<const int32_t *>(hb + layout->priv_indptr)[B] > layout->priv_pages_listed ||
+        reinterpret_cast<const int32_t *>(hb + layout->pub_indptr)[B] > layout->pub_pages_listed)
+        return SPD_ERR_INVALID_ARG;
     cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
-    uint8_t *base = static_cast<uint8_t *>(staging);
-    size_t off = 0;
-    bool ok = true;
-    auto push = [&](const void *src, size_t bytes) -> void * {
-        void *dst = base + off;
-        if (bytes) ok = ok && cudaMemcpyAsync(dst, src, bytes, cudaMemcpyHostToDevice, st) == cudaSuccess;
-        off = align_up(off + bytes, 256);
-        return dst;
-    };
-    const void *dq = push(q_host, rows * es);
-    spd_paged_kv dpriv = *priv, dpub = *pub;
-    dpriv.page_indptr = static_cast<const int32_t *>(push(priv->page_indptr, (B + 1) * 4));
-    dpriv.seq_lens = static_cast<const int32_t *>(push(priv->seq_lens, B * 4));
-    dpriv.page_indices = static_cast<const int32_t *>(push(priv->page_indices, static_cast<size_t>(n_in) * 4));
-    dpub.page_indptr = static_cast<const int32_t *>(push(pub->page_indptr, (B + 1) * 4));
-    dpub.seq_lens = static_cast<const int32_t *>(push(pub->seq_lens, B * 4));
-    dpub.page_indices = static_cast<const int32_t *>(push(pub->page_indices, static_cast<size_t>(n_out) * 4));
-    void *dout = base + off;
-    if (!ok) return SPD_ERR_CUDA;
-    rc = spd_decode_step(shape, dq, &dpriv, &dpub, dout, out_dtype, 1, ws, ws_bytes, cuda_stream);
+    uint8_t *db = static_cast<uint8_t *>(device_blob);
+    if (cudaMemcpyAsync(db, hb, layout->in_bytes, cudaMemcpyHostToDevice, st) != cudaSuccess) return SPD_ERR_CUDA;
+    spd_paged_kv a = *priv_pools, b = *pub_pools;
+    a.page_indptr = reinterpret_cast<const int32_t *>(db + layout->priv_indptr);
+    a.seq_lens = reinterpret_cast<const int32_t *>(db + layout->priv_lens);
+    a.page_indices = reinterpret_cast<const int32_t *>(db + layout->priv_indices);
+    b.page_indptr = reinterpret_cast<const int32_t *>(db + layout->pub_indptr);
+    b.seq_lens = reinterpret_cast<const int32_t *>(db + layout->pub_lens);
+    b.page_indices = reinterpret_cast<const int32_t *>(db + layout->pub_indices);
+    rc = spd_decode_step(shape, db + layout->q, &a, &b, db + layout->out, out_dtype, 1, ws, ws_bytes, cuda_stream);
     if (rc != SPD_OK) return rc;
-    if (cudaMemcpyAsync(out_host, dout, rows * oes, cudaMemcpyDeviceToHost, st) != cudaSuccess) return SPD_ERR_CUDA;
-    return spd_query_device_status(ws, cuda_stream, nullptr);
+    if (cudaMemcpyAsync(static_cast<uint8_t *>(host_blob) + layout->out, db + layout->out, layout->total_bytes - layout->out,
+                        cudaMemcpyDeviceToHost, st) != cudaSuccess)
+        return SPD_ERR_CUDA;
+    return spd_query_device_status(ws, cuda_stream, first_bad_user);
 }
 
 spd_status spd_query_device_status(void *ws, void *cuda_stream, int32_t *first_bad_user) {

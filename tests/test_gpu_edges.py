@@ -141,3 +141,38 @@ def test_full_size_sampled_outputs(name):
             ref.append(orc.full(q1, parts[0], parts[1], w.sm_scale)[0, 0])
             got.append(out[u, h].cpu().numpy())
     assert_close(np.stack(got), np.stack(ref), w.dtype, f"{name} sampled")
+
+
+@pytest.mark.parametrize("name", ["bf16_gqa4_d128", "f32_mha_d64"])
+def test_host_blob_step_matches_oracle(name):
+    """The end-to-end entry point: per-step inputs in one host buffer, output read back from it."""
+    w = wl.make_workload(dict(SMALL[name], name=name), slack=True)
+    q, kin, kout = oracle_inputs(w)
+    ref = orc.full(q, kin, kout, w.sm_scale)
+    shape = spd.make_shape(w.batch, w.num_q_heads, w.num_kv_heads, w.head_dim, w.dtype, w.sm_scale)
+    ws = spd.alloc_workspace(shape)
+    lay = spd.spd_step_blob_layout(shape, int(w.priv.page_indices.numel()), int(w.pub.page_indices.numel()), torch.float32)
+    host = torch.zeros(lay.total_bytes, dtype=torch.uint8).pin_memory()
+    spd.fill_step_blob(lay, host, w.q, w.priv, w.pub)
+    devb = torch.empty(lay.total_bytes, dtype=torch.uint8, device="cuda")
+    pools = [(p.k_pool.cuda(), p.v_pool.cuda()) for p in (w.priv, w.pub)]
+    n = w.batch * w.num_q_heads * w.head_dim
+    for _ in range(2):
+        host[lay.out:] = 0xFF
+        assert spd.spd_decode_step_host(shape, lay, host, devb, pools[0], pools[1], torch.float32, ws) == (spd.SPD_OK, -1)
+        out = host[lay.out:lay.out + 4 * n].view(torch.float32).reshape(w.batch, w.num_q_heads, w.head_dim)
+        assert_close(out.numpy(), ref, w.dtype, f"{name} host blob")
+    # a page index outside the pool, planted in the host blob: reported, contained, cleared
+    idx = host[lay.priv_indices:lay.priv_indices + 4 * w.priv.page_indices.numel()].view(torch.int32)
+    keep = int(idx[int(w.priv.page_indptr[1])])
+    idx[int(w.priv.page_indptr[1])] = w.priv.num_pages + 3
+    assert spd.spd_decode_step_host(shape, lay, host, devb, pools[0], pools[1], torch.float32, ws) == (4, 1)
+    out = host[lay.out:lay.out + 4 * n].view(torch.float32).reshape(w.batch, w.num_q_heads, w.head_dim)
+    assert bool((out[1] == 0).all())
+    idx[int(w.priv.page_indptr[1])] = keep
+    assert spd.spd_decode_step_host(shape, lay, host, devb, pools[0], pools[1], torch.float32, ws) == (spd.SPD_OK, -1)
+    # a table that claims more pages than the blob holds is refused on the host
+    ip = host[lay.priv_indptr:lay.priv_indptr + 4 * (w.batch + 1)].view(torch.int32)
+    ip[w.batch] += 1
+    with pytest.raises(spd.SpdError):
+        spd.spd_decode_step_host(shape, lay, host, devb, pools[0], pools[1], torch.float32, ws)
