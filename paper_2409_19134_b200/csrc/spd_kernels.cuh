@@ -782,6 +782,7 @@ attn_kernel(const __grid_constant__ Params p, const __grid_constant__ CUtensorMa
     seek(tb);
     int cur_t = tb;            // index in the tile stream of the next tile to issue
 
+    const uint64_t stream_policy = l2_evict_first_policy();
     int issued = 0;            // tiles handed to the TMA so far
     bool seg_from0 = false;    // the segment being issued began at the start of its sequence
     bool seg_has_t0 = false;   // ... and holds the share's first tile
@@ -824,8 +825,8 @@ attn_kernel(const __grid_constant__ Params p, const __grid_constant__ CUtensorMa
                 mbar_expect_tx(bar, 2 * TB);
 #pragma unroll
                 for (int b = 0; b < Math::kBoxes; ++b) {
-                    tma_load_2d(kdst + b * Math::kBoxBytes, mk, b * Math::kBoxCols, row, bar);
-                    tma_load_2d(vdst + b * Math::kBoxBytes, mv, b * Math::kBoxCols, row, bar);
+                    tma_load_2d(kdst + b * Math::kBoxBytes, mk, b * Math::kBoxCols, row, bar, stream_policy);
+                    tma_load_2d(vdst + b * Math::kBoxBytes, mv, b * Math::kBoxCols, row, bar, stream_policy);
                 }
             }
         }
