@@ -4,6 +4,7 @@
 
 #include <atomic>
 #include <cstdio>
+#include <cstdlib>
 #include <cstring>
 #include <mutex>
 #include <vector>
@@ -95,7 +96,7 @@ WsLayout ws_layout(const spd_shape &s, int sms) {
     size_t off = 0;
     const size_t B = s.batch;
     L.hdr = off;       off = align_up(off + HDR_WORDS * 4, 256);
-    L.rates = off;     off = align_up(off + 2 * kMaxGrid * sizeof(float2), 256);
+    L.rates = off;     off = align_up(off + 3 * kMaxGrid * sizeof(float2), 256);
     L.bad = off;       off = align_up(off + B * 4, 256);
     const int g = s.num_q_heads / s.num_kv_heads;
     const size_t seqs = B * s.num_kv_heads * (g > kHeadsPerItem ? g / kHeadsPerItem : 1);
@@ -168,9 +169,23 @@ spd_status launch_attn(const Params &p, const CUtensorMap *maps, int sms, cudaSt
                                         static_cast<int>(smem));
     });
     if (attr_err != cudaSuccess) return SPD_ERR_CUDA;
-    attn_kernel<Math><<<sms, Math::kWarps * 32, smem, st>>>(p, maps[0], maps[1], maps[2], maps[3]);
+    // Programmatic stream serialisation: this kernel's read-only preamble may overlap the tail of the
+    // previous kernel on the stream if that kernel allows it (this library's kernels do).  Setting
+    // SPD_NO_PDL in the environment launches with plain stream order.
+    static const bool pdl = getenv("SPD_NO_PDL") == nullptr;
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(sms);
+    cfg.blockDim = dim3(Math::kWarps * 32);
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = st;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = pdl ? 1 : 0;
+    const cudaError_t err = cudaLaunchKernelEx(&cfg, attn_kernel<Math>, p, maps[0], maps[1], maps[2], maps[3]);
     ++g_launches;
-    return cudaGetLastError() == cudaSuccess ? SPD_OK : SPD_ERR_CUDA;
+    return err == cudaSuccess ? SPD_OK : SPD_ERR_CUDA;
 }
 
 // What one library call boils down to: one launch of the attention kernel.
@@ -213,7 +228,7 @@ spd_status run_job(const Job &job, void *ws, size_t ws_bytes, void *stream) {
     p.bad = reinterpret_cast<int32_t *>(w + L.bad);
     p.tickets = reinterpret_cast<int32_t *>(w + L.tickets);
     p.rates = reinterpret_cast<float2 *>(w + L.rates);
-    p.rate_sel = static_cast<int32_t>(g_launches.load() & 1);   // launches alternate between the two halves
+    p.rate_sel = static_cast<int32_t>(g_launches.load() % 3);   // launches rotate through the three thirds
     p.epoch = job.epoch;
     p.scratch = reinterpret_cast<float *>(w + L.scratch);
     p.mode = job.mode;
@@ -425,7 +440,7 @@ spd_status spd_query_device_status(void *ws, void *cuda_stream, int32_t *first_b
     const size_t nbad = hdr[HDR_BATCH] > 0 ? align_up(static_cast<size_t>(hdr[HDR_BATCH]) * 4, 256) : 0;
     const size_t ntic = hdr[HDR_NSEQ] > 0 ? align_up(static_cast<size_t>(hdr[HDR_NSEQ]) * 4, 256) : 0;
     if (cudaMemsetAsync(ws, 0, 8, st) != cudaSuccess) return SPD_ERR_CUDA;
-    if (nbad + ntic && cudaMemsetAsync(static_cast<uint8_t *>(ws) + align_up(HDR_WORDS * 4, 256) + align_up(2 * kMaxGrid * sizeof(float2), 256), 0, nbad + ntic, st) != cudaSuccess)
+    if (nbad + ntic && cudaMemsetAsync(static_cast<uint8_t *>(ws) + align_up(HDR_WORDS * 4, 256) + align_up(3 * kMaxGrid * sizeof(float2), 256), 0, nbad + ntic, st) != cudaSuccess)
         return SPD_ERR_CUDA;
     if (cudaStreamSynchronize(st) != cudaSuccess) return SPD_ERR_CUDA;
     return static_cast<spd_status>(hdr[HDR_STATUS]);

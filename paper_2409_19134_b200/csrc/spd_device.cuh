@@ -49,8 +49,8 @@ struct Params {
     int32_t *bad;           // [B] per-user flags: holds `epoch` if the user was flagged by this call
     int32_t *tickets;       // [B * S] pieces delivered so far per sequence; zero between calls
     int32_t epoch;          // non-zero id of this call
-    float2 *rates;          // [2][kMaxGrid] per-CTA (share weight, cycles) of earlier launches, double-buffered
-    int32_t rate_sel;       // which half this launch reads (it writes the other)
+    float2 *rates;          // [3][kMaxGrid] per-CTA (share weight, cycles) of earlier launches
+    int32_t rate_sel;       // launch counter: this launch writes third rate_sel % 3, reads (rate_sel + 1) % 3
     float *scratch;         // [2 * num_warps][8 * D + 16]
     // outputs
     int32_t mode;           // OutMode
@@ -137,6 +137,12 @@ __device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
     __nv_bfloat162 v = __floats2bfloat162_rn(lo, hi);
     return *reinterpret_cast<uint32_t *>(&v);
 }
+
+// Programmatic dependent launch: let the next kernel on the stream start its own read-only preamble
+// early, and wait until the previous kernel on the stream has completed and its writes are visible.
+// Both are no-ops when the launch did not ask for programmatic serialisation.
+__device__ __forceinline__ void griddep_launch_dependents() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+__device__ __forceinline__ void griddep_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
 
 // Raise the sticky status and remember the lowest flagged user.
 __device__ __forceinline__ void flag_error(int32_t *hdr, int code, int user) {

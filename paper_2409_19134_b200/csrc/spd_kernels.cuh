@@ -34,9 +34,11 @@ constexpr float kLog2e = 1.4426950408889634f;
 
 // ------------------------------------------------------------------------------------------------
 // Validated page-tile counts of one user (private, public).  A pure function of the call's inputs,
-// so every CTA that evaluates it agrees.  A user whose tables are inconsistent owns no tile, is
-// flagged for this call, and gets zeros.
-__device__ __forceinline__ void user_tiles(const Params &p, int u, int &n0, int &n1) {
+// so every CTA that evaluates it agrees.  A user whose tables are inconsistent owns no tile and
+// gets zeros; with Flag the user is also flagged for this call (a write to the workspace, so only
+// done once the previous kernel on the stream has finished with it).
+template <bool Flag = false>
+__device__ __forceinline__ bool user_tiles(const Params &p, int u, int &n0, int &n1) {
     n0 = n1 = 0;
     bool bad = false;
 #pragma unroll
@@ -55,9 +57,12 @@ __device__ __forceinline__ void user_tiles(const Params &p, int u, int &n0, int 
     }
     if (bad) {
         n0 = n1 = 0;
-        p.bad[u] = p.epoch;
-        flag_error(p.hdr, 4 /* SPD_ERR_BAD_PAGE */, u);
+        if (Flag) {
+            p.bad[u] = p.epoch;
+            flag_error(p.hdr, 4 /* SPD_ERR_BAD_PAGE */, u);
+        }
     }
+    return bad;
 }
 
 // ------------------------------------------------------------------------------------------------
@@ -619,14 +624,17 @@ attn_kernel(const __grid_constant__ Params p, const __grid_constant__ CUtensorMa
     int4 *descs = reinterpret_cast<int4 *>(tail + attn_desc_offset<Math>()) + wid * NS * 2;
     uint8_t *extra = tail + attn_extra_offset<Math>() + static_cast<size_t>(wid) * Math::kExtraBytes;
 
+    griddep_launch_dependents();   // the next kernel on the stream may begin its own read-only preamble
+
     // ---- plan: every CTA computes the same thing from the inputs alone -------------------------
     // Thread t sums the tiles of users [t*C, (t+1)*C); a block scan gives chunk prefixes.
     const int C = (p.B + NT - 1) / NT;
     const int G = gridDim.x;
-    const float2 *rate_rd = p.rates + (p.rate_sel & 1) * kMaxGrid;
-    float2 *rate_wr = p.rates + ((p.rate_sel + 1) & 1) * kMaxGrid;
+    // launch N writes third N % 3 and reads the one launch N-2 wrote: launch N-1 may still be running
+    const float2 *rate_rd = p.rates + ((p.rate_sel + 1) % 3) * kMaxGrid;
+    float2 *rate_wr = p.rates + (p.rate_sel % 3) * kMaxGrid;
     {
-        if (threadIdx.x == 0) { cta_clock0 = clock64(); cta_exits = 0; }
+        if (threadIdx.x == 0) cta_exits = 0;
         for (int i = threadIdx.x; i < G; i += NT) {     // the rate table travels together with the lengths
             const float2 v = __ldcg(rate_rd + i);
             sh_w[i] = v.x;
@@ -655,11 +663,6 @@ attn_kernel(const __grid_constant__ Params p, const __grid_constant__ CUtensorMa
         __syncthreads();
     }
     const int64_t T64 = static_cast<int64_t>(chunk_pfx[NT]) * p.S;
-    if (blockIdx.x == 0 && threadIdx.x == 0) {
-        p.hdr[HDR_BATCH] = p.B;
-        p.hdr[HDR_NSEQ] = p.B * p.S;
-        if (T64 >= (1ll << 31)) flag_error(p.hdr, 2 /* SPD_ERR_UNSUPPORTED */, -1);   // 32-bit tile counter
-    }
     const int T = T64 >= (1ll << 31) ? 0 : static_cast<int>(T64);
 
     // ---- shares: warp w of the grid owns tiles [bnd[w], bnd[w+1]) ------------------------------
@@ -713,25 +716,39 @@ attn_kernel(const __grid_constant__ Params p, const __grid_constant__ CUtensorMa
     }
     __syncthreads();
 
-    // ---- users that own no tile (nothing cached, or flagged): their outputs are written here ----
-    for (int u = gwarp; u < p.B; u += p.num_warps) {
-        int n0, n1;
-        cached_tiles(p, sh_np, u, n0, n1);
-        if (n0 + n1 != 0) continue;
-        const bool bad = __ldcg(p.bad + u) == p.epoch;
-        for (int sq = 0; sq < p.S; ++sq) {
-            const int hbase = first_head(p, sq);
-            for (int hh = 0; hh < p.geff; ++hh) {
-                float o[D / 32];
-#pragma unroll
-                for (int i = 0; i < D / 32; ++i) o[i] = 0.f;
-                finalize_store<D>(p, u, hbase + hh, o, -INFINITY, 0.f, lane, bad);
-            }
-        }
-    }
-
     const int t0 = gwarp < A ? bnd[gwarp] : 0;
     const int n = gwarp < A ? bnd[gwarp + 1] - t0 : 0;
+
+    // Everything up to the first tile loads only READS the call's inputs (lengths, page tables, the
+    // KV pools, a rate table nobody writes any more), so it may run while the previous kernel on the
+    // stream is still finishing on other SMs.  What follows touches the workspace, q, an incoming
+    // partial and the outputs, and waits for that kernel (griddep_wait below).
+    auto after_previous_kernel = [&]() {
+        griddep_wait();
+        if (threadIdx.x == 0) cta_clock0 = clock64();
+        if (blockIdx.x == 0 && threadIdx.x == 0) {
+            p.hdr[HDR_BATCH] = p.B;
+            p.hdr[HDR_NSEQ] = p.B * p.S;
+            if (T64 >= (1ll << 31)) flag_error(p.hdr, 2 /* SPD_ERR_UNSUPPORTED */, -1);   // 32-bit tile counter
+        }
+        // users that own no tile (nothing cached, or tables inconsistent): written and flagged here
+        for (int u = gwarp; u < p.B; u += p.num_warps) {
+            int n0, n1;
+            cached_tiles(p, sh_np, u, n0, n1);
+            if (n0 + n1 != 0) continue;
+            const bool bad = user_tiles<true>(p, u, n0, n1);
+            for (int sq = 0; sq < p.S; ++sq) {
+                const int hbase = first_head(p, sq);
+                for (int hh = 0; hh < p.geff; ++hh) {
+                    float o[D / 32];
+#pragma unroll
+                    for (int i = 0; i < D / 32; ++i) o[i] = 0.f;
+                    finalize_store<D>(p, u, hbase + hh, o, -INFINITY, 0.f, lane, bad);
+                }
+            }
+        }
+    };
+    if (n <= 0) after_previous_kernel();
     if (n > 0) {
 
     if (lane == 0) {
@@ -807,10 +824,7 @@ attn_kernel(const __grid_constant__ Params p, const __grid_constant__ CUtensorMa
         if (first) { seg_from0 = (c.j == 0); seg_has_t0 = (cur_t == t0); }
         int kind = 0;
         if (last && !(seg_from0 && c.j == c.np - 1)) kind = seg_has_t0 ? 1 : 2;
-        if (page < 0 || page >= p.part[part].num_pages) {
-            valid = 0;
-            if (lane == 0) { p.bad[c.u] = p.epoch; flag_error(p.hdr, 4 /* SPD_ERR_BAD_PAGE */, c.u); }
-        }
+        if (page < 0 || page >= p.part[part].num_pages) valid = 0;   // never fetched; flagged when consumed
         if (lane == 0) {
             descs[2 * stage] = make_int4(valid, (first ? 1 : 0) | (last ? 2 : 0) | (kind << 8), c.u, c.sq);
             descs[2 * stage + 1] = make_int4(c.np, c.j, cur_t, 0);
@@ -845,6 +859,7 @@ attn_kernel(const __grid_constant__ Params p, const __grid_constant__ CUtensorMa
     };
 
     for (int s = 0; s < NS && s < n; ++s) issue(s);
+    after_previous_kernel();
 
     typename Math::State st;
     bool seg_bad = false, dead = false;
@@ -855,8 +870,12 @@ attn_kernel(const __grid_constant__ Params p, const __grid_constant__ CUtensorMa
         const int4 d = descs[2 * stage];
         uint8_t *Ks = ring + static_cast<size_t>(stage) * 2 * TB, *Vs = Ks + TB;
         if (d.y & 1) { Math::begin(st, p, d.z, d.w, lane, extra); seg_bad = false; }
-        if (d.x > 0) Math::tile(st, p, Ks, Vs, d.x, lane, extra);
-        else seg_bad = true;
+        if (d.x > 0) {
+            Math::tile(st, p, Ks, Vs, d.x, lane, extra);
+        } else {                                   // a page index outside the pool: flag the user, skip the tile
+            seg_bad = true;
+            if (lane == 0) { p.bad[d.z] = p.epoch; flag_error(p.hdr, 4 /* SPD_ERR_BAD_PAGE */, d.z); }
+        }
         if (d.y & 2) {
             // the stage just consumed doubles as the staging area of the epilogue
             const int4 e = descs[2 * stage + 1];
