@@ -253,6 +253,36 @@ def time_e2e(spd, w, shape, ws, steps, warmup):
     return e0.elapsed_time(e1) / steps, lay.in_bytes, d2h, outh
 
 
+def time_append(spd, w, shape, ws, calls=8):
+    """spd_append_kv on the public cache: `calls` tokens per user appended back to back (the lengths are
+    first moved back by `calls`, and restored afterwards, so that every row fits the pages already listed)."""
+    if int(w.pub.seq_lens.min()) < 1:
+        return None
+    dev = w.q.device
+    keep = w.pub.seq_lens.clone()
+    gen = torch.Generator(device=dev)
+    gen.manual_seed(99)
+    k_new = torch.randn((w.batch, w.num_kv_heads, w.head_dim), generator=gen, device=dev).to(w.dtype)
+    v_new = torch.randn((w.batch, w.num_kv_heads, w.head_dim), generator=gen, device=dev).to(w.dtype)
+    ms = []
+    for rep in range(4):
+        w.pub.seq_lens.copy_(torch.clamp(keep - calls, min=0))
+        torch.cuda.synchronize()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        for _ in range(calls):
+            spd.spd_append_kv(shape, k_new, v_new, w.pub, ws)
+        e1.record()
+        torch.cuda.synchronize()
+        ms.append(e0.elapsed_time(e1) / calls)
+    code, bad = spd.spd_query_device_status(ws)
+    w.pub.seq_lens.copy_(keep)     # the rows written sit where tokens already were or in unused slots: restore
+    if code != spd.SPD_OK:
+        raise RuntimeError(f"append failed: status {code}, user {bad}")
+    nbytes = 2 * w.batch * w.num_kv_heads * w.head_dim * w.elem_size
+    return {"us_per_call": min(ms) * 1e3, "bytes_written_per_call": nbytes, "note": "latency-bound: one small kernel"}
+
+
 def run_cuda(args):
     from paper_2409_19134_b200 import binding as spd
     rank, local_rank, world = dist_env()
@@ -333,6 +363,10 @@ def run_cuda(args):
             o["kv_bytes_per_step"] = w.kv_bytes()
             others[name] = o
         line["other_configs"] = others
+        del w
+        torch.cuda.empty_cache()
+        w = wl.make_workload(cfg, device=dev)
+        line["append_kv"] = time_append(spd, w, spd.make_shape(w.batch, w.num_q_heads, w.num_kv_heads, w.head_dim, w.dtype, w.sm_scale), ws)
         w = wl.make_workload(cfg, device="cpu")
         line["cpu_baseline"] = cpu_baseline(w)
     print(json.dumps(line), flush=True)

@@ -116,6 +116,22 @@ spd_status spd_decode_step(const spd_shape *shape, const void *q, const spd_page
                            void *ws, size_t ws_bytes, void *cuda_stream);
 
 /*
+ * Append of the new token's K and V rows to a paged cache -- what the service does to its public
+ * cache right before attention (protocol step 3a; Fig. 3 step 2), so that the new token attends to
+ * itself through the public partition.  k_new, v_new: [batch][num_kv_heads][head_dim] in the shape's
+ * dtype.  The row of user u lands at token position seq_lens[u] (page
+ * page_indices[page_indptr[u] + seq_lens[u] / page_size], slot seq_lens[u] % page_size) and seq_lens[u]
+ * grows by one, in place.  The caller provides the room: a user whose listed pages are already full
+ * (or whose table is inconsistent) is left untouched and raises SPD_ERR_BAD_PAGE in the workspace's
+ * status words.  One small kernel, enqueued on the stream in plain stream order (it starts after
+ * every earlier call on that stream has finished with the cache).
+ */
+spd_status spd_append_kv(const spd_shape *shape, const void *k_new, const void *v_new, void *k_pool,
+                         void *v_pool, int32_t num_pages, const int32_t *page_indptr,
+                         const int32_t *page_indices, int32_t *seq_lens, void *ws, size_t ws_bytes,
+                         void *cuda_stream);
+
+/*
  * spd_decode_step (fused) for a caller whose per-step data lives in HOST memory (no counterpart in
  * the paper, whose two processes exchange these arrays through the host on every layer).
  *

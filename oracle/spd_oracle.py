@@ -209,3 +209,29 @@ def kv_from_torch(part) -> KV:
 def q_from_torch(q) -> np.ndarray:
     import torch
     return bf16_bits(q) if q.dtype == torch.bfloat16 else q.contiguous().numpy()
+
+
+def append(kv: KV, k_new: np.ndarray, v_new: np.ndarray) -> np.ndarray:
+    """Append one token per user to a partition, in place (protocol step 3a; Fig. 3 step 2).
+
+    k_new, v_new: [B, Hkv, D] in the pools' dtype.  The row of user u goes to token position
+    len_u, i.e. page page_indices[page_indptr[u] + len_u // P], slot len_u % P, and len_u grows by
+    one.  A user whose listed pages are full is left untouched.  Returns a bool array: appended or not.
+    Pure indexing, written out as loops.
+    """
+    B, Hkv, D = k_new.shape
+    P = kv.k_pool.shape[2]
+    done = np.zeros(B, dtype=bool)
+    for u in range(B):
+        t = int(kv.seq_lens[u])
+        cap = int(kv.page_indptr[u + 1]) - int(kv.page_indptr[u])
+        if t < 0 or t >= cap * P:
+            continue
+        page = int(kv.page_indices[int(kv.page_indptr[u]) + t // P])
+        for h in range(Hkv):
+            for d in range(D):
+                kv.k_pool[page, h, t % P, d] = k_new[u, h, d]
+                kv.v_pool[page, h, t % P, d] = v_new[u, h, d]
+        kv.seq_lens[u] = t + 1
+        done[u] = True
+    return done

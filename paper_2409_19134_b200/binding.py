@@ -21,7 +21,7 @@ _STATUS_NAMES = {0: "SPD_OK", 1: "SPD_ERR_INVALID_ARG", 2: "SPD_ERR_UNSUPPORTED"
 EXPORTS = ["spd_workspace_size", "spd_partial_attn", "spd_service_attn_merge", "spd_decode_step",
            "spd_step_blob_layout", "spd_decode_step_host", "spd_query_device_status",
            "spd_kernel_launch_count", "spd_status_string", "spd_profile_begin", "spd_profile_end",
-           "spd_decode_step_static"]
+           "spd_decode_step_static", "spd_append_kv"]
 
 
 class SpdError(RuntimeError):
@@ -78,6 +78,7 @@ def lib() -> C.CDLL:
         L.spd_profile_end.argtypes = [C.POINTER(C.c_int32), C.POINTER(C.c_double)]
         L.spd_decode_step_static.argtypes = [C.POINTER(Shape), vp, C.POINTER(PagedKV), C.POINTER(PagedKV), vp, C.c_int,
                                              C.c_int32, C.POINTER(C.c_int32), vp]
+        L.spd_append_kv.argtypes = [C.POINTER(Shape), vp, vp, vp, vp, C.c_int32, vp, vp, vp, vp, sz, vp]
         for name in EXPORTS[:7] + EXPORTS[9:]:
             getattr(L, name).restype = C.c_int
         _lib = L
@@ -240,3 +241,12 @@ def spd_decode_step_static(shape, q, priv, pub, out, wait_and_check=True, stream
     if code not in (SPD_OK, 4, 6):
         raise SpdError(code, "spd_decode_step_static")
     return int(code), int(bad.value)
+
+
+def spd_append_kv(shape, k_new, v_new, part, ws, stream=None) -> None:
+    """Append one token per user to the partition `part` (its pools and seq_lens are updated in place)."""
+    assert k_new.is_contiguous() and v_new.is_contiguous()
+    _check(lib().spd_append_kv(C.byref(shape), k_new.data_ptr(), v_new.data_ptr(), part.k_pool.data_ptr(),
+                               part.v_pool.data_ptr(), int(part.k_pool.shape[0]), part.page_indptr.data_ptr(),
+                               _ptr(part.page_indices), part.seq_lens.data_ptr(), ws.data_ptr(), ws.numel(),
+                               _stream_ptr(stream)), "spd_append_kv")

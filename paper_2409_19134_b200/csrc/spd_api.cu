@@ -366,6 +366,28 @@ spd_status spd_decode_step(const spd_shape *shape, const void *q, const spd_page
     return run_job(b, ws, ws_bytes, cuda_stream);
 }
 
+spd_status spd_append_kv(const spd_shape *shape, const void *k_new, const void *v_new, void *k_pool, void *v_pool,
+                         int32_t num_pages, const int32_t *page_indptr, const int32_t *page_indices,
+                         int32_t *seq_lens, void *ws, size_t ws_bytes, void *cuda_stream) {
+    spd_status rc = check_shape(shape);
+    if (rc != SPD_OK) return rc;
+    if (!k_new || !v_new || !k_pool || !v_pool || !page_indptr || !seq_lens || !ws || num_pages <= 0) return SPD_ERR_INVALID_ARG;
+    if (misaligned(k_new, 16) || misaligned(v_new, 16) || misaligned(k_pool, 128) || misaligned(v_pool, 128) ||
+        misaligned(ws, 256))
+        return SPD_ERR_INVALID_ARG;
+    if (ws_bytes < HDR_WORDS * 4) return SPD_ERR_WORKSPACE;
+    AppendParams ap;
+    ap.B = shape->batch; ap.Hkv = shape->num_kv_heads;
+    ap.row_bytes = shape->head_dim * (shape->dtype == SPD_BF16 ? 2 : 4);
+    ap.k_new = static_cast<const uint8_t *>(k_new); ap.v_new = static_cast<const uint8_t *>(v_new);
+    ap.k_pool = static_cast<uint8_t *>(k_pool); ap.v_pool = static_cast<uint8_t *>(v_pool);
+    ap.num_pages = num_pages; ap.indptr = page_indptr; ap.indices = page_indices; ap.lens = seq_lens;
+    ap.hdr = static_cast<int32_t *>(ws);
+    append_kernel<<<shape->batch, 128, 0, static_cast<cudaStream_t>(cuda_stream)>>>(ap);
+    ++g_launches;
+    return cudaGetLastError() == cudaSuccess ? SPD_OK : SPD_ERR_CUDA;
+}
+
 spd_status spd_step_blob_layout(const spd_shape *shape, int64_t priv_pages_listed, int64_t pub_pages_listed,
                                 spd_dtype out_dtype, spd_step_blob *layout) {
     spd_status rc = check_shape(shape);

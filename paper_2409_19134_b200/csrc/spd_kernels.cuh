@@ -917,4 +917,47 @@ attn_kernel(const __grid_constant__ Params p, const __grid_constant__ CUtensorMa
     }
 }
 
+// ------------------------------------------------------------------------------------------------
+// Append of the new token's K and V rows to a paged cache (protocol step 3a; Fig. 3 step 2): one CTA
+// per user.  The row of user u goes to token position len_u -- page indices[indptr[u] + len_u / 16],
+// slot len_u % 16 -- and len_u grows by one.  A user whose listed pages are full, or whose table is
+// inconsistent, is left untouched and flagged.  Plain 16-byte copies: a few hundred KB per call.
+struct AppendParams {
+    int32_t B, Hkv, row_bytes;      // row_bytes = head_dim * element size
+    const uint8_t *k_new, *v_new;   // [B][Hkv][row_bytes]
+    uint8_t *k_pool, *v_pool;
+    int32_t num_pages;
+    const int32_t *indptr, *indices;
+    int32_t *lens;
+    int32_t *hdr;
+};
+
+__global__ void __launch_bounds__(128) append_kernel(AppendParams p) {
+    const int u = blockIdx.x;
+    __shared__ int64_t dst_row;   // byte offset of (page, kv head 0, slot) in a pool, or -1
+    if (threadIdx.x == 0) {
+        const int64_t lo = p.indptr[u], hi = p.indptr[u + 1], end = p.indptr[p.B], t = p.lens[u];
+        int64_t off = -1;
+        if (lo >= 0 && hi >= lo && hi <= end && t >= 0 && t < (hi - lo) * kPage && p.indices != nullptr) {
+            const int64_t page = p.indices[lo + t / kPage];
+            if (page >= 0 && page < p.num_pages) off = ((page * p.Hkv) * kPage + t % kPage) * p.row_bytes;
+        }
+        if (off < 0) flag_error(p.hdr, 4 /* SPD_ERR_BAD_PAGE */, u);
+        dst_row = off;
+    }
+    __syncthreads();
+    const int64_t off = dst_row;
+    if (off < 0) return;
+    const int chunks = p.row_bytes / 16, total = p.Hkv * chunks;
+    for (int i = threadIdx.x; i < total; i += blockDim.x) {
+        const int h = i / chunks, c = i - h * chunks;
+        const int64_t src = (static_cast<int64_t>(u) * p.Hkv + h) * p.row_bytes + c * 16;
+        const int64_t dst = off + static_cast<int64_t>(h) * kPage * p.row_bytes + c * 16;
+        *reinterpret_cast<uint4 *>(p.k_pool + dst) = *reinterpret_cast<const uint4 *>(p.k_new + src);
+        *reinterpret_cast<uint4 *>(p.v_pool + dst) = *reinterpret_cast<const uint4 *>(p.v_new + src);
+    }
+    __syncthreads();
+    if (threadIdx.x == 0) p.lens[u] += 1;
+}
+
 }  // namespace spd

@@ -176,3 +176,54 @@ def test_host_blob_step_matches_oracle(name):
     ip[w.batch] += 1
     with pytest.raises(spd.SpdError):
         spd.spd_decode_step_host(shape, lay, host, devb, pools[0], pools[1], torch.float32, ws)
+
+
+@pytest.mark.parametrize("dtype", ["bf16", "f32"])
+def test_append_kv_is_bit_exact_and_feeds_the_next_step(dtype):
+    """Step 3a: the new token's K/V rows go into the public cache, then attention sees them."""
+    rng = np.random.default_rng(51)
+    B, hq, hkv, d = 6, 8, 4, 128
+    lout = np.array([0, 15, 16, 31, 5, 32])           # page boundaries on both sides
+    lin = rng.integers(1, 200, size=B)
+    cfg = dict(name="append", batch=B, hq=hq, hkv=hkv, d=d, dtype=dtype, lin=("const", 0), lout=("const", 0), seed=52)
+    w = wl.make_workload(cfg, lengths=(lin, lout), slack=False, over_alloc=2.0)   # leaves free pages in the pools
+    # one spare page for everybody except the last user, whose pages are exactly full
+    need = (lout + 15) // 16
+    cap = need + 1
+    cap[-1] = need[-1]
+    used = set(w.pub.page_indices.tolist())
+    free = iter(sorted(set(range(w.pub.num_pages)) - used))
+    indices, indptr = [], [0]
+    for u in range(B):
+        own = w.pub.page_indices[int(w.pub.page_indptr[u]):int(w.pub.page_indptr[u + 1])].tolist()
+        while len(own) < cap[u]:
+            own.append(next(free))
+        indices += own
+        indptr.append(len(indices))
+    w.pub.page_indptr = torch.tensor(indptr, dtype=torch.int32)
+    w.pub.page_indices = torch.tensor(indices, dtype=torch.int32)
+    gen = torch.Generator().manual_seed(53)
+    k_new = torch.randn((B, hkv, d), generator=gen).to(w.dtype)
+    v_new = torch.randn((B, hkv, d), generator=gen).to(w.dtype)
+
+    wg = w.to("cuda")
+    shape = spd.make_shape(B, hq, hkv, d, w.dtype, w.sm_scale)
+    ws = spd.alloc_workspace(shape)
+    spd.spd_append_kv(shape, k_new.cuda(), v_new.cuda(), wg.pub, ws)
+    status = spd.spd_query_device_status(ws)
+    assert status == (4, B - 1)                        # the full user is reported, everybody else appended
+
+    q, kin, kout = oracle_inputs(w)
+    done = orc.append(kout, orc.q_from_torch(k_new), orc.q_from_torch(v_new))
+    assert done.tolist() == [True] * (B - 1) + [False]
+    assert np.array_equal(wg.pub.seq_lens.cpu().numpy(), kout.seq_lens)
+
+    def bits(t):
+        return t.cpu().view(torch.int16 if t.dtype == torch.bfloat16 else torch.int32).numpy()
+    assert np.array_equal(bits(wg.pub.k_pool), kout.k_pool.view(bits(wg.pub.k_pool).dtype))
+    assert np.array_equal(bits(wg.pub.v_pool), kout.v_pool.view(bits(wg.pub.v_pool).dtype))
+
+    out = torch.full((B, hq, d), float("nan"), dtype=torch.float32, device="cuda")
+    spd.spd_decode_step(shape, wg.q, wg.priv, wg.pub, out, ws, fused=True)
+    assert spd.spd_query_device_status(ws) == (spd.SPD_OK, -1)
+    assert_close(out.cpu().numpy(), orc.full(q, kin, kout, w.sm_scale), w.dtype, "decode after append")

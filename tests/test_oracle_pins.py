@@ -322,3 +322,46 @@ def test_workload_generator_recipes():
     n_tok = int(w.priv.seq_lens.sum())
     assert int((~torch.isnan(w.priv.k_pool.float()[..., 0])).sum()) == n_tok
     assert w.pub.page_indices.numel() >= 0 and torch.isnan(w.pub.k_pool.float()).all()
+
+
+# ---------------------------------------------------------------- append of the new token (step 3a)
+def test_append_then_attend_equals_dense_concatenation():
+    rng = np.random.default_rng(21)
+    Hkv, Hq, D, P = 2, 4, 8, 16
+    lens = [15, 16, 0, 31]                      # last slot of a page, first slot of a fresh page, empty, mid-page
+    ks, vs = _rand_dense(rng, lens, Hkv, D)
+    kv = dense_to_paged(ks, vs, rng=rng)
+    # give every user one spare page beyond what its tokens need, except user 3 (full after one more token)
+    need = [(n + P - 1) // P for n in lens]
+    cap = [need[0], need[1] + 1, 1, need[3]]
+    indptr = np.concatenate([[0], np.cumsum(cap)]).astype(np.int32)
+    spare = iter(sorted(set(range(kv.k_pool.shape[0])) - set(kv.page_indices.tolist())))   # the 3 unused pages
+    indices = []
+    for u in range(4):
+        own = list(kv.page_indices[kv.page_indptr[u]:kv.page_indptr[u + 1]])
+        while len(own) < cap[u]:
+            own.append(next(spare))
+        indices += own
+    kv = orc.KV(kv.k_pool, kv.v_pool, indptr, np.array(indices, np.int32), kv.seq_lens)
+    before_k = kv.k_pool.copy()
+    k_new = rng.standard_normal((4, Hkv, D)).astype(np.float32)
+    v_new = rng.standard_normal((4, Hkv, D)).astype(np.float32)
+    done = orc.append(kv, k_new, v_new)
+    assert done.tolist() == [True, True, True, True] and kv.seq_lens.tolist() == [16, 17, 1, 32]
+    # exactly one row per (user, kv head) changed
+    changed = ~((before_k == kv.k_pool) | (np.isnan(before_k) & np.isnan(kv.k_pool)))
+    assert int(changed.any(axis=-1).sum()) == 4 * Hkv
+    q = rng.standard_normal((4, Hq, D)).astype(np.float32)
+    y = orc.full(q, kv, None, 0.4)
+    for u in range(4):
+        for h in range(Hq):
+            kd = np.concatenate([ks[u][h // 2], k_new[u, h // 2][None]], axis=0)
+            vd = np.concatenate([vs[u][h // 2], v_new[u, h // 2][None]], axis=0)
+            assert np.max(np.abs(y[u, h] - orc.brute_force(q[u, h], kd, vd, 0.4))) < 1e-12
+    # users 0 and 3 are now full: a second append leaves them alone, the others grow
+    snap = (kv.k_pool.copy(), kv.seq_lens.copy())
+    done = orc.append(kv, k_new, v_new)
+    assert done.tolist() == [False, True, True, False] and kv.seq_lens.tolist() == [16, 18, 2, 32]
+    for u in (0, 3):
+        pages = kv.page_indices[kv.page_indptr[u]:kv.page_indptr[u + 1]]
+        assert np.array_equal(np.nan_to_num(kv.k_pool[pages]), np.nan_to_num(snap[0][pages]))
