@@ -247,7 +247,7 @@ def time_e2e(spd, w, shape, ws, steps, warmup):
         call()
     e1.record()
     torch.cuda.synchronize()
-    d2h = lay.total_bytes - lay.out + 32
+    d2h = lay.total_bytes - lay.status
     n_out = w.batch * w.num_q_heads * w.head_dim
     outh = host[lay.out:lay.out + 4 * n_out].view(torch.float32).reshape(w.batch, w.num_q_heads, w.head_dim).clone()
     return e0.elapsed_time(e1) / steps, lay.in_bytes, d2h, outh

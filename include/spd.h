@@ -138,20 +138,23 @@ spd_status spd_append_kv(const spd_shape *shape, const void *k_new, const void *
  * Everything that changes from step to step -- q, both partitions' page_indptr / seq_lens /
  * page_indices -- sits in ONE host buffer (pinned memory makes the copy asynchronous) at the offsets
  * that spd_step_blob_layout() reports, so that a step costs one host-to-device copy, one kernel and
- * two device-to-host copies (the output, the status words).  The KV pools stay resident on the
+ * one device-to-host copy (status words and output, which sit side by side in the blob).  The host
+ * blob must start out zeroed; the call leaves its status block zeroed again.  The KV pools stay resident on the
  * device: `priv_pools` and `pub_pools` carry k_pool, v_pool and num_pages only (their table pointers
  * are ignored).  `device_blob` is device memory of layout->total_bytes, 256-byte aligned.
  *
- * The call copies host_blob[0, in_bytes) to the device, runs the step, copies the output to
- * host_blob + layout->out, waits for the stream and returns the device status as
- * spd_query_device_status() would (*first_bad_user likewise; may be NULL).
+ * The call copies host_blob[0, in_bytes) to the device, runs the step, copies status and output back
+ * (the output to host_blob + layout->out), waits for the stream and returns the device status of
+ * this step (*first_bad_user: lowest flagged user or -1; may be NULL).  The workspace's own sticky
+ * status is not involved.
  */
 typedef struct {
     int64_t priv_pages_listed, pub_pages_listed;   /* entries of the two page_indices arrays */
     size_t  q;                                      /* [batch][num_q_heads][head_dim], shape dtype */
     size_t  priv_indptr, priv_lens, priv_indices;   /* int32 [batch+1], [batch], [priv_pages_listed] */
     size_t  pub_indptr, pub_lens, pub_indices;
-    size_t  in_bytes;                               /* the inputs occupy [0, in_bytes) */
+    size_t  status;                                 /* 256 bytes the caller keeps ZERO on the host */
+    size_t  in_bytes;                               /* the inputs (and the status block) occupy [0, in_bytes) */
     size_t  out;                                    /* [batch][num_q_heads][head_dim], out_dtype */
     size_t  total_bytes;
 } spd_step_blob;

@@ -44,7 +44,7 @@ class StepBlob(C.Structure):
     _fields_ = [("priv_pages_listed", C.c_int64), ("pub_pages_listed", C.c_int64), ("q", C.c_size_t),
                 ("priv_indptr", C.c_size_t), ("priv_lens", C.c_size_t), ("priv_indices", C.c_size_t),
                 ("pub_indptr", C.c_size_t), ("pub_lens", C.c_size_t), ("pub_indices", C.c_size_t),
-                ("in_bytes", C.c_size_t), ("out", C.c_size_t), ("total_bytes", C.c_size_t)]
+                ("status", C.c_size_t), ("in_bytes", C.c_size_t), ("out", C.c_size_t), ("total_bytes", C.c_size_t)]
 
 
 class Partial(C.Structure):

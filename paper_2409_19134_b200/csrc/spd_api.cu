@@ -199,6 +199,7 @@ struct Job {
     void *out;
     spd_dtype out_dtype;
     int32_t epoch;                 // id of the call (both halves of a chained step share one)
+    int32_t *status_words;         // where the kernel raises its status; null = the workspace header
 };
 
 spd_status run_job(const Job &job, void *ws, size_t ws_bytes, void *stream) {
@@ -224,7 +225,7 @@ spd_status run_job(const Job &job, void *ws, size_t ws_bytes, void *stream) {
     const bool bf = s.dtype == SPD_BF16;
     const int warps_per_cta = bf ? MathBF16<128>::kWarps : MathF32<128, 1>::kWarps;
     p.num_warps = di.sms * warps_per_cta;
-    p.hdr = reinterpret_cast<int32_t *>(w + L.hdr);
+    p.hdr = job.status_words ? job.status_words : reinterpret_cast<int32_t *>(w + L.hdr);
     p.bad = reinterpret_cast<int32_t *>(w + L.bad);
     p.tickets = reinterpret_cast<int32_t *>(w + L.tickets);
     p.rates = reinterpret_cast<float2 *>(w + L.rates);
@@ -407,6 +408,7 @@ spd_status spd_step_blob_layout(const spd_shape *shape, int64_t priv_pages_liste
     layout->pub_indptr = take((B + 1) * 4);
     layout->pub_lens = take(B * 4);
     layout->pub_indices = take(static_cast<size_t>(pub_pages_listed) * 4);
+    layout->status = take(HDR_WORDS * 4);      // zero on the host: the upload clears the device copy
     layout->in_bytes = off;
     layout->out = take(rows * oes);
     layout->total_bytes = off;
@@ -441,12 +443,33 @@ spd_status spd_decode_step_host(const spd_shape *shape, const spd_step_blob *lay
     b.page_indptr = reinterpret_cast<const int32_t *>(db + layout->pub_indptr);
     b.seq_lens = reinterpret_cast<const int32_t *>(db + layout->pub_lens);
     b.page_indices = reinterpret_cast<const int32_t *>(db + layout->pub_indices);
-    rc = spd_decode_step(shape, db + layout->q, &a, &b, db + layout->out, out_dtype, 1, ws, ws_bytes, cuda_stream);
-    if (rc != SPD_OK) return rc;
-    if (cudaMemcpyAsync(static_cast<uint8_t *>(host_blob) + layout->out, db + layout->out, layout->total_bytes - layout->out,
-                        cudaMemcpyDeviceToHost, st) != cudaSuccess)
+    if ((rc = check_kv(shape, &a)) != SPD_OK || (rc = check_kv(shape, &b)) != SPD_OK) return rc;
+    if (out_dtype != SPD_F32 && out_dtype != SPD_BF16) return SPD_ERR_UNSUPPORTED;
+    // The step raises its status in the blob (uploaded as zeros a moment ago), right in front of the
+    // output, so that one copy brings both back.
+    Job job{};
+    job.shape = shape; job.q = db + layout->q; job.part[0] = &a; job.part[1] = &b;
+    job.mode = OUT_FINAL; job.pin = nullptr; job.out = db + layout->out; job.out_dtype = out_dtype;
+    job.epoch = next_epoch();
+    job.status_words = reinterpret_cast<int32_t *>(db + layout->status);
+    if ((rc = run_job(job, ws, ws_bytes, cuda_stream)) != SPD_OK) return rc;
+    uint8_t *hs = static_cast<uint8_t *>(host_blob) + layout->status;
+    if (cudaMemcpyAsync(hs, db + layout->status, layout->total_bytes - layout->status, cudaMemcpyDeviceToHost, st) != cudaSuccess)
         return SPD_ERR_CUDA;
-    return spd_query_device_status(ws, cuda_stream, first_bad_user);
+    if (cudaStreamSynchronize(st) != cudaSuccess) return SPD_ERR_CUDA;
+    int32_t *hdr = reinterpret_cast<int32_t *>(hs);
+    const int32_t code = hdr[HDR_STATUS], enc = hdr[HDR_BAD_ENC];
+    memset(hs, 0, HDR_WORDS * 4);              // ready for the next upload
+    if (first_bad_user) *first_bad_user = enc ? 0x7fffffff - enc : -1;
+    if (code == SPD_ERR_TIMEOUT) {             // a kernel that gave up may have left merge tickets drawn
+        DeviceInfo di;
+        if (device_info(&di) != SPD_OK) return SPD_ERR_CUDA;
+        const WsLayout L = ws_layout(*shape, di.sms);
+        if (cudaMemsetAsync(static_cast<uint8_t *>(ws) + L.tickets, 0, L.scratch - L.tickets, st) != cudaSuccess ||
+            cudaStreamSynchronize(st) != cudaSuccess)
+            return SPD_ERR_CUDA;
+    }
+    return static_cast<spd_status>(code);
 }
 
 spd_status spd_query_device_status(void *ws, void *cuda_stream, int32_t *first_bad_user) {

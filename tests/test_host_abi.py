@@ -43,7 +43,7 @@ def test_struct_layouts_match_header(lib):
     assert C.sizeof(spd.Shape) == 28
     assert C.sizeof(spd.PagedKV) == 48 and spd.PagedKV.page_indptr.offset == 24
     assert C.sizeof(spd.Partial) == 24
-    assert C.sizeof(spd.StepBlob) == 96
+    assert C.sizeof(spd.StepBlob) == 104
 
 
 def test_bad_arguments_are_rejected_on_the_host(lib):
@@ -68,7 +68,7 @@ def test_bad_arguments_are_rejected_on_the_host(lib):
     assert lib.spd_step_blob_layout(C.byref(ok), -1, 0, 0, C.byref(lay)) == 1
     assert lib.spd_step_blob_layout(C.byref(ok), 10, 10, 0, C.byref(lay)) == 0
     assert lay.in_bytes >= 4 * 8 * 64 * 4 + 2 * (5 + 4 + 10) * 4 and lay.total_bytes >= lay.out + 4 * 8 * 64 * 4
-    assert lay.q == 0 and lay.out == lay.in_bytes and lay.priv_indices % 256 == 0
+    assert lay.q == 0 and lay.out == lay.in_bytes and lay.status + 256 == lay.in_bytes and lay.priv_indices % 256 == 0
     assert lib.spd_decode_step_host(C.byref(ok), C.byref(lay), None, None, None, None, 0, None, None, 0, None) == 1
 
 
