@@ -116,6 +116,31 @@ spd_status spd_decode_step(const spd_shape *shape, const void *q, const spd_page
                            void *ws, size_t ws_bytes, void *cuda_stream);
 
 /*
+ * Input-attention monitor (Sec. 2.4.4 and Sec. 7.1.1: watching how much attention the query pays to
+ * the user's original instruction, inside the per-user process, to notice an instruction injected by
+ * the service).  For every user, tokens [tok_lo[u], tok_hi[u]) of the PRIVATE partition are watched
+ * (an empty or out-of-range interval watches nothing).  All pointers are device memory.
+ *
+ *   spd_partial_attn_watch : spd_partial_attn, plus out[u][h] = sum of exp(s_i - m) over the watched
+ *                            tokens -- the watched part of l, in l's gauge; out / l is the share of the
+ *                            private partition's softmax mass that sits on the watched tokens.
+ *   spd_decode_step_watch  : spd_decode_step (fused), plus out[u][h] = share of the FULL softmax mass
+ *                            (both partitions) that sits on the watched tokens, in [0, 1].
+ * The attention output itself is what the unwatched calls give.
+ */
+typedef struct {
+    const int32_t *tok_lo;   /* [batch] */
+    const int32_t *tok_hi;   /* [batch] */
+    float         *out;      /* [batch][num_q_heads] */
+} spd_watch;
+spd_status spd_partial_attn_watch(const spd_shape *shape, const void *q, const spd_paged_kv *priv,
+                                  spd_partial out, const spd_watch *watch, void *ws, size_t ws_bytes,
+                                  void *cuda_stream);
+spd_status spd_decode_step_watch(const spd_shape *shape, const void *q, const spd_paged_kv *priv,
+                                 const spd_paged_kv *pub, void *out, spd_dtype out_dtype,
+                                 const spd_watch *watch, void *ws, size_t ws_bytes, void *cuda_stream);
+
+/*
  * Append of the new token's K and V rows to a paged cache -- what the service does to its public
  * cache right before attention (protocol step 3a; Fig. 3 step 2), so that the new token attends to
  * itself through the public partition.  k_new, v_new: [batch][num_kv_heads][head_dim] in the shape's

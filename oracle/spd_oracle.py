@@ -235,3 +235,37 @@ def append(kv: KV, k_new: np.ndarray, v_new: np.ndarray) -> np.ndarray:
         kv.seq_lens[u] = t + 1
         done[u] = True
     return done
+
+
+def watched_mass(q: np.ndarray, priv: KV, pub: Optional[KV], sm_scale: float, tok_lo, tok_hi):
+    """Share of the softmax mass that sits on tokens [tok_lo[u], tok_hi[u]) of the private partition
+    (Sec. 2.4.4 / 7.1.1: attention paid to the watched instruction).
+
+    Returns (share_full [B, Hq], share_private [B, Hq]): relative to the attention over both partitions
+    and over the private partition alone.  Written from the definition: with the partials
+    (m_w, l_w) of the watched range, (m_in, l_in) of the private and (m_out, l_out) of the public
+    partition, the mass of a set is l * exp(m) and a share is a ratio of masses.
+    """
+    B, Hq, _ = q.shape
+    _, m_in, l_in = partial(q, priv, sm_scale)
+    if pub is not None:
+        _, m_out, l_out = partial(q, pub, sm_scale)
+    else:
+        m_out, l_out = np.full((B, Hq), -np.inf), np.zeros((B, Hq))
+    full = np.zeros((B, Hq))
+    own = np.zeros((B, Hq))
+    for u in range(B):
+        lo, hi = max(int(tok_lo[u]), 0), int(tok_hi[u])
+        if hi <= lo:
+            continue
+        _, m_w, l_w = partial(q, priv, sm_scale, lo, hi)
+        for h in range(Hq):
+            if l_w[u, h] == 0.0:
+                continue
+            M = max(m_in[u, h], m_out[u, h])
+            mass_w = l_w[u, h] * np.exp(m_w[u, h] - M)
+            mass_in = l_in[u, h] * np.exp(m_in[u, h] - M)
+            mass_out = l_out[u, h] * np.exp(m_out[u, h] - M) if l_out[u, h] > 0 else 0.0
+            full[u, h] = mass_w / (mass_in + mass_out)
+            own[u, h] = mass_w / mass_in
+    return full, own

@@ -21,7 +21,8 @@ _STATUS_NAMES = {0: "SPD_OK", 1: "SPD_ERR_INVALID_ARG", 2: "SPD_ERR_UNSUPPORTED"
 EXPORTS = ["spd_workspace_size", "spd_partial_attn", "spd_service_attn_merge", "spd_decode_step",
            "spd_step_blob_layout", "spd_decode_step_host", "spd_query_device_status",
            "spd_kernel_launch_count", "spd_status_string", "spd_profile_begin", "spd_profile_end",
-           "spd_decode_step_static", "spd_append_kv"]
+           "spd_decode_step_static", "spd_append_kv",
+           "spd_partial_attn_watch", "spd_decode_step_watch"]
 
 
 class SpdError(RuntimeError):
@@ -45,6 +46,10 @@ class StepBlob(C.Structure):
                 ("priv_indptr", C.c_size_t), ("priv_lens", C.c_size_t), ("priv_indices", C.c_size_t),
                 ("pub_indptr", C.c_size_t), ("pub_lens", C.c_size_t), ("pub_indices", C.c_size_t),
                 ("status", C.c_size_t), ("in_bytes", C.c_size_t), ("out", C.c_size_t), ("total_bytes", C.c_size_t)]
+
+
+class Watch(C.Structure):
+    _fields_ = [("tok_lo", C.c_void_p), ("tok_hi", C.c_void_p), ("out", C.c_void_p)]
 
 
 class Partial(C.Structure):
@@ -78,6 +83,9 @@ def lib() -> C.CDLL:
         L.spd_profile_end.argtypes = [C.POINTER(C.c_int32), C.POINTER(C.c_double)]
         L.spd_decode_step_static.argtypes = [C.POINTER(Shape), vp, C.POINTER(PagedKV), C.POINTER(PagedKV), vp, C.c_int,
                                              C.c_int32, C.POINTER(C.c_int32), vp]
+        L.spd_partial_attn_watch.argtypes = [C.POINTER(Shape), vp, C.POINTER(PagedKV), Partial, C.POINTER(Watch), vp, sz, vp]
+        L.spd_decode_step_watch.argtypes = [C.POINTER(Shape), vp, C.POINTER(PagedKV), C.POINTER(PagedKV), vp, C.c_int,
+                                            C.POINTER(Watch), vp, sz, vp]
         L.spd_append_kv.argtypes = [C.POINTER(Shape), vp, vp, vp, vp, C.c_int32, vp, vp, vp, vp, sz, vp]
         for name in EXPORTS[:7] + EXPORTS[9:]:
             getattr(L, name).restype = C.c_int
@@ -250,3 +258,22 @@ def spd_append_kv(shape, k_new, v_new, part, ws, stream=None) -> None:
                                part.v_pool.data_ptr(), int(part.k_pool.shape[0]), part.page_indptr.data_ptr(),
                                _ptr(part.page_indices), part.seq_lens.data_ptr(), ws.data_ptr(), ws.numel(),
                                _stream_ptr(stream)), "spd_append_kv")
+
+
+def _watch(tok_lo, tok_hi, out) -> Watch:
+    assert tok_lo.dtype == torch.int32 and tok_hi.dtype == torch.int32 and out.dtype == torch.float32
+    return Watch(tok_lo.data_ptr(), tok_hi.data_ptr(), out.data_ptr())
+
+
+def spd_partial_attn_watch(shape, q, priv, out, tok_lo, tok_hi, watch_out, ws, stream=None) -> None:
+    kv, w = paged_kv(priv), _watch(tok_lo, tok_hi, watch_out)
+    part = Partial(out[0].data_ptr(), out[1].data_ptr(), out[2].data_ptr())
+    _check(lib().spd_partial_attn_watch(C.byref(shape), q.data_ptr(), C.byref(kv), part, C.byref(w), ws.data_ptr(),
+                                        ws.numel(), _stream_ptr(stream)), "spd_partial_attn_watch")
+
+
+def spd_decode_step_watch(shape, q, priv, pub, out, tok_lo, tok_hi, watch_out, ws, stream=None) -> None:
+    a, b, w = paged_kv(priv), paged_kv(pub), _watch(tok_lo, tok_hi, watch_out)
+    _check(lib().spd_decode_step_watch(C.byref(shape), q.data_ptr(), C.byref(a), C.byref(b), out.data_ptr(),
+                                       _dtype_code(out.dtype), C.byref(w), ws.data_ptr(), ws.numel(),
+                                       _stream_ptr(stream)), "spd_decode_step_watch")

@@ -200,6 +200,7 @@ struct Job {
     spd_dtype out_dtype;
     int32_t epoch;                 // id of the call (both halves of a chained step share one)
     int32_t *status_words;         // where the kernel raises its status; null = the workspace header
+    const spd_watch *watch;        // optional monitor of a private token range
 };
 
 spd_status run_job(const Job &job, void *ws, size_t ws_bytes, void *stream) {
@@ -237,6 +238,7 @@ spd_status run_job(const Job &job, void *ws, size_t ws_bytes, void *stream) {
     if (job.pin) { p.in_o = job.pin->o; p.in_m = job.pin->m; p.in_l = job.pin->l; }
     p.out = job.out;
     p.out_bf16 = job.out_dtype == SPD_BF16;
+    if (job.watch) { p.watch_lo = job.watch->tok_lo; p.watch_hi = job.watch->tok_hi; p.watch_out = job.watch->out; }
 
     CUtensorMap maps[4];
     int have = -1;
@@ -365,6 +367,44 @@ spd_status spd_decode_step(const spd_shape *shape, const void *q, const spd_page
     a.epoch = b.epoch = next_epoch();
     if ((rc = run_job(a, ws, ws_bytes, cuda_stream)) != SPD_OK) return rc;
     return run_job(b, ws, ws_bytes, cuda_stream);
+}
+
+static spd_status check_watch(const spd_watch *w) {
+    if (!w || !w->tok_lo || !w->tok_hi || !w->out) return SPD_ERR_INVALID_ARG;
+    return SPD_OK;
+}
+
+spd_status spd_partial_attn_watch(const spd_shape *shape, const void *q, const spd_paged_kv *priv, spd_partial out,
+                                  const spd_watch *watch, void *ws, size_t ws_bytes, void *cuda_stream) {
+    spd_status rc = check_shape(shape);
+    if (rc != SPD_OK) return rc;
+    if ((rc = check_kv(shape, priv)) != SPD_OK) return rc;
+    if ((rc = check_watch(watch)) != SPD_OK) return rc;
+    if (!out.o || !out.m || !out.l || misaligned(out.o, 16)) return SPD_ERR_INVALID_ARG;
+    Job job{};
+    job.shape = shape; job.q = q; job.part[0] = priv;
+    job.mode = OUT_PARTIAL; job.pout = out; job.out_dtype = SPD_F32;
+    job.epoch = next_epoch();
+    job.watch = watch;
+    return run_job(job, ws, ws_bytes, cuda_stream);
+}
+
+spd_status spd_decode_step_watch(const spd_shape *shape, const void *q, const spd_paged_kv *priv,
+                                 const spd_paged_kv *pub, void *out, spd_dtype out_dtype, const spd_watch *watch,
+                                 void *ws, size_t ws_bytes, void *cuda_stream) {
+    spd_status rc = check_shape(shape);
+    if (rc != SPD_OK) return rc;
+    if ((rc = check_kv(shape, priv)) != SPD_OK) return rc;
+    if ((rc = check_kv(shape, pub)) != SPD_OK) return rc;
+    if ((rc = check_watch(watch)) != SPD_OK) return rc;
+    if (!out || misaligned(out, 16)) return SPD_ERR_INVALID_ARG;
+    if (out_dtype != SPD_F32 && out_dtype != SPD_BF16) return SPD_ERR_UNSUPPORTED;
+    Job job{};
+    job.shape = shape; job.q = q; job.part[0] = priv; job.part[1] = pub;
+    job.mode = OUT_FINAL; job.out = out; job.out_dtype = out_dtype;
+    job.epoch = next_epoch();
+    job.watch = watch;
+    return run_job(job, ws, ws_bytes, cuda_stream);
 }
 
 spd_status spd_append_kv(const spd_shape *shape, const void *k_new, const void *v_new, void *k_pool, void *v_pool,

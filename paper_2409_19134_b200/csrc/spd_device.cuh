@@ -58,6 +58,9 @@ struct Params {
     const float *in_o, *in_m, *in_l;  // OUT_FINAL: optional partial to merge in (may be null)
     void *out;              // OUT_FINAL destination
     int32_t out_bf16;
+    // optional monitor: softmax mass on tokens [watch_lo[u], watch_hi[u]) of the private partition
+    const int32_t *watch_lo, *watch_hi;   // [B]
+    float *watch_out;                      // [B][Hq]; null = not watching
 };
 
 // ---------------------------------------------------------------------------------------------

@@ -71,7 +71,7 @@ __device__ __forceinline__ bool user_tiles(const Params &p, int u, int &n0, int 
 // Each lane holds V = D/32 consecutive channels of O; m and l are warp-uniform.
 template <int D>
 __device__ __forceinline__ void finalize_store(const Params &p, int u, int h, float (&o)[D / 32], float m, float l,
-                                               int lane, bool bad) {
+                                               int lane, bool bad, float lw = 0.f) {
     constexpr int V = D / 32;
     const int64_t idx = static_cast<int64_t>(u) * p.Hq + h;
     if (p.mode == OUT_PARTIAL) {
@@ -84,10 +84,15 @@ __device__ __forceinline__ void finalize_store(const Params &p, int u, int h, fl
         float *dst = p.po + idx * D + lane * V;
         if constexpr (V == 4) *reinterpret_cast<float4 *>(dst) = make_float4(o[0], o[1], o[2], o[3]);
         else *reinterpret_cast<float2 *>(dst) = make_float2(o[0], o[1]);
-        if (lane == 0) { p.pm[idx] = m; p.pl[idx] = l; }
+        if (lane == 0) {
+            p.pm[idx] = m;
+            p.pl[idx] = l;
+            if (p.watch_out) p.watch_out[idx] = bad ? 0.f : lw;   // same gauge as l: relative to m
+        }
         return;
     }
     float L = l;
+    float wself = 1.f;   // weight of this side after the merge with an incoming partial
     if (p.in_o != nullptr) {
         const float mi = p.in_m[idx], li = p.in_l[idx];
         const float M = fmaxf(m, mi);
@@ -98,10 +103,12 @@ __device__ __forceinline__ void finalize_store(const Params &p, int u, int h, fl
         if constexpr (V == 4) { float4 t = *reinterpret_cast<const float4 *>(src); oi[0] = t.x; oi[1] = t.y; oi[2] = t.z; oi[3] = t.w; }
         else { float2 t = *reinterpret_cast<const float2 *>(src); oi[0] = t.x; oi[1] = t.y; }
         L = w * l + wi * li;
+        wself = w;
 #pragma unroll
         for (int i = 0; i < V; ++i) o[i] = w * o[i] + wi * oi[i];
     }
     const float inv = (L > 0.f && !bad) ? 1.f / L : 0.f;
+    if (p.watch_out && lane == 0) p.watch_out[idx] = wself * lw * inv;   // share of the full softmax mass
 #pragma unroll
     for (int i = 0; i < V; ++i) o[i] = (inv == 0.f) ? 0.f : o[i] * inv;
     if (p.out_bf16) {
@@ -116,7 +123,7 @@ __device__ __forceinline__ void finalize_store(const Params &p, int u, int h, fl
     }
 }
 
-__host__ __device__ constexpr int slot_floats(int D) { return kHeadsPerItem * D + 16; }   // O[8][D], m[8], l[8]
+__host__ __device__ constexpr int slot_floats(int D) { return kHeadsPerItem * D + 24; }   // O[8][D], m[8], l[8], watched l[8]
 
 __device__ __forceinline__ int first_head(const Params &p, int sq) {
     const int kvh = sq / p.hgroups, hg = sq - kvh * p.hgroups;
@@ -148,11 +155,12 @@ template <int D, int GE>
 __device__ __noinline__ void merge_pieces(const Params &p, int u, int sq, int w_first, int w_last, const int32_t *bnd,
                                           int s0, int lane, bool bad) {
     constexpr int V = D / 32, H = kHeadsPerItem, PB = 16 / GE;   // PB pieces per batch of loads
-    float M[GE], L[GE], o[GE][V];
+    float M[GE], L[GE], LW[GE], o[GE][V];
 #pragma unroll
     for (int hh = 0; hh < GE; ++hh) {
         M[hh] = -INFINITY;
         L[hh] = 0.f;
+        LW[hh] = 0.f;
 #pragma unroll
         for (int i = 0; i < V; ++i) o[hh][i] = 0.f;
     }
@@ -165,16 +173,21 @@ __device__ __noinline__ void merge_pieces(const Params &p, int u, int sq, int w_
         for (int hh = 0; hh < GE; ++hh) {
             const float mc = mine ? __ldcg(ms + hh) : -INFINITY;
             const float lc = mine ? __ldcg(ms + H + hh) : 0.f;
+            const float lwc = (mine && p.watch_out) ? __ldcg(ms + 2 * H + hh) : 0.f;
             float mb = mc;
 #pragma unroll
             for (int d = 16; d >= 1; d >>= 1) mb = fmaxf(mb, __shfl_xor_sync(0xffffffffu, mb, d));
             const float Mn = fmaxf(M[hh], mb);
             const float resc = (M[hh] == -INFINITY) ? 0.f : expf(M[hh] - Mn);
             wgt[hh] = (mc == -INFINITY) ? 0.f : expf(mc - Mn);
-            float ls = wgt[hh] * lc;
+            float ls = wgt[hh] * lc, lws = wgt[hh] * lwc;
 #pragma unroll
-            for (int d = 16; d >= 1; d >>= 1) ls += __shfl_xor_sync(0xffffffffu, ls, d);
+            for (int d = 16; d >= 1; d >>= 1) {
+                ls += __shfl_xor_sync(0xffffffffu, ls, d);
+                lws += __shfl_xor_sync(0xffffffffu, lws, d);
+            }
             L[hh] = L[hh] * resc + ls;
+            LW[hh] = LW[hh] * resc + lws;
             M[hh] = Mn;
 #pragma unroll
             for (int i = 0; i < V; ++i) o[hh][i] *= resc;
@@ -211,10 +224,11 @@ __device__ __noinline__ void merge_pieces(const Params &p, int u, int sq, int w_
     }
     const int hbase = first_head(p, sq);
 #pragma unroll
-    for (int hh = 0; hh < GE; ++hh) finalize_store<D>(p, u, hbase + hh, o[hh], M[hh], L[hh], lane, bad);
+    for (int hh = 0; hh < GE; ++hh) finalize_store<D>(p, u, hbase + hh, o[hh], M[hh], L[hh], lane, bad, LW[hh]);
 }
 
-// A finished segment sits in shared memory as So[8][D+4], Sm[8], Sl[8].  A segment that is a whole
+// A finished segment sits in shared memory as So[8][D+4], Sm[8], Sl[8], Sw[8] (Sw = watched part of l,
+// right behind Sl).  A segment that is a whole
 // sequence is finalised on the spot (the warp has seen every page of it, so `bad` is complete).
 template <int D>
 __device__ __forceinline__ void finalize_segment(const Params &p, const float *So, const float *Sm, const float *Sl,
@@ -225,7 +239,7 @@ __device__ __forceinline__ void finalize_segment(const Params &p, const float *S
         float o[V];
 #pragma unroll
         for (int i = 0; i < V; ++i) o[i] = So[hh * PITCH + lane * V + i];
-        finalize_store<D>(p, u, hbase + hh, o, Sm[hh], Sl[hh], lane, bad);
+        finalize_store<D>(p, u, hbase + hh, o, Sm[hh], Sl[hh], lane, bad, Sl[kHeadsPerItem + hh]);
     }
 }
 
@@ -247,6 +261,7 @@ __device__ __forceinline__ void piece_store(const Params &p, const float *So, co
     if (lane < 8) {
         __stcg(dst + kHeadsPerItem * D + lane, Sm[lane]);
         __stcg(dst + kHeadsPerItem * D + 8 + lane, Sl[lane]);
+        __stcg(dst + kHeadsPerItem * D + 16 + lane, Sl[kHeadsPerItem + lane]);
     }
 }
 
@@ -308,6 +323,8 @@ struct MathBF16 {
         uint32_t qf[KS][2];
         float o[KS][4];
         float m, l;
+        float lw;          // part of l that came from the watched token range
+        int wlo, whi;      // watched range of the private partition, [wlo, whi); empty = not watching
     };
 
     __device__ static __forceinline__ void begin(State &st, const Params &p, int u, int sq, int lane, uint8_t *) {
@@ -329,10 +346,15 @@ struct MathBF16 {
             for (int i = 0; i < 4; ++i) st.o[mt][i] = 0.f;
         st.m = -INFINITY;
         st.l = 0.f;
+        st.lw = 0.f;
+        st.wlo = p.watch_out ? p.watch_lo[u] : 0;
+        st.whi = p.watch_out ? p.watch_hi[u] : 0;
     }
 
+    // watch_base: index within the private partition of the tile's first token (hugely negative for
+    // a tile of the public partition, so that nothing of it counts as watched)
     __device__ static __forceinline__ void tile(State &st, const Params &p, uint8_t *Ks, uint8_t *Vs, int valid,
-                                                int lane, uint8_t *) {
+                                                int lane, uint8_t *, int watch_base) {
         const int mat = lane >> 3, r = lane & 7;
         const int tok = ((mat >> 1) << 3) + r;
         const uint32_t lane_off = tok * 128;
@@ -376,6 +398,14 @@ struct MathBF16 {
         const float p2 = ex2_approx((v2 - m_new) * kLog2e), p3 = ex2_approx((v3 - m_new) * kLog2e);
         st.l = st.l * alpha + ((p0 + p1) + (p2 + p3));
         st.m = m_new;
+        if (st.whi > st.wlo) {   // warp-uniform
+            const int t0 = watch_base + tk;
+            float w = (t0 >= st.wlo && t0 < st.whi) ? p0 : 0.f;
+            w += (t0 + 1 >= st.wlo && t0 + 1 < st.whi) ? p1 : 0.f;
+            w += (t0 + 8 >= st.wlo && t0 + 8 < st.whi) ? p2 : 0.f;
+            w += (t0 + 9 >= st.wlo && t0 + 9 < st.whi) ? p3 : 0.f;
+            st.lw = st.lw * alpha + w;
+        }
         const uint32_t bh0 = pack_bf16(p0, p1), bh1 = pack_bf16(p2, p3);
         const __nv_bfloat162 h0 = *reinterpret_cast<const __nv_bfloat162 *>(&bh0);
         const __nv_bfloat162 h1 = *reinterpret_cast<const __nv_bfloat162 *>(&bh1);
@@ -408,10 +438,12 @@ struct MathBF16 {
             So[hd * PITCH + mt * 16 + dr + 8] = st.o[mt][2];
             So[(hd + 1) * PITCH + mt * 16 + dr + 8] = st.o[mt][3];
         }
-        float l = st.l;
+        float l = st.l, lw = st.lw;
         l += __shfl_xor_sync(0xffffffffu, l, 1);
         l += __shfl_xor_sync(0xffffffffu, l, 2);
-        if ((lane & 3) == 0) { Sm[lane >> 2] = st.m; Sl[lane >> 2] = l; }
+        lw += __shfl_xor_sync(0xffffffffu, lw, 1);
+        lw += __shfl_xor_sync(0xffffffffu, lw, 2);
+        if ((lane & 3) == 0) { Sm[lane >> 2] = st.m; Sl[lane >> 2] = l; Sl[kHeadsPerItem + (lane >> 2)] = lw; }
     }
 };
 
@@ -435,7 +467,8 @@ struct MathF32 {
 
     struct State {
         float o[GE][V];
-        float m[GE], l[GE];
+        float m[GE], l[GE], lw[GE];
+        int wlo, whi;
     };
 
     __device__ static __forceinline__ void begin(State &st, const Params &p, int u, int sq, int lane, uint8_t *extra) {
@@ -452,11 +485,14 @@ struct MathF32 {
             for (int i = 0; i < V; ++i) st.o[hh][i] = 0.f;
             st.m[hh] = -INFINITY;
             st.l[hh] = 0.f;
+            st.lw[hh] = 0.f;
         }
+        st.wlo = p.watch_out ? p.watch_lo[u] : 0;
+        st.whi = p.watch_out ? p.watch_hi[u] : 0;
     }
 
     __device__ static __forceinline__ void tile(State &st, const Params &p, uint8_t *Ks, uint8_t *Vs, int valid,
-                                                int lane, uint8_t *extra) {
+                                                int lane, uint8_t *extra, int watch_base) {
         const float *qs = reinterpret_cast<const float *>(extra);
         float *Ps = reinterpret_cast<float *>(extra) + kHeadsPerItem * D;
         const int t = lane & 15, hf = lane >> 4;
@@ -490,6 +526,7 @@ struct MathF32 {
             const float alpha = exp2f((st.m[hh] - m_new) * kLog2e);
             const float pr = exp2f((v - m_new) * kLog2e);
             st.l[hh] = st.l[hh] * alpha + (hf == 0 ? pr : 0.f);
+            st.lw[hh] = st.lw[hh] * alpha + ((hf == 0 && watch_base + t >= st.wlo && watch_base + t < st.whi) ? pr : 0.f);
             st.m[hh] = m_new;
 #pragma unroll
             for (int i = 0; i < V; ++i) st.o[hh][i] *= alpha;
@@ -516,16 +553,19 @@ struct MathF32 {
         for (int hh = 0; hh < GE; ++hh) {
 #pragma unroll
             for (int i = 0; i < V; ++i) So[hh * PITCH + lane * V + i] = st.o[hh][i];
-            float l = st.l[hh];
+            float l = st.l[hh], lw = st.lw[hh];
 #pragma unroll
-            for (int d = 8; d >= 1; d >>= 1) l += __shfl_xor_sync(0xffffffffu, l, d);
-            if (lane == 0) { Sm[hh] = st.m[hh]; Sl[hh] = l; }
+            for (int d = 8; d >= 1; d >>= 1) {
+                l += __shfl_xor_sync(0xffffffffu, l, d);
+                lw += __shfl_xor_sync(0xffffffffu, lw, d);
+            }
+            if (lane == 0) { Sm[hh] = st.m[hh]; Sl[hh] = l; Sl[kHeadsPerItem + hh] = lw; }
         }
         // rows beyond GE are never read by a complete segment, but a piece copies all 8 rows
         for (int hh = GE; hh < kHeadsPerItem; ++hh) {
 #pragma unroll
             for (int i = 0; i < V; ++i) So[hh * PITCH + lane * V + i] = 0.f;
-            if (lane == 0) { Sm[hh] = -INFINITY; Sl[hh] = 0.f; }
+            if (lane == 0) { Sm[hh] = -INFINITY; Sl[hh] = 0.f; Sl[kHeadsPerItem + hh] = 0.f; }
         }
     }
 };
@@ -604,7 +644,7 @@ attn_kernel(const __grid_constant__ Params p, const __grid_constant__ CUtensorMa
     constexpr int D = Math::D, NS = Math::kStages, TB = Math::kTileBytes, NT = Math::kWarps * 32;
     static_assert(TB % 1024 == 0, "swizzled tiles need 1024-byte aligned bases");
     static_assert(Math::kExtraBytes % 16 == 0, "per-warp extra area holds float4 data");
-    static_assert(2 * TB >= (kHeadsPerItem * (D + 4) + 2 * kHeadsPerItem) * 4, "a stage must hold the epilogue staging");
+    static_assert(2 * TB >= (kHeadsPerItem * (D + 4) + 3 * kHeadsPerItem) * 4, "a stage must hold the epilogue staging");
     static_assert(attn_smem_bytes<Math>(kMaxGrid) + 16384 <= 227 * 1024, "ring does not fit shared memory");
     static_assert(Math::kWarps <= 16 && Math::kStages >= 2, "CTA shape");
     extern __shared__ uint8_t smem_raw[];
@@ -827,7 +867,7 @@ attn_kernel(const __grid_constant__ Params p, const __grid_constant__ CUtensorMa
         if (page < 0 || page >= p.part[part].num_pages) valid = 0;   // never fetched; flagged when consumed
         if (lane == 0) {
             descs[2 * stage] = make_int4(valid, (first ? 1 : 0) | (last ? 2 : 0) | (kind << 8), c.u, c.sq);
-            descs[2 * stage + 1] = make_int4(c.np, c.j, cur_t, 0);
+            descs[2 * stage + 1] = make_int4(c.np, c.j, cur_t, c.npp);
             const uint32_t bar = smem_u32(&bars[stage]);
             if (valid == 0) {
                 mbar_arrive(bar);
@@ -870,15 +910,15 @@ attn_kernel(const __grid_constant__ Params p, const __grid_constant__ CUtensorMa
         const int4 d = descs[2 * stage];
         uint8_t *Ks = ring + static_cast<size_t>(stage) * 2 * TB, *Vs = Ks + TB;
         if (d.y & 1) { Math::begin(st, p, d.z, d.w, lane, extra); seg_bad = false; }
+        const int4 e = descs[2 * stage + 1];
         if (d.x > 0) {
-            Math::tile(st, p, Ks, Vs, d.x, lane, extra);
+            Math::tile(st, p, Ks, Vs, d.x, lane, extra, e.y < e.w ? e.y * kPage : -(1 << 30));
         } else {                                   // a page index outside the pool: flag the user, skip the tile
             seg_bad = true;
             if (lane == 0) { p.bad[d.z] = p.epoch; flag_error(p.hdr, 4 /* SPD_ERR_BAD_PAGE */, d.z); }
         }
         if (d.y & 2) {
             // the stage just consumed doubles as the staging area of the epilogue
-            const int4 e = descs[2 * stage + 1];
             __syncwarp();
             float *So = reinterpret_cast<float *>(Ks);
             float *Sm = So + kHeadsPerItem * (D + 4), *Sl = Sm + kHeadsPerItem;

@@ -227,3 +227,43 @@ def test_append_kv_is_bit_exact_and_feeds_the_next_step(dtype):
     spd.spd_decode_step(shape, wg.q, wg.priv, wg.pub, out, ws, fused=True)
     assert spd.spd_query_device_status(ws) == (spd.SPD_OK, -1)
     assert_close(out.cpu().numpy(), orc.full(q, kin, kout, w.sm_scale), w.dtype, "decode after append")
+
+
+@pytest.mark.parametrize("name", ["bf16_gqa4_d128", "bf16_gqa8_d128", "bf16_long_split", "f32_mha_d64", "f32_long_split"])
+def test_watched_attention_mass(name):
+    """The input-attention monitor: softmax mass on a watched range of the private partition."""
+    w = wl.make_workload(dict(SMALL[name], name=name), slack=True)
+    rng = np.random.default_rng(61)
+    lin = w.priv.seq_lens.numpy()
+    lo = np.array([rng.integers(0, max(1, n)) for n in lin])
+    hi = np.array([rng.integers(l, n + 40) for l, n in zip(lo, lin)])       # some reach past the partition
+    if w.batch > 2:
+        hi[0], lo[1], hi[1] = lo[0], 5, 2                                    # an empty and an inverted interval
+    q, kin, kout = oracle_inputs(w)
+    ref = orc.full(q, kin, kout, w.sm_scale)
+    full_ref, own_ref = orc.watched_mass(q, kin, kout, w.sm_scale, lo, hi)
+    wg = w.to("cuda")
+    shape = spd.make_shape(w.batch, w.num_q_heads, w.num_kv_heads, w.head_dim, w.dtype, w.sm_scale)
+    ws = spd.alloc_workspace(shape)
+    tlo = torch.tensor(lo, dtype=torch.int32, device="cuda")
+    thi = torch.tensor(hi, dtype=torch.int32, device="cuda")
+    mass = torch.full((w.batch, w.num_q_heads), float("nan"), dtype=torch.float32, device="cuda")
+    out = torch.full((w.batch, w.num_q_heads, w.head_dim), float("nan"), dtype=torch.float32, device="cuda")
+    tol = TOL[w.dtype][0]
+    for _ in range(2):
+        spd.spd_decode_step_watch(shape, wg.q, wg.priv, wg.pub, out, tlo, thi, mass, ws)
+        assert spd.spd_query_device_status(ws) == (spd.SPD_OK, -1)
+        assert_close(out.cpu().numpy(), ref, w.dtype, f"{name} output with the monitor on")
+        got = mass.cpu().numpy().astype(np.float64)
+        assert np.all(np.isfinite(got)) and np.max(np.abs(got - full_ref)) <= tol, np.max(np.abs(got - full_ref))
+    part = spd.alloc_partial(shape)
+    lw = torch.full((w.batch, w.num_q_heads), float("nan"), dtype=torch.float32, device="cuda")
+    spd.spd_partial_attn_watch(shape, wg.q, wg.priv, part, tlo, thi, lw, ws)
+    assert spd.spd_query_device_status(ws) == (spd.SPD_OK, -1)
+    l = part[2].cpu().numpy().astype(np.float64)
+    share = np.divide(lw.cpu().numpy().astype(np.float64), l, out=np.zeros_like(l), where=l > 0)
+    assert np.max(np.abs(share - own_ref)) <= tol
+    # the unwatched calls give the same attention output
+    out2 = torch.empty_like(out)
+    spd.spd_decode_step(shape, wg.q, wg.priv, wg.pub, out2, ws, fused=True)
+    assert float((out2 - out).abs().max()) <= 2 * tol

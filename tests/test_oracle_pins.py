@@ -365,3 +365,37 @@ def test_append_then_attend_equals_dense_concatenation():
     for u in (0, 3):
         pages = kv.page_indices[kv.page_indptr[u]:kv.page_indptr[u + 1]]
         assert np.array_equal(np.nan_to_num(kv.k_pool[pages]), np.nan_to_num(snap[0][pages]))
+
+
+# ---------------------------------------------------------------- watched attention mass (Sec. 2.4.4)
+def test_watched_mass_is_the_sum_of_softmax_probabilities():
+    rng = np.random.default_rng(31)
+    B, Hkv, Hq, D = 3, 2, 4, 8
+    lin, lout = [40, 7, 16], [9, 0, 3]
+    ks, vs = _rand_dense(rng, lin, Hkv, D)
+    ko, vo = _rand_dense(rng, lout, Hkv, D)
+    kin, kout = dense_to_paged(ks, vs, rng=rng), dense_to_paged(ko, vo, rng=rng)
+    q = rng.standard_normal((B, Hq, D)).astype(np.float32)
+    lo, hi = np.array([5, 0, 16]), np.array([23, 7, 30])     # the last range lies past the partition: watches nothing
+    full, own = orc.watched_mass(q, kin, kout, 0.6, lo, hi)
+    for u in range(B):
+        for h in range(Hq):
+            K = np.concatenate([ks[u][h // 2], ko[u][h // 2]]).astype(np.float64)
+            s = 0.6 * K @ q[u, h].astype(np.float64)
+            pr = np.exp(s - s.max())
+            pr /= pr.sum()
+            a, b = min(lo[u], lin[u]), min(hi[u], lin[u])
+            assert abs(full[u, h] - pr[a:b].sum()) < 1e-12
+            pin = np.exp(s[:lin[u]] - s[:lin[u]].max())
+            pin /= pin.sum()
+            assert abs(own[u, h] - pin[a:b].sum()) < 1e-12
+    # the whole private partition with no public tokens holds all the mass; disjoint ranges add up
+    f1, o1 = orc.watched_mass(q, kin, None, 0.6, np.zeros(B), np.array(lin))
+    assert np.allclose(f1, 1.0, atol=1e-12) and np.allclose(o1, 1.0, atol=1e-12)
+    fa, _ = orc.watched_mass(q, kin, kout, 0.6, np.zeros(B), np.array([20, 3, 8]))
+    fb, _ = orc.watched_mass(q, kin, kout, 0.6, np.array([20, 3, 8]), np.array(lin))
+    fall, _ = orc.watched_mass(q, kin, kout, 0.6, np.zeros(B), np.array(lin))
+    assert np.allclose(fa + fb, fall, atol=1e-12)
+    # uniform scores: the share is the fraction of tokens watched
+    fu, ou = orc.watched_mass(np.zeros_like(q), kin, kout, 0.6, np.array([2, 2, 2]), np.array([12, 5, 10]))
+    assert np.allclose(fu[:, 0], [10 / 49, 3 / 7, 8 / 19], atol=1e-12) and np.allclose(ou[:, 0], [10 / 40, 3 / 7, 8 / 16], atol=1e-12)
