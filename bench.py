@@ -234,8 +234,10 @@ def time_e2e(spd, w, shape, ws, steps, warmup):
     devb = torch.empty(lay.total_bytes, dtype=torch.uint8, device=dev)
     pools = [(w.priv.k_pool, w.priv.v_pool), (w.pub.k_pool, w.pub.v_pool)]
 
+    step = spd.HostStep(shape, lay, host, devb, pools[0], pools[1], torch.float32, ws)
+
     def call():
-        code, bad = spd.spd_decode_step_host(shape, lay, host, devb, pools[0], pools[1], torch.float32, ws)
+        code, bad = step()
         if code != spd.SPD_OK:
             raise RuntimeError(f"host-buffer step failed: status {code}, user {bad}")
     for _ in range(warmup):

@@ -197,6 +197,27 @@ def spd_decode_step_host(shape, layout, host_blob, device_blob, priv_pools, pub_
     return int(code), int(bad.value)
 
 
+class HostStep:
+    """spd_decode_step_host with its arguments marshalled once: for a serving loop that reuses the same
+    buffers every step and only rewrites the host blob.  Calling the object runs one step."""
+
+    def __init__(self, shape, layout, host_blob, device_blob, priv_pools, pub_pools, out_dtype, ws, stream=None):
+        self._keep = (shape, layout, host_blob, device_blob, priv_pools, pub_pools, ws)   # keep the memory alive
+        self._a = PagedKV(_ptr(priv_pools[0]), _ptr(priv_pools[1]), int(priv_pools[0].shape[0]), None, None, None)
+        self._b = PagedKV(_ptr(pub_pools[0]), _ptr(pub_pools[1]), int(pub_pools[0].shape[0]), None, None, None)
+        self._bad = C.c_int32(-1)
+        self._fn = lib().spd_decode_step_host
+        self._args = (C.byref(shape), C.byref(layout), C.c_void_p(host_blob.data_ptr()), C.c_void_p(device_blob.data_ptr()),
+                      C.byref(self._a), C.byref(self._b), _dtype_code(out_dtype), C.byref(self._bad),
+                      C.c_void_p(ws.data_ptr()), C.c_size_t(ws.numel()), C.c_void_p(_stream_ptr(stream)))
+
+    def __call__(self) -> Tuple[int, int]:
+        code = self._fn(*self._args)
+        if code not in (SPD_OK, 4, 6):
+            raise SpdError(code, "spd_decode_step_host")
+        return int(code), int(self._bad.value)
+
+
 def fill_step_blob(layout, host_blob, q, priv, pub) -> None:
     """Copy q and the two partitions' tables (any device) into a host blob at the layout's offsets."""
     def put(off, t):

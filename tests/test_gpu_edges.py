@@ -162,6 +162,11 @@ def test_host_blob_step_matches_oracle(name):
         assert spd.spd_decode_step_host(shape, lay, host, devb, pools[0], pools[1], torch.float32, ws) == (spd.SPD_OK, -1)
         out = host[lay.out:lay.out + 4 * n].view(torch.float32).reshape(w.batch, w.num_q_heads, w.head_dim)
         assert_close(out.numpy(), ref, w.dtype, f"{name} host blob")
+    step = spd.HostStep(shape, lay, host, devb, pools[0], pools[1], torch.float32, ws)   # marshalled once
+    host[lay.out:] = 0xFF
+    assert step() == (spd.SPD_OK, -1)
+    assert_close(host[lay.out:lay.out + 4 * n].view(torch.float32).reshape(w.batch, w.num_q_heads, w.head_dim).numpy(),
+                 ref, w.dtype, f"{name} prepared host step")
     # a page index outside the pool, planted in the host blob: reported, contained, cleared
     idx = host[lay.priv_indices:lay.priv_indices + 4 * w.priv.page_indices.numel()].view(torch.int32)
     keep = int(idx[int(w.priv.page_indptr[1])])
