@@ -301,6 +301,7 @@ def run_cuda(args):
     w = wl.make_workload(cfg, device=dev)     # every rank: its own replica of the same seeded workload
     kvb = w.kv_bytes()
     spd.lib()
+    spd.spd_set_bf16_math(1 if args.bf16_math == "fma" else 0)
 
     def barrier():
         if world > 1:
@@ -333,7 +334,7 @@ def run_cuda(args):
         "dtype": "bf16" if w.dtype == torch.bfloat16 else "f32", "data": "synthetic",
         "config": {"workload": cfg, "users": w.batch, "q_heads": w.num_q_heads, "kv_heads": w.num_kv_heads,
                    "head_dim": w.head_dim, "page_size": w.page_size, "kv_bytes_per_step": kvb,
-                   "parallelism": "replicas only" if world > 1 else "single GPU", "call": "spd_decode_step(fused=1)",
+                   "parallelism": "replicas only" if world > 1 else "single GPU", "call": "spd_decode_step(fused=1)", "bf16_math": args.bf16_math,
                    "l2": "inputs larger than L2 (KV bytes per step >> 126 MB); no flush"},
         "user_tokens_per_s": world * w.batch / ms_max * 1e3,
         "pct_of_nominal_hbm_8000": 100.0 * value / world / NOMINAL_HBM_GBS,
@@ -389,6 +390,8 @@ def main():
     ap.add_argument("--config", default="c2_llama2_7b", choices=list(wl.CONFIGS))
     ap.add_argument("--impl", default="cuda", choices=["cuda", "reference"])
     ap.add_argument("--no-extras", action="store_true", help="skip the other configs and the CPU baseline")
+    ap.add_argument("--bf16-math", default="mma", choices=["mma", "fma"],
+                    help="arithmetic of the bf16 kernels: tensor cores (default) or the FMA-pipe comparison arm")
     args = ap.parse_args()
     if args.impl == "reference":
         run_reference(args)

@@ -240,6 +240,14 @@ spd_status spd_decode_step_static(const spd_shape *shape, const void *q, const s
                                   const spd_paged_kv *pub, void *out, spd_dtype out_dtype,
                                   int32_t wait_and_check, int32_t *first_bad_user, void *cuda_stream);
 
+/*
+ * Measurement aid (no counterpart in the paper): which arithmetic the bf16 kernels use from now on,
+ * process-wide.  0 (default) = tensor cores (mma.sync, fp32 accumulate); 1 = the FMA pipes with K and V
+ * widened to fp32 on the fly.  Same tiles, same memory traffic, same results within tolerance; path 1
+ * exists to show where the tensor cores are needed (it falls behind HBM as the GQA group grows).
+ */
+spd_status spd_set_bf16_math(int32_t path);
+
 /* Static text for a status code. */
 const char *spd_status_string(spd_status status);
 

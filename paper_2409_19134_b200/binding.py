@@ -22,7 +22,7 @@ EXPORTS = ["spd_workspace_size", "spd_partial_attn", "spd_service_attn_merge", "
            "spd_step_blob_layout", "spd_decode_step_host", "spd_query_device_status",
            "spd_kernel_launch_count", "spd_status_string", "spd_profile_begin", "spd_profile_end",
            "spd_decode_step_static", "spd_append_kv",
-           "spd_partial_attn_watch", "spd_decode_step_watch"]
+           "spd_partial_attn_watch", "spd_decode_step_watch", "spd_set_bf16_math"]
 
 
 class SpdError(RuntimeError):
@@ -86,6 +86,7 @@ def lib() -> C.CDLL:
         L.spd_partial_attn_watch.argtypes = [C.POINTER(Shape), vp, C.POINTER(PagedKV), Partial, C.POINTER(Watch), vp, sz, vp]
         L.spd_decode_step_watch.argtypes = [C.POINTER(Shape), vp, C.POINTER(PagedKV), C.POINTER(PagedKV), vp, C.c_int,
                                             C.POINTER(Watch), vp, sz, vp]
+        L.spd_set_bf16_math.argtypes = [C.c_int32]
         L.spd_append_kv.argtypes = [C.POINTER(Shape), vp, vp, vp, vp, C.c_int32, vp, vp, vp, vp, sz, vp]
         for name in EXPORTS[:7] + EXPORTS[9:]:
             getattr(L, name).restype = C.c_int
@@ -298,3 +299,8 @@ def spd_decode_step_watch(shape, q, priv, pub, out, tok_lo, tok_hi, watch_out, w
     _check(lib().spd_decode_step_watch(C.byref(shape), q.data_ptr(), C.byref(a), C.byref(b), out.data_ptr(),
                                        _dtype_code(out.dtype), C.byref(w), ws.data_ptr(), ws.numel(),
                                        _stream_ptr(stream)), "spd_decode_step_watch")
+
+
+def spd_set_bf16_math(path: int) -> None:
+    """0 = tensor cores (default), 1 = FMA pipes (comparison arm); process-wide."""
+    _check(lib().spd_set_bf16_math(int(path)), "spd_set_bf16_math")

@@ -30,6 +30,7 @@ void prof_mark(int job, int k, cudaStream_t st) {
 }
 
 std::atomic<uint32_t> g_epoch{0};
+std::atomic<int> g_bf16_math{0};   // 0 = tensor cores (default), 1 = FMA pipes (comparison arm)
 
 // Ids of calls: non-zero, so that a zeroed workspace matches none.
 int32_t next_epoch() {
@@ -157,8 +158,10 @@ spd_status make_map(CUtensorMap *map, const spd_shape &s, const void *pool, int6
 }
 
 template <class Math>
-spd_status launch_attn(const Params &p, const CUtensorMap *maps, int sms, cudaStream_t st) {
+spd_status launch_attn(const Params &p_in, const CUtensorMap *maps, int sms, cudaStream_t st) {
     if (sms > kMaxGrid) return SPD_ERR_UNSUPPORTED;
+    Params p = p_in;
+    p.num_warps = sms * Math::kWarps;   // the plan cuts the tile stream into one share per warp of THIS grid
     const size_t smem = attn_smem_bytes<Math>(sms);
     static std::once_flag once[64];
     int dev = 0;
@@ -224,8 +227,6 @@ spd_status run_job(const Job &job, void *ws, size_t ws_bytes, void *stream) {
     p.sm_scale = s.sm_scale;
     p.q = job.q;
     const bool bf = s.dtype == SPD_BF16;
-    const int warps_per_cta = bf ? MathBF16<128>::kWarps : MathF32<128, 1>::kWarps;
-    p.num_warps = di.sms * warps_per_cta;
     p.hdr = job.status_words ? job.status_words : reinterpret_cast<int32_t *>(w + L.hdr);
     p.bad = reinterpret_cast<int32_t *>(w + L.bad);
     p.tickets = reinterpret_cast<int32_t *>(w + L.tickets);
@@ -274,7 +275,12 @@ spd_status run_job(const Job &job, void *ws, size_t ws_bytes, void *stream) {
     }
     prof_mark(pj, 0, st);
     const int D = s.head_dim;
-    if (bf) {
+    if (bf && g_bf16_math.load() == 1) {
+#define SPD_SIMT_CASE(DD, GG) if (D == DD && p.geff == GG) rc = launch_attn<MathBF16Simt<DD, GG>>(p, maps, di.sms, st);
+        SPD_SIMT_CASE(64, 1) SPD_SIMT_CASE(64, 2) SPD_SIMT_CASE(64, 4) SPD_SIMT_CASE(64, 8)
+        SPD_SIMT_CASE(128, 1) SPD_SIMT_CASE(128, 2) SPD_SIMT_CASE(128, 4) SPD_SIMT_CASE(128, 8)
+#undef SPD_SIMT_CASE
+    } else if (bf) {
         rc = D == 128 ? launch_attn<MathBF16<128>>(p, maps, di.sms, st) : launch_attn<MathBF16<64>>(p, maps, di.sms, st);
     } else {
 #define SPD_F32_CASE(DD, GG) if (D == DD && p.geff == GG) rc = launch_attn<MathF32<DD, GG>>(p, maps, di.sms, st);
@@ -532,6 +538,12 @@ spd_status spd_query_device_status(void *ws, void *cuda_stream, int32_t *first_b
 }
 
 int64_t spd_kernel_launch_count(void) { return g_launches.load(); }
+
+spd_status spd_set_bf16_math(int32_t path) {
+    if (path != 0 && path != 1) return SPD_ERR_INVALID_ARG;
+    g_bf16_math.store(path);
+    return SPD_OK;
+}
 
 spd_status spd_profile_begin(int32_t max_calls) {
     if (max_calls <= 0 || max_calls > (1 << 16)) return SPD_ERR_INVALID_ARG;

@@ -448,6 +448,144 @@ struct MathBF16 {
 };
 
 // ------------------------------------------------------------------------------------------------
+// bf16 tile math on the FMA pipes: the comparison arm for the tensor-core policy above (same tiles,
+// same TMA descriptors, same 128-byte-swizzled layout in shared memory; only the arithmetic differs).
+// K and V are widened to fp32 on the fly.  Costs grow with the group size, which is the point of the
+// comparison: at one query head per KV head the FMA pipes keep up with HBM, at eight they do not.
+template <int D_, int GE_>
+struct MathBF16Simt {
+    static constexpr int D = D_, GE = GE_;
+    static constexpr int kTileBytes = kPage * D * 2;
+    static constexpr int kBoxes = D / 64;
+    static constexpr int kBoxBytes = kPage * 128;
+    static constexpr int kBoxCols = 64;
+    static constexpr int kWarps = 7;       // one fewer than the tensor-core policy: q and P need 4.6 KB per warp
+    static constexpr int kStages = SPD_BF16_STAGES;
+    static constexpr int kExtraBytes = (kHeadsPerItem * D + kHeadsPerItem * kPage) * 4;  // q (fp32), P
+    static constexpr int V = D / 32;
+
+    struct State {
+        float o[GE][V];
+        float m[GE], l[GE], lw[GE];
+        int wlo, whi;
+    };
+
+    __device__ static __forceinline__ void begin(State &st, const Params &p, int u, int sq, int lane, uint8_t *extra) {
+        float *qs = reinterpret_cast<float *>(extra);
+        const int hbase = first_head(p, sq);
+        const __nv_bfloat16 *qg = reinterpret_cast<const __nv_bfloat16 *>(p.q) + (static_cast<int64_t>(u) * p.Hq + hbase) * D;
+        __syncwarp();
+        for (int i = lane; i < GE * D; i += 32) qs[i] = __bfloat162float(qg[i]);
+        __syncwarp();
+#pragma unroll
+        for (int hh = 0; hh < GE; ++hh) {
+#pragma unroll
+            for (int i = 0; i < V; ++i) st.o[hh][i] = 0.f;
+            st.m[hh] = -INFINITY;
+            st.l[hh] = 0.f;
+            st.lw[hh] = 0.f;
+        }
+        st.wlo = p.watch_out ? p.watch_lo[u] : 0;
+        st.whi = p.watch_out ? p.watch_hi[u] : 0;
+    }
+
+    __device__ static __forceinline__ void tile(State &st, const Params &p, uint8_t *Ks, uint8_t *Vs, int valid,
+                                                int lane, uint8_t *extra, int watch_base) {
+        const float *qs = reinterpret_cast<const float *>(extra);
+        float *Ps = reinterpret_cast<float *>(extra) + kHeadsPerItem * D;
+        // scores: lane = (token t, half of head_dim); a half is 64 columns = one swizzled box (D = 128)
+        // or half a box (D = 64); 16-byte chunk c of row t sits at chunk c ^ (t & 7) of its 128-byte line
+        const int t = lane & 15, hf = lane >> 4;
+        constexpr int NCH = D / 16;                       // chunks of 8 channels per half row
+        const int chunk0 = (D == 128) ? 0 : hf * NCH;     // first chunk of this half within its box
+        const uint8_t *kline = Ks + ((D == 128) ? hf * kBoxBytes : 0) + t * 128;
+        float s[GE];
+#pragma unroll
+        for (int hh = 0; hh < GE; ++hh) s[hh] = 0.f;
+#pragma unroll
+        for (int j = 0; j < NCH; ++j) {
+            const int c = chunk0 + j;
+            const uint4 raw = *reinterpret_cast<const uint4 *>(kline + ((c ^ (t & 7)) << 4));
+            const __nv_bfloat162 *k2 = reinterpret_cast<const __nv_bfloat162 *>(&raw);
+            float kf[8];
+#pragma unroll
+            for (int i = 0; i < 4; ++i) { const float2 f = __bfloat1622float2(k2[i]); kf[2 * i] = f.x; kf[2 * i + 1] = f.y; }
+#pragma unroll
+            for (int hh = 0; hh < GE; ++hh) {
+                const float4 qa = *reinterpret_cast<const float4 *>(qs + hh * D + hf * (D / 2) + 8 * j);
+                const float4 qb = *reinterpret_cast<const float4 *>(qs + hh * D + hf * (D / 2) + 8 * j + 4);
+                s[hh] = fmaf(kf[0], qa.x, s[hh]); s[hh] = fmaf(kf[1], qa.y, s[hh]);
+                s[hh] = fmaf(kf[2], qa.z, s[hh]); s[hh] = fmaf(kf[3], qa.w, s[hh]);
+                s[hh] = fmaf(kf[4], qb.x, s[hh]); s[hh] = fmaf(kf[5], qb.y, s[hh]);
+                s[hh] = fmaf(kf[6], qb.z, s[hh]); s[hh] = fmaf(kf[7], qb.w, s[hh]);
+            }
+        }
+        __syncwarp();   // the previous tile's readers of Ps are done
+#pragma unroll
+        for (int hh = 0; hh < GE; ++hh) {
+            float v = s[hh] + __shfl_xor_sync(0xffffffffu, s[hh], 16);
+            v = (t < valid) ? v * p.sm_scale : -INFINITY;
+            float tmax = v;
+#pragma unroll
+            for (int d = 8; d >= 1; d >>= 1) tmax = fmaxf(tmax, __shfl_xor_sync(0xffffffffu, tmax, d));
+            const float m_new = fmaxf(st.m[hh], tmax);
+            const float alpha = ex2_approx((st.m[hh] - m_new) * kLog2e);
+            const float pr = ex2_approx((v - m_new) * kLog2e);
+            st.l[hh] = st.l[hh] * alpha + (hf == 0 ? pr : 0.f);
+            st.lw[hh] = st.lw[hh] * alpha + ((hf == 0 && watch_base + t >= st.wlo && watch_base + t < st.whi) ? pr : 0.f);
+            st.m[hh] = m_new;
+#pragma unroll
+            for (int i = 0; i < V; ++i) st.o[hh][i] *= alpha;
+            if (hf == 0) Ps[hh * kPage + t] = pr;
+        }
+        __syncwarp();
+        // P V: lane owns channels [lane * V, lane * V + V): V bf16 inside one 16-byte chunk
+        const int col = lane * V;                                   // channel
+        const int box = col / 64, cc = (col % 64) / 8, within = (col % 8) * 2;   // box, chunk, byte in chunk
+        for (int tt = 0; tt < valid; ++tt) {   // rows past `valid` are never touched
+            const uint8_t *src = Vs + box * kBoxBytes + tt * 128 + ((cc ^ (tt & 7)) << 4) + within;
+            float vv[V];
+            if constexpr (V == 4) {
+                const uint2 raw = *reinterpret_cast<const uint2 *>(src);
+                const __nv_bfloat162 *v2 = reinterpret_cast<const __nv_bfloat162 *>(&raw);
+                const float2 a = __bfloat1622float2(v2[0]), b = __bfloat1622float2(v2[1]);
+                vv[0] = a.x; vv[1] = a.y; vv[2] = b.x; vv[3] = b.y;
+            } else {
+                const float2 a = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162 *>(src));
+                vv[0] = a.x; vv[1] = a.y;
+            }
+#pragma unroll
+            for (int hh = 0; hh < GE; ++hh) {
+                const float pr = Ps[hh * kPage + tt];
+#pragma unroll
+                for (int i = 0; i < V; ++i) st.o[hh][i] = fmaf(pr, vv[i], st.o[hh][i]);
+            }
+        }
+    }
+
+    __device__ static __forceinline__ void finish(State &st, float *So, float *Sm, float *Sl, int lane) {
+        constexpr int PITCH = D + 4;
+#pragma unroll
+        for (int hh = 0; hh < GE; ++hh) {
+#pragma unroll
+            for (int i = 0; i < V; ++i) So[hh * PITCH + lane * V + i] = st.o[hh][i];
+            float l = st.l[hh], lw = st.lw[hh];
+#pragma unroll
+            for (int d = 8; d >= 1; d >>= 1) {
+                l += __shfl_xor_sync(0xffffffffu, l, d);
+                lw += __shfl_xor_sync(0xffffffffu, lw, d);
+            }
+            if (lane == 0) { Sm[hh] = st.m[hh]; Sl[hh] = l; Sl[kHeadsPerItem + hh] = lw; }
+        }
+        for (int hh = GE; hh < kHeadsPerItem; ++hh) {
+#pragma unroll
+            for (int i = 0; i < V; ++i) So[hh * PITCH + lane * V + i] = 0.f;
+            if (lane == 0) { Sm[hh] = -INFINITY; Sl[hh] = 0.f; Sl[kHeadsPerItem + hh] = 0.f; }
+        }
+    }
+};
+
+// ------------------------------------------------------------------------------------------------
 // fp32 tile math on the FMA pipes (no reduced precision anywhere).
 //   scores : lane = (token t = lane & 15, half of head_dim = lane >> 4); each lane walks its half
 //            row of K in float4 steps, starting at a chunk rotated by t so that the 8 lanes of a

@@ -129,3 +129,17 @@ def test_bf16_output_dtype():
     got = run_decode(w.to("cuda"), True, out_dtype=torch.bfloat16)
     # output rounded to bf16: half an ulp of values up to ~4 on top of the compute error
     assert np.max(np.abs(got - ref)) <= 2e-3 + 2.0 ** -8 * np.max(np.abs(ref))
+
+
+@pytest.mark.parametrize("name", ["bf16_mha_d128", "bf16_gqa4_d128", "bf16_gqa8_d128", "bf16_gqa16_d128", "bf16_gqa2_d64", "bf16_long_split"])
+def test_bf16_fma_pipe_arm_matches_oracle(name):
+    """The comparison arm (bf16 tiles on the FMA pipes instead of the tensor cores) computes the same thing."""
+    w = wl.make_workload(dict(SMALL[name], name=name), slack=True)
+    q, kin, kout = oracle_inputs(w)
+    ref = orc.full(q, kin, kout, w.sm_scale)
+    spd.spd_set_bf16_math(1)
+    try:
+        for fused in (True, False):
+            assert_close(run_decode(w.to("cuda"), fused), ref, w.dtype, f"{name} FMA arm fused={fused}")
+    finally:
+        spd.spd_set_bf16_math(0)
