@@ -859,12 +859,16 @@ attn_kernel(const __grid_constant__ Params p, const __grid_constant__ CUtensorMa
         }
         ok = __all_sync(0xffffffffu, ok);
         const float nw = ok ? G / sw : 0.f, nr = ok ? G / sr : 0.f;
-        // weight of CTA i: 1/4 of the weight it had last time + 3/4 of the rate it achieved, both
-        // relative to the mean; lane l looks after CTAs [l*cpl, (l+1)*cpl)
+        // lane l looks after CTAs [l*cpl, (l+1)*cpl)
         const int cpl = (G + 31) / 32;
         int mysum = 0;
         for (int i = lane * cpl; i < min(G, (lane + 1) * cpl); ++i) {
-            const float m = ok ? 0.25f * sh_w[i] * nw + 0.75f * sh_r[i] * nr : 1.f;
+            // new weight = old weight moved towards the measured rate (both relative to the mean): most of
+            // the way when they disagree by more than 4 % (a real difference between SMs), a quarter of
+            // the way otherwise (so that run-to-run noise is averaged out instead of chased)
+            const float wn = sh_w[i] * nw, rn = sh_r[i] * nr;
+            const float gain = fabsf(rn - wn) > 0.04f * wn ? 0.75f : 0.25f;
+            const float m = ok ? wn + gain * (rn - wn) : 1.f;
             int q = static_cast<int>(m * 1024.f + 0.5f);
             q = q < 512 ? 512 : (q > 2048 ? 2048 : q);
             sh_wq[i] = q;
