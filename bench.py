@@ -255,6 +255,56 @@ def time_e2e(spd, w, shape, ws, steps, warmup):
     return e0.elapsed_time(e1) / steps, lay.in_bytes, d2h, outh
 
 
+def time_schedules(spd, w, shape, steps=200):
+    """The same step scheduled four ways, microseconds per step by CUDA events: the two halves chained on one
+    stream, the halves on two streams followed by the stand-alone merge, the fused step, and the fused
+    step replayed from a CUDA graph (20 steps per graph)."""
+    dev = w.q.device
+    out = torch.empty((w.batch, w.num_q_heads, w.head_dim), dtype=torch.float32, device=dev)
+    ws_a, ws_b = spd.alloc_workspace(shape), spd.alloc_workspace(shape)
+    pa, pb = spd.alloc_partial(shape), spd.alloc_partial(shape)
+    sa, sb = torch.cuda.Stream(), torch.cuda.Stream()
+
+    def chained():
+        spd.spd_decode_step(shape, w.q, w.priv, w.pub, out, ws_a, fused=False, stream=sa)
+
+    def fused():
+        spd.spd_decode_step(shape, w.q, w.priv, w.pub, out, ws_a, fused=True, stream=sa)
+
+    def two_streams():
+        sb.wait_stream(sa)                                   # the previous merge has read pb
+        spd.spd_partial_attn(shape, w.q, w.priv, pa, ws_a, stream=sa)
+        spd.spd_partial_attn(shape, w.q, w.pub, pb, ws_b, stream=sb)
+        sa.wait_stream(sb)
+        spd.spd_merge_partials(shape, [pa, pb], out, stream=sa)
+
+    def timed(fn, n):
+        for _ in range(10):
+            fn()
+        torch.cuda.synchronize()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record(sa)
+        for _ in range(n):
+            fn()
+        e1.record(sa)
+        torch.cuda.synchronize()
+        return e0.elapsed_time(e1) / n * 1e3
+
+    res = {"chained_us": timed(chained, steps), "two_streams_us": timed(two_streams, steps), "fused_us": timed(fused, steps)}
+    per_graph = 20
+    graph = torch.cuda.CUDAGraph()
+    with torch.cuda.stream(sa):
+        with torch.cuda.graph(graph, stream=sa):
+            for _ in range(per_graph):
+                spd.spd_decode_step(shape, w.q, w.priv, w.pub, out, ws_a, fused=True, stream=sa)
+        res["fused_graph_us"] = timed(graph.replay, max(1, steps // per_graph)) / per_graph
+    for ws in (ws_a, ws_b):
+        code, bad = spd.spd_query_device_status(ws, stream=sa)
+        if code != spd.SPD_OK:
+            raise RuntimeError(f"schedule study failed: status {code}, user {bad}")
+    return res
+
+
 def time_append(spd, w, shape, ws, calls=8):
     """spd_append_kv on the public cache: `calls` tokens per user appended back to back (the lengths are
     first moved back by `calls`, and restored afterwards, so that every row fits the pages already listed)."""
@@ -369,6 +419,7 @@ def run_cuda(args):
         del w
         torch.cuda.empty_cache()
         w = wl.make_workload(cfg, device=dev)
+        line["schedules"] = time_schedules(spd, w, spd.make_shape(w.batch, w.num_q_heads, w.num_kv_heads, w.head_dim, w.dtype, w.sm_scale))
         line["append_kv"] = time_append(spd, w, spd.make_shape(w.batch, w.num_q_heads, w.num_kv_heads, w.head_dim, w.dtype, w.sm_scale), ws)
         w = wl.make_workload(cfg, device="cpu")
         line["cpu_baseline"] = cpu_baseline(w)

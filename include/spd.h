@@ -105,6 +105,17 @@ spd_status spd_service_attn_merge(const spd_shape *shape, const void *q, const s
                                   void *ws, size_t ws_bytes, void *cuda_stream);
 
 /*
+ * The merge on its own (Theorem 1, Eq. 1; maxima as in Sec. 4.2; Fig. 3 step 5), n-way: combines `n`
+ * partials (1 <= n <= 8; `parts` is a HOST array of n structs holding device pointers) into the
+ * normalised attention output.  For a caller that obtains the partials separately -- from other
+ * processes, or from private and public halves run on different streams -- instead of letting
+ * spd_service_attn_merge fuse the merge into the public half.  Rows whose partials are all empty give 0.
+ * One small kernel on `cuda_stream`; no workspace.
+ */
+spd_status spd_merge_partials(const spd_shape *shape, int32_t n, const spd_partial *parts, void *out,
+                              spd_dtype out_dtype, void *cuda_stream);
+
+/*
  * One whole decode step of attention for one layer (protocol step 3, b and c): the private
  * partial, the public partial and their merge.  `fused` = 0 chains spd_partial_attn and
  * spd_service_attn_merge through a partial held in the workspace; `fused` != 0 streams both

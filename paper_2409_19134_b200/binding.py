@@ -22,7 +22,7 @@ EXPORTS = ["spd_workspace_size", "spd_partial_attn", "spd_service_attn_merge", "
            "spd_step_blob_layout", "spd_decode_step_host", "spd_query_device_status",
            "spd_kernel_launch_count", "spd_status_string", "spd_profile_begin", "spd_profile_end",
            "spd_decode_step_static", "spd_append_kv",
-           "spd_partial_attn_watch", "spd_decode_step_watch", "spd_set_bf16_math"]
+           "spd_partial_attn_watch", "spd_decode_step_watch", "spd_set_bf16_math", "spd_merge_partials"]
 
 
 class SpdError(RuntimeError):
@@ -87,6 +87,7 @@ def lib() -> C.CDLL:
         L.spd_decode_step_watch.argtypes = [C.POINTER(Shape), vp, C.POINTER(PagedKV), C.POINTER(PagedKV), vp, C.c_int,
                                             C.POINTER(Watch), vp, sz, vp]
         L.spd_set_bf16_math.argtypes = [C.c_int32]
+        L.spd_merge_partials.argtypes = [C.POINTER(Shape), C.c_int32, C.POINTER(Partial), vp, C.c_int, vp]
         L.spd_append_kv.argtypes = [C.POINTER(Shape), vp, vp, vp, vp, C.c_int32, vp, vp, vp, vp, sz, vp]
         for name in EXPORTS[:7] + EXPORTS[9:]:
             getattr(L, name).restype = C.c_int
@@ -304,3 +305,10 @@ def spd_decode_step_watch(shape, q, priv, pub, out, tok_lo, tok_hi, watch_out, w
 def spd_set_bf16_math(path: int) -> None:
     """0 = tensor cores (default), 1 = FMA pipes (comparison arm); process-wide."""
     _check(lib().spd_set_bf16_math(int(path)), "spd_set_bf16_math")
+
+
+def spd_merge_partials(shape, parts, out, stream=None) -> None:
+    """parts: a sequence of (o, m, l) tensor triples; writes the merged, normalised output."""
+    arr = (Partial * len(parts))(*[Partial(o.data_ptr(), m.data_ptr(), l.data_ptr()) for o, m, l in parts])
+    _check(lib().spd_merge_partials(C.byref(shape), len(parts), arr, out.data_ptr(), _dtype_code(out.dtype),
+                                    _stream_ptr(stream)), "spd_merge_partials")

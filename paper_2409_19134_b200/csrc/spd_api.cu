@@ -413,6 +413,31 @@ spd_status spd_decode_step_watch(const spd_shape *shape, const void *q, const sp
     return run_job(job, ws, ws_bytes, cuda_stream);
 }
 
+spd_status spd_merge_partials(const spd_shape *shape, int32_t n, const spd_partial *parts, void *out,
+                               spd_dtype out_dtype, void *cuda_stream) {
+    spd_status rc = check_shape(shape);
+    if (rc != SPD_OK) return rc;
+    if (n < 1 || n > kMaxMergeParts) return SPD_ERR_UNSUPPORTED;
+    if (!parts || !out || misaligned(out, 16)) return SPD_ERR_INVALID_ARG;
+    if (out_dtype != SPD_F32 && out_dtype != SPD_BF16) return SPD_ERR_UNSUPPORTED;
+    MergeParams mp;
+    memset(&mp, 0, sizeof mp);
+    mp.rows = shape->batch * shape->num_q_heads;
+    mp.n = n;
+    mp.out_bf16 = out_dtype == SPD_BF16;
+    mp.out = out;
+    for (int c = 0; c < n; ++c) {
+        if (!parts[c].o || !parts[c].m || !parts[c].l || misaligned(parts[c].o, 16)) return SPD_ERR_INVALID_ARG;
+        mp.o[c] = parts[c].o; mp.m[c] = parts[c].m; mp.l[c] = parts[c].l;
+    }
+    cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+    const int blocks = (mp.rows + 3) / 4;
+    if (shape->head_dim == 128) merge_partials_kernel<128><<<blocks, 128, 0, st>>>(mp);
+    else merge_partials_kernel<64><<<blocks, 128, 0, st>>>(mp);
+    ++g_launches;
+    return cudaGetLastError() == cudaSuccess ? SPD_OK : SPD_ERR_CUDA;
+}
+
 spd_status spd_append_kv(const spd_shape *shape, const void *k_new, const void *v_new, void *k_pool, void *v_pool,
                          int32_t num_pages, const int32_t *page_indptr, const int32_t *page_indices,
                          int32_t *seq_lens, void *ws, size_t ws_bytes, void *cuda_stream) {

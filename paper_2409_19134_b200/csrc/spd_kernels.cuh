@@ -1142,4 +1142,47 @@ __global__ void __launch_bounds__(128) append_kernel(AppendParams p) {
     if (threadIdx.x == 0) p.lens[u] += 1;
 }
 
+// ------------------------------------------------------------------------------------------------
+// Merge of up to kMaxMergeParts partials into the normalised attention output (Theorem 1 / Eq. 1 with
+// the maxima of Sec. 4.2, n-way): one warp per (user, query head), lane = D/32 channels.
+constexpr int kMaxMergeParts = 8;
+struct MergeParams {
+    int32_t rows, n, out_bf16;     // rows = batch * num_q_heads
+    const float *o[kMaxMergeParts], *m[kMaxMergeParts], *l[kMaxMergeParts];
+    void *out;
+};
+
+template <int D>
+__global__ void __launch_bounds__(128) merge_partials_kernel(MergeParams p) {
+    constexpr int V = D / 32;
+    const int lane = threadIdx.x & 31;
+    const int64_t row = static_cast<int64_t>(blockIdx.x) * 4 + (threadIdx.x >> 5);
+    if (row >= p.rows) return;
+    float M = -INFINITY;
+    for (int c = 0; c < p.n; ++c) M = fmaxf(M, p.m[c][row]);
+    float L = 0.f, o[V];
+#pragma unroll
+    for (int i = 0; i < V; ++i) o[i] = 0.f;
+    for (int c = 0; c < p.n; ++c) {
+        const float mc = p.m[c][row];
+        const float w = (mc == -INFINITY) ? 0.f : expf(mc - M);
+        L = fmaf(w, p.l[c][row], L);
+        const float *src = p.o[c] + row * D + lane * V;
+#pragma unroll
+        for (int i = 0; i < V; ++i) o[i] = fmaf(w, src[i], o[i]);
+    }
+    const float inv = L > 0.f ? 1.f / L : 0.f;
+#pragma unroll
+    for (int i = 0; i < V; ++i) o[i] = inv == 0.f ? 0.f : o[i] * inv;
+    if (p.out_bf16) {
+        __nv_bfloat16 *dst = reinterpret_cast<__nv_bfloat16 *>(p.out) + row * D + lane * V;
+#pragma unroll
+        for (int i = 0; i < V; i += 2) *reinterpret_cast<__nv_bfloat162 *>(dst + i) = __floats2bfloat162_rn(o[i], o[i + 1]);
+    } else {
+        float *dst = reinterpret_cast<float *>(p.out) + row * D + lane * V;
+#pragma unroll
+        for (int i = 0; i < V; ++i) dst[i] = o[i];
+    }
+}
+
 }  // namespace spd
