@@ -214,3 +214,43 @@ void spd_oracle_merge_alpha(int64_t rows, int D, const double *o_in, const doubl
             y[r * D + d] = c_in * (o_in[r * D + d] / l_in[r]) + c_out * (o_out[r * D + d] / l_out[r]);
     }
 }
+
+/*
+ * Prefill: causal self-attention over each user's prompt (protocol step 2; Fig. 3 step 0; the causal
+ * property of Sec. 2.1: token i attends to tokens 0..i of its own prompt).  q: [T][Hq][D], k, v:
+ * [T][Hkv][D], dense, users laid end to end; tok_indptr[B+1] are token offsets.  Computes the rows
+ * listed in `rows` (global token indices, n_rows of them): y[r][h][:] for r-th listed row.
+ */
+void spd_oracle_prefill(const oracle_shape *s, const void *q, const void *k, const void *v,
+                        const int32_t *tok_indptr, const int64_t *rows, int64_t n_rows, double *y)
+{
+    int Hq = s->num_q_heads, Hkv = s->num_kv_heads, D = s->head_dim;
+    int g = Hq / Hkv;
+#pragma omp parallel for collapse(2) schedule(dynamic, 1)
+    for (int64_t r = 0; r < n_rows; ++r) {
+        for (int h = 0; h < Hq; ++h) {
+            int64_t i = rows[r];
+            int u = 0;
+            while (u + 1 < s->batch && tok_indptr[u + 1] <= i) ++u;
+            int64_t first = tok_indptr[u], n = i - first + 1;       /* keys first..i */
+            int kvh = h / g;
+            double *yo = y + (r * Hq + h) * D;
+            for (int d = 0; d < D; ++d) yo[d] = 0.0;
+            double *sc = (double *)malloc(sizeof(double) * (size_t)n);
+            double mx = -INFINITY;
+            for (int64_t j = 0; j < n; ++j) {
+                double acc = 0.0;
+                for (int d = 0; d < D; ++d)
+                    acc += widen(q, (i * Hq + h) * D + d, s->dtype) * widen(k, ((first + j) * Hkv + kvh) * D + d, s->dtype);
+                sc[j] = s->sm_scale * acc;
+                if (sc[j] > mx) mx = sc[j];
+            }
+            double den = 0.0;
+            for (int64_t j = 0; j < n; ++j) { sc[j] = exp(sc[j] - mx); den += sc[j]; }
+            for (int64_t j = 0; j < n; ++j)
+                for (int d = 0; d < D; ++d)
+                    yo[d] += sc[j] / den * widen(v, ((first + j) * Hkv + kvh) * D + d, s->dtype);
+            free(sc);
+        }
+    }
+}

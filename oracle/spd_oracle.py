@@ -269,3 +269,38 @@ def watched_mass(q: np.ndarray, priv: KV, pub: Optional[KV], sm_scale: float, to
             full[u, h] = mass_w / (mass_in + mass_out)
             own[u, h] = mass_w / mass_in
     return full, own
+
+
+def prefill(q: np.ndarray, k: np.ndarray, v: np.ndarray, tok_indptr, sm_scale: float, rows=None) -> np.ndarray:
+    """Causal self-attention over each user's prompt (protocol step 2).
+
+    q [T, Hq, D], k, v [T, Hkv, D] (float32 or uint16 bf16 bits), users laid end to end with token offsets
+    tok_indptr [B+1].  Returns y [len(rows), Hq, D] float64 for the listed global token indices
+    (all tokens when rows is None)."""
+    lib = _load()
+    q, k, v = (np.ascontiguousarray(a) for a in (q, k, v))
+    T, Hq, D = q.shape
+    Hkv = k.shape[1]
+    ip = np.ascontiguousarray(tok_indptr, dtype=np.int32)
+    rows = np.arange(T, dtype=np.int64) if rows is None else np.ascontiguousarray(rows, dtype=np.int64)
+    dt = F32 if q.dtype == np.float32 else BF16
+    sh = _Shape(len(ip) - 1, Hq, Hkv, D, 16, dt, float(sm_scale))
+    y = np.zeros((len(rows), Hq, D), dtype=np.float64)
+    lib.spd_oracle_prefill(C.byref(sh), C.c_void_p(q.ctypes.data), C.c_void_p(k.ctypes.data), C.c_void_p(v.ctypes.data),
+                           C.c_void_p(ip.ctypes.data), C.c_void_p(rows.ctypes.data), C.c_int64(len(rows)),
+                           C.c_void_p(y.ctypes.data))
+    return y
+
+
+def write_prompt_kv(kv: KV, k: np.ndarray, v: np.ndarray, tok_indptr) -> None:
+    """Store every prompt token's K and V row in the paged cache, in place, and set seq_lens (what prefill
+    leaves behind for decode).  Token t of user u goes to page page_indices[page_indptr[u] + t // P], slot
+    t % P.  Pure indexing."""
+    P = kv.k_pool.shape[2]
+    for u in range(len(tok_indptr) - 1):
+        a, b = int(tok_indptr[u]), int(tok_indptr[u + 1])
+        for t in range(b - a):
+            page = int(kv.page_indices[int(kv.page_indptr[u]) + t // P])
+            kv.k_pool[page, :, t % P, :] = k[a + t]
+            kv.v_pool[page, :, t % P, :] = v[a + t]
+        kv.seq_lens[u] = b - a

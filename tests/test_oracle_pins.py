@@ -399,3 +399,39 @@ def test_watched_mass_is_the_sum_of_softmax_probabilities():
     # uniform scores: the share is the fraction of tokens watched
     fu, ou = orc.watched_mass(np.zeros_like(q), kin, kout, 0.6, np.array([2, 2, 2]), np.array([12, 5, 10]))
     assert np.allclose(fu[:, 0], [10 / 49, 3 / 7, 8 / 19], atol=1e-12) and np.allclose(ou[:, 0], [10 / 40, 3 / 7, 8 / 16], atol=1e-12)
+
+
+# ---------------------------------------------------------------- prefill: causal attention over the prompt
+def test_prefill_is_causal_softmax_and_hands_over_to_decode():
+    rng = np.random.default_rng(41)
+    Hq, Hkv, D = 4, 2, 8
+    lens = [37, 1, 20]
+    ip = np.concatenate([[0], np.cumsum(lens)])
+    T = int(ip[-1])
+    q = rng.standard_normal((T, Hq, D)).astype(np.float32)
+    k = rng.standard_normal((T, Hkv, D)).astype(np.float32)
+    v = rng.standard_normal((T, Hkv, D)).astype(np.float32)
+    y = orc.prefill(q, k, v, ip, 0.45)
+    # textbook: per user, lower-triangular mask, softmax, times V (dense NumPy, float64)
+    for u, L in enumerate(lens):
+        a = int(ip[u])
+        for h in range(Hq):
+            S = 0.45 * q[a:a + L, h].astype(np.float64) @ k[a:a + L, h // 2].astype(np.float64).T
+            S = np.where(np.tril(np.ones((L, L), bool)), S, -np.inf)
+            Pm = np.exp(S - S.max(1, keepdims=True))
+            Pm /= Pm.sum(1, keepdims=True)
+            assert np.max(np.abs(y[a:a + L, h] - Pm @ v[a:a + L, h // 2].astype(np.float64))) < 1e-12
+        assert np.array_equal(y[a, 0], v[a, 0].astype(np.float64))          # the first token sees only itself
+    # the listed-rows form agrees with the full form
+    rows = np.array([0, 5, 36, 37, 38, 57])
+    assert np.array_equal(orc.prefill(q, k, v, ip, 0.45, rows), y[rows])
+    # hand-over: store the prompt's K/V in a paged cache; a decode query equal to the last prompt token's q
+    # must reproduce that token's prefill output (it attends to the same keys)
+    ks = [np.zeros((Hkv, L, D), np.float32) for L in lens]
+    kv = dense_to_paged(ks, ks, rng=rng)
+    kv.seq_lens[:] = 0
+    orc.write_prompt_kv(kv, k, v, ip)
+    assert kv.seq_lens.tolist() == lens
+    last = ip[1:] - 1
+    yd = orc.full(q[last], kv, None, 0.45)
+    assert np.max(np.abs(yd - y[last])) < 1e-12
