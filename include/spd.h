@@ -152,6 +152,26 @@ spd_status spd_decode_step_watch(const spd_shape *shape, const void *q, const sp
                                  const spd_watch *watch, void *ws, size_t ws_bytes, void *cuda_stream);
 
 /*
+ * Prefill (protocol step 2; Fig. 3 step 0): causal self-attention over every user's prompt, and the
+ * hand-over of the prompt's K and V rows to the private paged cache that the decode calls read.
+ *   q [total_tokens][num_q_heads][head_dim], k, v [total_tokens][num_kv_heads][head_dim]: the prompts of
+ *   all users laid end to end; tok_indptr [batch+1] (device) gives each user's first token.
+ *   out [total_tokens][num_q_heads][head_dim] in out_dtype: token i of a prompt attends to tokens 0..i of
+ *   the same prompt (softmax of sm_scale * q.k, as in the decode calls).
+ *   k_pool / v_pool / page tables: the private partition; token t of user u is stored in page
+ *   page_indices[page_indptr[u] + t / page_size], slot t % page_size, and seq_lens[u] is set to the
+ *   prompt's length.  A user whose listed pages cannot hold its prompt, or whose offsets are inconsistent,
+ *   is skipped and raises SPD_ERR_BAD_PAGE in the status words at the start of `ws`.
+ * Supported: BF16, head_dim 128.  Two kernels on `cuda_stream`: the copy into the cache and the attention
+ * (tcgen05 tensor-core MMAs with accumulators in tensor memory).
+ */
+spd_status spd_prefill_attn(const spd_shape *shape, int64_t total_tokens, const void *q, const void *k,
+                            const void *v, const int32_t *tok_indptr, void *k_pool, void *v_pool,
+                            int32_t num_pages, const int32_t *page_indptr, const int32_t *page_indices,
+                            int32_t *seq_lens, void *out, spd_dtype out_dtype, void *ws, size_t ws_bytes,
+                            void *cuda_stream);
+
+/*
  * Append of the new token's K and V rows to a paged cache -- what the service does to its public
  * cache right before attention (protocol step 3a; Fig. 3 step 2), so that the new token attends to
  * itself through the public partition.  k_new, v_new: [batch][num_kv_heads][head_dim] in the shape's

@@ -22,7 +22,7 @@ EXPORTS = ["spd_workspace_size", "spd_partial_attn", "spd_service_attn_merge", "
            "spd_step_blob_layout", "spd_decode_step_host", "spd_query_device_status",
            "spd_kernel_launch_count", "spd_status_string", "spd_profile_begin", "spd_profile_end",
            "spd_decode_step_static", "spd_append_kv",
-           "spd_partial_attn_watch", "spd_decode_step_watch", "spd_set_bf16_math", "spd_merge_partials"]
+           "spd_partial_attn_watch", "spd_decode_step_watch", "spd_set_bf16_math", "spd_merge_partials", "spd_prefill_attn"]
 
 
 class SpdError(RuntimeError):
@@ -88,6 +88,8 @@ def lib() -> C.CDLL:
                                             C.POINTER(Watch), vp, sz, vp]
         L.spd_set_bf16_math.argtypes = [C.c_int32]
         L.spd_merge_partials.argtypes = [C.POINTER(Shape), C.c_int32, C.POINTER(Partial), vp, C.c_int, vp]
+        L.spd_prefill_attn.argtypes = [C.POINTER(Shape), C.c_int64, vp, vp, vp, vp, vp, vp, C.c_int32, vp, vp, vp, vp,
+                                       C.c_int, vp, sz, vp]
         L.spd_append_kv.argtypes = [C.POINTER(Shape), vp, vp, vp, vp, C.c_int32, vp, vp, vp, vp, sz, vp]
         for name in EXPORTS[:7] + EXPORTS[9:]:
             getattr(L, name).restype = C.c_int
@@ -312,3 +314,16 @@ def spd_merge_partials(shape, parts, out, stream=None) -> None:
     arr = (Partial * len(parts))(*[Partial(o.data_ptr(), m.data_ptr(), l.data_ptr()) for o, m, l in parts])
     _check(lib().spd_merge_partials(C.byref(shape), len(parts), arr, out.data_ptr(), _dtype_code(out.dtype),
                                     _stream_ptr(stream)), "spd_merge_partials")
+
+
+def spd_prefill_attn(shape, q, k, v, tok_indptr, part, out, ws, stream=None) -> None:
+    """Causal attention over the prompts (q [T,Hq,D], k, v [T,Hkv,D], tok_indptr int32 [B+1]) into `out`
+    [T,Hq,D]; the prompts' K/V rows go into the partition `part` (pools and seq_lens updated in place)."""
+    for t in (q, k, v, out):
+        assert t.is_contiguous()
+    assert tok_indptr.dtype == torch.int32
+    _check(lib().spd_prefill_attn(C.byref(shape), int(q.shape[0]), _ptr(q), _ptr(k), _ptr(v), tok_indptr.data_ptr(),
+                                  part.k_pool.data_ptr(), part.v_pool.data_ptr(), int(part.k_pool.shape[0]),
+                                  part.page_indptr.data_ptr(), _ptr(part.page_indices), part.seq_lens.data_ptr(),
+                                  _ptr(out), _dtype_code(out.dtype), ws.data_ptr(), ws.numel(), _stream_ptr(stream)),
+           "spd_prefill_attn")

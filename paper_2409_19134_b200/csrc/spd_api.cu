@@ -10,6 +10,7 @@
 #include <vector>
 
 #include "spd_kernels.cuh"
+#include "spd_prefill.cuh"
 
 namespace {
 
@@ -411,6 +412,74 @@ spd_status spd_decode_step_watch(const spd_shape *shape, const void *q, const sp
     job.epoch = next_epoch();
     job.watch = watch;
     return run_job(job, ws, ws_bytes, cuda_stream);
+}
+
+// [T][H][128] bf16 as a 3-D tensor map; one box = 128 tokens x 64 channels of one head, 128-byte swizzle.
+static spd_status make_prompt_map(CUtensorMap *map, const void *ptr, int64_t T, int heads) {
+    EncodeTiledFn fn = encode_fn();
+    if (!fn) return SPD_ERR_CUDA;
+    cuuint64_t dims[3] = {128, static_cast<cuuint64_t>(heads), static_cast<cuuint64_t>(T)};
+    cuuint64_t strides[2] = {128 * 2, static_cast<cuuint64_t>(heads) * 128 * 2};
+    cuuint32_t box[3] = {64, 1, static_cast<cuuint32_t>(kPfBlock)};
+    cuuint32_t estr[3] = {1, 1, 1};
+    CUresult r = fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void *>(ptr), dims, strides, box, estr,
+                    CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                    CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    return r == CUDA_SUCCESS ? SPD_OK : SPD_ERR_CUDA;
+}
+
+spd_status spd_prefill_attn(const spd_shape *shape, int64_t total_tokens, const void *q, const void *k, const void *v,
+                            const int32_t *tok_indptr, void *k_pool, void *v_pool, int32_t num_pages,
+                            const int32_t *page_indptr, const int32_t *page_indices, int32_t *seq_lens, void *out,
+                            spd_dtype out_dtype, void *ws, size_t ws_bytes, void *cuda_stream) {
+    spd_status rc = check_shape(shape);
+    if (rc != SPD_OK) return rc;
+    if (shape->dtype != SPD_BF16 || shape->head_dim != 128) return SPD_ERR_UNSUPPORTED;
+    if (out_dtype != SPD_F32 && out_dtype != SPD_BF16) return SPD_ERR_UNSUPPORTED;
+    if (total_tokens < 0 || total_tokens >= (1ll << 31) - kPfBlock) return SPD_ERR_INVALID_ARG;
+    if (!tok_indptr || !page_indptr || !seq_lens || !ws || misaligned(ws, 256)) return SPD_ERR_INVALID_ARG;
+    if (ws_bytes < HDR_WORDS * 4) return SPD_ERR_WORKSPACE;
+    if (total_tokens > 0 && (!q || !k || !v || !out || !k_pool || !v_pool || num_pages <= 0)) return SPD_ERR_INVALID_ARG;
+    if (misaligned(q, 16) || misaligned(k, 16) || misaligned(v, 16) || misaligned(out, 16) || misaligned(k_pool, 128) ||
+        misaligned(v_pool, 128))
+        return SPD_ERR_INVALID_ARG;
+    DeviceInfo di;
+    if ((rc = device_info(&di)) != SPD_OK) return rc;
+    cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+    const int64_t T = total_tokens;
+
+    PromptKvParams kp;
+    kp.B = shape->batch; kp.Hkv = shape->num_kv_heads; kp.row_bytes = 128 * 2; kp.T = T;
+    kp.k = static_cast<const uint8_t *>(k); kp.v = static_cast<const uint8_t *>(v); kp.tok_indptr = tok_indptr;
+    kp.k_pool = static_cast<uint8_t *>(k_pool); kp.v_pool = static_cast<uint8_t *>(v_pool); kp.num_pages = num_pages;
+    kp.page_indptr = page_indptr; kp.page_indices = page_indices; kp.lens = seq_lens; kp.hdr = static_cast<int32_t *>(ws);
+    prompt_kv_kernel<<<static_cast<unsigned>(T + 1), 128, 0, st>>>(kp);
+    ++g_launches;
+    if (cudaGetLastError() != cudaSuccess) return SPD_ERR_CUDA;
+    if (T == 0) return SPD_OK;
+
+    CUtensorMap mq, mk, mv;
+    if ((rc = make_prompt_map(&mq, q, T, shape->num_q_heads)) != SPD_OK) return rc;
+    if ((rc = make_prompt_map(&mk, k, T, shape->num_kv_heads)) != SPD_OK) return rc;
+    if ((rc = make_prompt_map(&mv, v, T, shape->num_kv_heads)) != SPD_OK) return rc;
+    PrefillParams pp;
+    pp.B = shape->batch; pp.Hq = shape->num_q_heads; pp.Hkv = shape->num_kv_heads; pp.T = T;
+    pp.sm_scale = shape->sm_scale; pp.tok_indptr = tok_indptr; pp.out = out; pp.out_bf16 = out_dtype == SPD_BF16;
+    pp.hdr = static_cast<int32_t *>(ws);
+    static std::once_flag once[64];
+    int dev = 0;
+    cudaGetDevice(&dev);
+    cudaError_t attr_err = cudaSuccess;
+    std::call_once(once[dev & 63], [&] {
+        attr_err = cudaFuncSetAttribute(prefill_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                        static_cast<int>(prefill_smem_bytes()));
+    });
+    if (attr_err != cudaSuccess) return SPD_ERR_CUDA;
+    const int64_t max_blocks = (T + kPfBlock - 1) / kPfBlock + shape->batch;   // >= sum over users of ceil(len / 128)
+    dim3 grid(static_cast<unsigned>(max_blocks), static_cast<unsigned>(shape->num_q_heads));
+    prefill_kernel<<<grid, 128, prefill_smem_bytes(), st>>>(pp, mq, mk, mv);
+    ++g_launches;
+    return cudaGetLastError() == cudaSuccess ? SPD_OK : SPD_ERR_CUDA;
 }
 
 spd_status spd_merge_partials(const spd_shape *shape, int32_t n, const spd_partial *parts, void *out,

@@ -1,0 +1,360 @@
+// Prefill: causal self-attention over each user's prompt (protocol step 2; Fig. 3 step 0), and the
+// hand-over of the prompt's K/V rows to the private paged cache that decode reads.
+//
+// This is the one dense contraction next to the decode path, so it runs on the fifth-generation
+// tensor cores: tcgen05.mma with both operands in 128-byte-swizzled shared memory (filled by TMA),
+// accumulators in tensor memory (TMEM).  One CTA (128 threads) owns 128 query rows of one (user,
+// query head) and walks the key blocks up to the diagonal:
+//     S = Q K^T            128 x 128 x head_dim   -> TMEM columns [0, 128)
+//     online softmax       one query row per thread (TMEM lane = row), P written to shared memory as bf16
+//     O += P V             128 x head_dim x 128   -> TMEM columns [128, 256)
+// K and V blocks are double-buffered; every wait is bounded and TMEM is freed on every way out.
+// bf16, head_dim 128.
+#pragma once
+
+#include "spd_kernels.cuh"
+
+namespace spd {
+
+constexpr int kPfBlock = 128;                       // query rows per CTA = keys per block
+constexpr int kPfTileBytes = kPfBlock * 128 * 2;    // one 128 x 128 bf16 tile: two swizzled boxes of 16 KB
+constexpr int kPfBoxBytes = kPfBlock * 128;         // 128 rows x 128 bytes
+constexpr int kPfTmemCols = 256;
+
+struct PrefillParams {
+    int32_t B, Hq, Hkv;
+    int64_t T;                   // tokens of all prompts together
+    float sm_scale;
+    const int32_t *tok_indptr;   // [B+1] token offsets of the users
+    void *out;                   // [T][Hq][128]
+    int32_t out_bf16;
+    int32_t *hdr;
+};
+
+__device__ __forceinline__ void tma_load_3d(uint32_t dst, const CUtensorMap *map, int x, int y, int z, uint32_t bar) {
+    asm volatile(
+        "cp.async.bulk.tensor.3d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3, %4}], [%5];"
+        ::"r"(dst), "l"(reinterpret_cast<uint64_t>(map)), "r"(x), "r"(y), "r"(z), "r"(bar) : "memory");
+}
+
+// Shared-memory matrix descriptor of the tensor core: start address, leading and stride byte offsets
+// (all in 16-byte units), descriptor version 1, 128-byte swizzle.
+__device__ __forceinline__ uint64_t umma_desc(uint32_t saddr, uint32_t lbo_bytes, uint32_t sbo_bytes) {
+    uint64_t d = static_cast<uint64_t>((saddr >> 4) & 0x3FFFu);
+    d |= static_cast<uint64_t>((lbo_bytes >> 4) & 0x3FFFu) << 16;
+    d |= static_cast<uint64_t>((sbo_bytes >> 4) & 0x3FFFu) << 32;
+    d |= 1ull << 46;
+    d |= 2ull << 61;
+    return d;
+}
+// Instruction descriptor: fp32 accumulate, bf16 x bf16, A K-major, B K-major or MN-major, M = N = 128.
+__device__ __forceinline__ constexpr uint32_t umma_idesc(bool b_mn_major) {
+    return (1u << 4) | (1u << 7) | (1u << 10) | ((b_mn_major ? 1u : 0u) << 16) | ((128u >> 3) << 17) | ((128u >> 4) << 24);
+}
+__device__ __forceinline__ void umma_bf16(uint32_t tmem_d, uint64_t adesc, uint64_t bdesc, uint32_t idesc, uint32_t accumulate) {
+    asm volatile(
+        "{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"
+        "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
+        ::"r"(tmem_d), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate) : "memory");
+}
+__device__ __forceinline__ void umma_commit(uint32_t bar) {
+    asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tmem_wait_ld() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
+__device__ __forceinline__ void tmem_wait_st() { asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory"); }
+
+// 32 consecutive fp32 columns of this thread's TMEM lane.
+__device__ __forceinline__ void tmem_ld32(uint32_t taddr, float (&v)[32]) {
+    uint32_t r[32];
+    asm volatile(
+        "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
+        "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
+        "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];"
+        : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]),
+          "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]),
+          "=r"(r[16]), "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]),
+          "=r"(r[24]), "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
+        : "r"(taddr) : "memory");
+    tmem_wait_ld();
+#pragma unroll
+    for (int i = 0; i < 32; ++i) v[i] = __uint_as_float(r[i]);
+}
+__device__ __forceinline__ void tmem_st32(uint32_t taddr, const float (&v)[32]) {
+    asm volatile(
+        "tcgen05.st.sync.aligned.32x32b.x32.b32 [%0], "
+        "{%1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, %16, "
+        "%17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31, %32};"
+        ::"r"(taddr),
+          "r"(__float_as_uint(v[0])), "r"(__float_as_uint(v[1])), "r"(__float_as_uint(v[2])), "r"(__float_as_uint(v[3])),
+          "r"(__float_as_uint(v[4])), "r"(__float_as_uint(v[5])), "r"(__float_as_uint(v[6])), "r"(__float_as_uint(v[7])),
+          "r"(__float_as_uint(v[8])), "r"(__float_as_uint(v[9])), "r"(__float_as_uint(v[10])), "r"(__float_as_uint(v[11])),
+          "r"(__float_as_uint(v[12])), "r"(__float_as_uint(v[13])), "r"(__float_as_uint(v[14])), "r"(__float_as_uint(v[15])),
+          "r"(__float_as_uint(v[16])), "r"(__float_as_uint(v[17])), "r"(__float_as_uint(v[18])), "r"(__float_as_uint(v[19])),
+          "r"(__float_as_uint(v[20])), "r"(__float_as_uint(v[21])), "r"(__float_as_uint(v[22])), "r"(__float_as_uint(v[23])),
+          "r"(__float_as_uint(v[24])), "r"(__float_as_uint(v[25])), "r"(__float_as_uint(v[26])), "r"(__float_as_uint(v[27])),
+          "r"(__float_as_uint(v[28])), "r"(__float_as_uint(v[29])), "r"(__float_as_uint(v[30])), "r"(__float_as_uint(v[31]))
+        : "memory");
+}
+
+constexpr size_t prefill_smem_bytes() { return 1024 + 6 * static_cast<size_t>(kPfTileBytes); }   // Q, K x2, V x2, P
+
+__global__ void __launch_bounds__(128, 1)
+prefill_kernel(const __grid_constant__ PrefillParams p, const __grid_constant__ CUtensorMap mq,
+               const __grid_constant__ CUtensorMap mk, const __grid_constant__ CUtensorMap mv) {
+    extern __shared__ uint8_t pf_smem_raw[];
+    __shared__ uint64_t bar_q, bar_kv[2], bar_mma;
+    __shared__ uint32_t tmem_slot;
+    __shared__ int32_t gave_up;
+    uint8_t *base = reinterpret_cast<uint8_t *>((reinterpret_cast<uintptr_t>(pf_smem_raw) + 1023) & ~uintptr_t(1023));
+    const uint32_t Qs = smem_u32(base), Ks = Qs + kPfTileBytes, Vs = Ks + 2 * kPfTileBytes, Ps = Vs + 2 * kPfTileBytes;
+    uint8_t *Pp = base + 5 * kPfTileBytes;
+    const int tid = threadIdx.x, wid = tid >> 5;
+    const int h = blockIdx.y, kvh = h / (p.Hq / p.Hkv);
+
+    // which (user, query block) this CTA owns; the heaviest blocks (closest to the prompt's end) come first
+    int u = 0, qb = -1, first = 0, len = 0;
+    {
+        int blk = blockIdx.x;
+        for (u = 0; u < p.B; ++u) {
+            const int64_t a = p.tok_indptr[u], b = p.tok_indptr[u + 1];
+            if (a < 0 || b < a || b > p.T) { u = p.B; break; }          // inconsistent offsets: nothing to do here
+            const int nb = static_cast<int>((b - a + kPfBlock - 1) / kPfBlock);
+            if (blk < nb) { qb = nb - 1 - blk; first = static_cast<int>(a); len = static_cast<int>(b - a); break; }
+            blk -= nb;
+        }
+    }
+    if (qb < 0) return;   // uniform over the CTA: no barrier, no TMEM touched yet
+    const int nkv = qb + 1;
+
+    if (tid == 0) {
+        mbar_init(smem_u32(&bar_q), 1);
+        mbar_init(smem_u32(&bar_kv[0]), 1);
+        mbar_init(smem_u32(&bar_kv[1]), 1);
+        mbar_init(smem_u32(&bar_mma), 1);
+        fence_mbar_init();
+        gave_up = 0;
+    }
+    if (wid == 0) {       // one warp allocates the accumulator columns for the CTA
+        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&tmem_slot)), "r"(kPfTmemCols) : "memory");
+        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+    }
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem = tmem_slot;
+    const uint32_t t_lane = tmem + (static_cast<uint32_t>(wid * 32) << 16);   // this warp's 32 lanes
+    const uint32_t tS = tmem, tO = tmem + 128;
+
+    auto load_kv = [&](int j) {           // key block j into stage j & 1
+        const int s = j & 1;
+        const uint32_t bar = smem_u32(&bar_kv[s]);
+        mbar_expect_tx(bar, 2 * kPfTileBytes);
+#pragma unroll
+        for (int b = 0; b < 2; ++b) {
+            tma_load_3d(Ks + s * kPfTileBytes + b * kPfBoxBytes, &mk, b * 64, kvh, first + j * kPfBlock, bar);
+            tma_load_3d(Vs + s * kPfTileBytes + b * kPfBoxBytes, &mv, b * 64, kvh, first + j * kPfBlock, bar);
+        }
+    };
+    if (tid == 0) {
+        const uint32_t bar = smem_u32(&bar_q);
+        mbar_expect_tx(bar, kPfTileBytes);
+        tma_load_3d(Qs, &mq, 0, h, first + qb * kPfBlock, bar);
+        tma_load_3d(Qs + kPfBoxBytes, &mq, 64, h, first + qb * kPfBlock, bar);
+        load_kv(0);
+    }
+
+    const float c2 = p.sm_scale * kLog2e;   // scores in log2 units
+    const int row = tid;                     // query row of this thread within the block
+    float m = -INFINITY, l = 0.f;
+    uint32_t mma_phase = 0;
+    // Every wait is bounded; its verdict is made uniform over the CTA (one thread's poll may run out a
+    // moment before another's succeeds), so that all threads keep meeting at the same barriers.
+    bool ok = __syncthreads_and(mbar_wait(smem_u32(&bar_q), 0));
+
+    for (int j = 0; j < nkv && ok; ++j) {
+        const int s = j & 1;
+        if (tid == 0 && j + 1 < nkv) load_kv(j + 1);       // the other stage was released by the previous block's last MMA
+        ok = __syncthreads_and(mbar_wait(smem_u32(&bar_kv[s]), (j >> 1) & 1));
+        if (!ok) break;
+        // ---- S = Q K^T ------------------------------------------------------------------------
+        if (tid == 0) {
+            tc_fence_after();
+#pragma unroll
+            for (int kk = 0; kk < 8; ++kk) {               // 16 channels per MMA; 4 MMAs per 64-channel box
+                const uint32_t off = (kk >> 2) * kPfBoxBytes + (kk & 3) * 32;
+                umma_bf16(tS, umma_desc(Qs + off, 16, 1024), umma_desc(Ks + s * kPfTileBytes + off, 16, 1024),
+                          umma_idesc(false), kk > 0 ? 1u : 0u);
+            }
+            umma_commit(smem_u32(&bar_mma));
+        }
+        ok = __syncthreads_and(mbar_wait(smem_u32(&bar_mma), mma_phase));
+        mma_phase ^= 1;
+        if (!ok) break;
+        tc_fence_after();
+        // ---- online softmax over this thread's row ------------------------------------------------
+        const bool diag = (j == qb);
+        float rmax = -INFINITY;
+#pragma unroll 1
+        for (int c = 0; c < 4; ++c) {
+            float sv[32];
+            tmem_ld32(t_lane + (tS - tmem) + c * 32, sv);
+#pragma unroll
+            for (int i = 0; i < 32; ++i) {
+                const float x = (diag && c * 32 + i > row) ? -INFINITY : sv[i] * c2;
+                rmax = fmaxf(rmax, x);
+            }
+        }
+        const float m_new = fmaxf(m, rmax);
+        const float alpha = ex2_approx(m - m_new);
+        float lsum = 0.f;
+#pragma unroll 1
+        for (int c = 0; c < 4; ++c) {
+            float sv[32];
+            tmem_ld32(t_lane + (tS - tmem) + c * 32, sv);
+            uint32_t pk[16];
+#pragma unroll
+            for (int i = 0; i < 32; i += 2) {
+                const float x0 = (diag && c * 32 + i > row) ? -INFINITY : sv[i] * c2;
+                const float x1 = (diag && c * 32 + i + 1 > row) ? -INFINITY : sv[i + 1] * c2;
+                const __nv_bfloat162 pb = __floats2bfloat162_rn(ex2_approx(x0 - m_new), ex2_approx(x1 - m_new));
+                lsum += __low2float(pb) + __high2float(pb);     // the rounded weights are the ones that multiply V
+                pk[i >> 1] = *reinterpret_cast<const uint32_t *>(&pb);
+            }
+            // P tile, K-major with 128-byte swizzle: keys 64b..64b+63 of row r at box b, line r, chunk ^ (r & 7)
+            uint8_t *line = Pp + (c >> 1) * kPfBoxBytes + row * 128;
+#pragma unroll
+            for (int q4 = 0; q4 < 4; ++q4) {
+                const int chunk = (c & 1) * 4 + q4;
+                *reinterpret_cast<uint4 *>(line + ((chunk ^ (row & 7)) << 4)) =
+                    make_uint4(pk[4 * q4], pk[4 * q4 + 1], pk[4 * q4 + 2], pk[4 * q4 + 3]);
+            }
+        }
+        l = l * alpha + lsum;
+        m = m_new;
+        // ---- rescale O where the maximum moved (skipped when no row of the warp moved) ---------------
+        if (j > 0 && !__all_sync(0xffffffffu, alpha == 1.f)) {
+#pragma unroll 1
+            for (int c = 0; c < 4; ++c) {
+                float ov[32];
+                tmem_ld32(t_lane + (tO - tmem) + c * 32, ov);
+#pragma unroll
+                for (int i = 0; i < 32; ++i) ov[i] *= alpha;
+                tmem_st32(t_lane + (tO - tmem) + c * 32, ov);
+            }
+            tmem_wait_st();
+        }
+        fence_proxy_async();     // P was written with ordinary stores; the tensor core reads it through the async proxy
+        tc_fence_before();
+        __syncthreads();
+        // ---- O += P V ---------------------------------------------------------------------------
+        if (tid == 0) {
+            tc_fence_after();
+#pragma unroll
+            for (int kk = 0; kk < 8; ++kk) {               // 16 keys per MMA
+                const uint64_t a = umma_desc(Ps + (kk >> 2) * kPfBoxBytes + (kk & 3) * 32, 16, 1024);
+                // V is [key][channel]: MN-major for the B operand; 8-key groups 1024 bytes apart, 64-channel boxes 16 KB apart
+                const uint64_t b = umma_desc(Vs + s * kPfTileBytes + kk * 2048, kPfBoxBytes, 1024);
+                umma_bf16(tO, a, b, umma_idesc(true), (j > 0 || kk > 0) ? 1u : 0u);
+            }
+            umma_commit(smem_u32(&bar_mma));
+        }
+        ok = __syncthreads_and(mbar_wait(smem_u32(&bar_mma), mma_phase));
+        mma_phase ^= 1;
+        if (!ok) break;
+        tc_fence_after();
+    }
+
+    if (!ok) gave_up = 1;
+    __syncthreads();
+    if (gave_up) {
+        if (tid == 0) flag_error(p.hdr, 6 /* SPD_ERR_TIMEOUT */, -1);
+    } else {
+        // ---- normalise and store this thread's row (every thread reads its TMEM lane; rows past the
+        //      prompt's end are not stored) --------------------------------------------------------------
+        const bool live = qb * kPfBlock + row < len;
+        const float inv = 1.f / l;
+        const int64_t tok = static_cast<int64_t>(first) + qb * kPfBlock + row;
+#pragma unroll 1
+        for (int c = 0; c < 4; ++c) {
+            float ov[32];
+            __syncwarp();        // the TMEM load is warp-wide: rows that skipped the stores rejoin here
+            tmem_ld32(t_lane + (tO - tmem) + c * 32, ov);
+            if (!live) continue;
+            if (p.out_bf16) {
+                uint4 *dst = reinterpret_cast<uint4 *>(reinterpret_cast<__nv_bfloat16 *>(p.out) + (tok * p.Hq + h) * 128 + c * 32);
+#pragma unroll
+                for (int q4 = 0; q4 < 4; ++q4)
+                    dst[q4] = make_uint4(pack_bf16(ov[8 * q4] * inv, ov[8 * q4 + 1] * inv), pack_bf16(ov[8 * q4 + 2] * inv, ov[8 * q4 + 3] * inv),
+                                         pack_bf16(ov[8 * q4 + 4] * inv, ov[8 * q4 + 5] * inv), pack_bf16(ov[8 * q4 + 6] * inv, ov[8 * q4 + 7] * inv));
+            } else {
+                float4 *dst = reinterpret_cast<float4 *>(reinterpret_cast<float *>(p.out) + (tok * p.Hq + h) * 128 + c * 32);
+#pragma unroll
+                for (int q4 = 0; q4 < 8; ++q4)
+                    dst[q4] = make_float4(ov[4 * q4] * inv, ov[4 * q4 + 1] * inv, ov[4 * q4 + 2] * inv, ov[4 * q4 + 3] * inv);
+            }
+        }
+    }
+    tc_fence_before();
+    __syncthreads();
+    if (wid == 0) asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"(kPfTmemCols) : "memory");
+}
+
+// ------------------------------------------------------------------------------------------------
+// The prompt's K and V rows into the private paged cache (what prefill leaves for decode): one CTA
+// per token.  Token t of user u goes to page indices[page_indptr[u] + t / 16], slot t % 16.  A user
+// whose listed pages cannot hold its prompt is flagged and skipped; seq_lens[u] is set for the rest.
+struct PromptKvParams {
+    int32_t B, Hkv, row_bytes;
+    int64_t T;
+    const uint8_t *k, *v;            // [T][Hkv][row_bytes]
+    const int32_t *tok_indptr;
+    uint8_t *k_pool, *v_pool;
+    int32_t num_pages;
+    const int32_t *page_indptr, *page_indices;
+    int32_t *lens;
+    int32_t *hdr;
+};
+
+__global__ void __launch_bounds__(128) prompt_kv_kernel(PromptKvParams p) {
+    __shared__ int64_t dst_row;
+    const int64_t tok = blockIdx.x;
+    if (tok == p.T) {                              // the extra block: users without a prompt hold no tokens
+        for (int u = threadIdx.x; u < p.B; u += blockDim.x)
+            if (p.tok_indptr[u + 1] == p.tok_indptr[u]) p.lens[u] = 0;
+        return;
+    }
+    if (threadIdx.x == 0) {
+        int64_t off = -1;
+        int lo = 0, hi = p.B;                      // user u with tok_indptr[u] <= tok < tok_indptr[u + 1]
+        while (hi - lo > 1) { const int mid = (lo + hi) >> 1; if (p.tok_indptr[mid] <= tok) lo = mid; else hi = mid; }
+        while (lo + 1 < p.B && p.tok_indptr[lo + 1] <= tok) ++lo;       // skip users without tokens
+        const int u = lo;
+        const int64_t a = p.tok_indptr[u], b = p.tok_indptr[u + 1], t = tok - a;
+        const int64_t plo = p.page_indptr[u], phi = p.page_indptr[u + 1];
+        bool good = a <= tok && tok < b && plo >= 0 && phi >= plo && phi <= p.page_indptr[p.B] &&
+                    (b - a) <= (phi - plo) * kPage && p.page_indices != nullptr;
+        if (good) {
+            const int64_t page = p.page_indices[plo + t / kPage];
+            if (page >= 0 && page < p.num_pages) off = ((page * p.Hkv) * kPage + t % kPage) * p.row_bytes;
+            else good = false;
+        }
+        if (!good) flag_error(p.hdr, 4 /* SPD_ERR_BAD_PAGE */, u);
+        else if (t == 0) p.lens[u] = static_cast<int32_t>(b - a);
+        dst_row = off;
+    }
+    __syncthreads();
+    const int64_t off = dst_row;
+    if (off < 0) return;
+    const int chunks = p.row_bytes / 16, total = p.Hkv * chunks;
+    for (int i = threadIdx.x; i < total; i += blockDim.x) {
+        const int hh = i / chunks, c = i - hh * chunks;
+        const int64_t src = (tok * p.Hkv + hh) * p.row_bytes + c * 16;
+        const int64_t dst = off + static_cast<int64_t>(hh) * kPage * p.row_bytes + c * 16;
+        *reinterpret_cast<uint4 *>(p.k_pool + dst) = *reinterpret_cast<const uint4 *>(p.k + src);
+        *reinterpret_cast<uint4 *>(p.v_pool + dst) = *reinterpret_cast<const uint4 *>(p.v + src);
+    }
+}
+
+}  // namespace spd

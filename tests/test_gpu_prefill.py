@@ -1,0 +1,90 @@
+"""Prefill on the GPU (tcgen05 tensor cores, accumulators in tensor memory) against the oracle: causal attention
+over ragged prompts, the hand-over of the prompts' K/V to the paged cache (bit-exact), and the first decode
+step on top of it.
+
+Tolerance of the attention output: P is rounded to bf16 before the P V product (one MMA, no hi/lo split, the
+row sum taken over the rounded weights), so each weight carries up to 2^-9 relative error; with |v| of a few
+units that allows 4e-3 max-abs on short, peaked rows and far less on long ones; rel-L2 2e-3."""
+import numpy as np
+import pytest
+import torch
+
+from oracle import spd_oracle as orc
+from paper_2409_19134_b200 import binding as spd
+from paper_2409_19134_b200 import workloads as wl
+
+pytestmark = pytest.mark.gpu
+
+TOL_ABS, TOL_REL = 4e-3, 2e-3
+
+
+def _case(lens, hq, hkv, seed, slack_pages=1):
+    B, D = len(lens), 128
+    rng = np.random.default_rng(seed)
+    gen = torch.Generator().manual_seed(seed)
+    ip = np.concatenate([[0], np.cumsum(lens)]).astype(np.int32)
+    T = int(ip[-1])
+    q = torch.randn((T, hq, D), generator=gen).to(torch.bfloat16)
+    k = torch.randn((T, hkv, D), generator=gen).to(torch.bfloat16)
+    v = torch.randn((T, hkv, D), generator=gen).to(torch.bfloat16)
+    # an empty private partition with room for the prompts: pages handed out in a shuffled order, all NaN
+    need = (np.asarray(lens) + 15) // 16 + slack_pages
+    pidx = np.concatenate([[0], np.cumsum(need)]).astype(np.int32)
+    total = int(pidx[-1])
+    perm = rng.permutation(total + 5)[:total].astype(np.int32)
+    pool = torch.full((total + 5, hkv, 16, D), float("nan"), dtype=torch.bfloat16)
+    part = wl.PagedKV(pool.clone(), pool.clone(), torch.from_numpy(pidx), torch.from_numpy(perm),
+                      torch.full((B,), -7, dtype=torch.int32))
+    return q, k, v, ip, part
+
+
+@pytest.mark.parametrize("lens,hq,hkv", [([128], 1, 1), ([100], 2, 1), ([300, 1, 129, 0, 257], 4, 2), ([1000, 640], 8, 2)])
+def test_prefill_matches_oracle_and_hands_over(lens, hq, hkv):
+    q, k, v, ip, part = _case(lens, hq, hkv, seed=sum(lens) + hq)
+    B, T = len(lens), int(ip[-1])
+    scale = 1.0 / np.sqrt(128.0)
+    rows = np.arange(T) if T <= 700 else np.unique(np.concatenate([np.arange(0, T, 37), ip[1:] - 1, ip[:-1],
+                                                                   np.array([127, 128, 255, 256, 999, 1000, 1127, 1128])]))
+    rows = rows[(rows >= 0) & (rows < T)]
+    ref = orc.prefill(orc.q_from_torch(q), orc.q_from_torch(k), orc.q_from_torch(v), ip, scale, rows)
+    shape = spd.make_shape(B, hq, hkv, 128, torch.bfloat16, scale)
+    ws = spd.alloc_workspace(shape)
+    pg = part.to("cuda")
+    out = torch.full((T, hq, 128), float("nan"), dtype=torch.float32, device="cuda")
+    spd.spd_prefill_attn(shape, q.cuda(), k.cuda(), v.cuda(), torch.from_numpy(ip).cuda(), pg, out, ws)
+    assert spd.spd_query_device_status(ws) == (spd.SPD_OK, -1)
+    got = out.cpu().numpy().astype(np.float64)[rows]
+    assert np.all(np.isfinite(got))
+    err = np.abs(got - ref)
+    assert err.max() <= TOL_ABS and np.linalg.norm(got - ref) / np.linalg.norm(ref) <= TOL_REL, (err.max(),)
+    # the cache now holds the prompts, bit for bit, and nothing else changed
+    okv = orc.kv_from_torch(part)
+    orc.write_prompt_kv(okv, orc.q_from_torch(k), orc.q_from_torch(v), ip)
+    assert np.array_equal(pg.seq_lens.cpu().numpy(), okv.seq_lens)
+    assert np.array_equal(pg.k_pool.cpu().view(torch.int16).numpy().view(np.uint16), okv.k_pool)
+    assert np.array_equal(pg.v_pool.cpu().view(torch.int16).numpy().view(np.uint16), okv.v_pool)
+    # first decode step on top of the prefilled cache: a query per user against its whole prompt
+    qd = torch.randn((B, hq, 128), generator=torch.Generator().manual_seed(3)).to(torch.bfloat16)
+    empty = wl.PagedKV(torch.zeros((1, hkv, 16, 128), dtype=torch.bfloat16), torch.zeros((1, hkv, 16, 128), dtype=torch.bfloat16),
+                       torch.zeros(B + 1, dtype=torch.int32), torch.zeros(0, dtype=torch.int32), torch.zeros(B, dtype=torch.int32))
+    yd = torch.full((B, hq, 128), float("nan"), dtype=torch.float32, device="cuda")
+    spd.spd_decode_step(shape, qd.cuda(), pg, empty.to("cuda"), yd, ws, fused=True)
+    assert spd.spd_query_device_status(ws) == (spd.SPD_OK, -1)
+    refd = orc.full(orc.q_from_torch(qd), okv, None, scale)
+    assert np.max(np.abs(yd.cpu().numpy() - refd)) <= 2e-3
+
+
+def test_prefill_bf16_output_and_full_cache_is_flagged():
+    q, k, v, ip, part = _case([200, 90], 2, 2, seed=9, slack_pages=0)
+    part.page_indptr = torch.tensor([0, 13, 18], dtype=torch.int32)        # user 1 needs 6 pages, gets 5
+    scale = 0.09
+    shape = spd.make_shape(2, 2, 2, 128, torch.bfloat16, scale)
+    ws = spd.alloc_workspace(shape)
+    pg = part.to("cuda")
+    out = torch.full((290, 2, 128), float("nan"), dtype=torch.bfloat16, device="cuda")
+    spd.spd_prefill_attn(shape, q.cuda(), k.cuda(), v.cuda(), torch.from_numpy(ip).cuda(), pg, out, ws)
+    assert spd.spd_query_device_status(ws) == (4, 1)                      # user 1's prompt does not fit its pages
+    assert pg.seq_lens.cpu().tolist() == [200, -7]
+    ref = orc.prefill(orc.q_from_torch(q), orc.q_from_torch(k), orc.q_from_torch(v), ip, scale)
+    got = out.float().cpu().numpy()
+    assert np.max(np.abs(got - ref)) <= TOL_ABS + 2.0 ** -8 * np.max(np.abs(ref))   # attention itself is still computed
