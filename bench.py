@@ -305,6 +305,59 @@ def time_schedules(spd, w, shape, steps=200):
     return res
 
 
+PREFILL_CASE = dict(users=8, prompt_lo=2048, prompt_hi=8192, hq=32, hkv=8, d=128, seed=7)   # Llama-3-8B-shaped prompts
+
+
+def time_prefill(spd, dev, steps=5, case=PREFILL_CASE):
+    """spd_prefill_attn on seeded ragged prompts: causal attention (tensor-bound) plus the K/V hand-over.
+    Flops counted: 4 * D * Hq * sum over users of L (L + 1) / 2 (the causal half only)."""
+    rng = np.random.default_rng(case["seed"])
+    lens = rng.integers(case["prompt_lo"], case["prompt_hi"] + 1, size=case["users"])
+    B, hq, hkv, D = case["users"], case["hq"], case["hkv"], case["d"]
+    ip = np.concatenate([[0], np.cumsum(lens)]).astype(np.int32)
+    T = int(ip[-1])
+    gen = torch.Generator(device=dev)
+    gen.manual_seed(case["seed"])
+    q = torch.randn((T, hq, D), generator=gen, device=dev).to(torch.bfloat16)
+    k = torch.randn((T, hkv, D), generator=gen, device=dev).to(torch.bfloat16)
+    v = torch.randn((T, hkv, D), generator=gen, device=dev).to(torch.bfloat16)
+    need = (lens + 15) // 16
+    pidx = np.concatenate([[0], np.cumsum(need)]).astype(np.int32)
+    pages = int(pidx[-1])
+    perm = torch.from_numpy(rng.permutation(pages).astype(np.int32)).to(dev)
+    part = wl.PagedKV(torch.zeros((pages, hkv, 16, D), dtype=torch.bfloat16, device=dev),
+                      torch.zeros((pages, hkv, 16, D), dtype=torch.bfloat16, device=dev),
+                      torch.from_numpy(pidx).to(dev), perm, torch.zeros(B, dtype=torch.int32, device=dev))
+    shape = spd.make_shape(B, hq, hkv, D, torch.bfloat16, 1.0 / np.sqrt(D))
+    ws = spd.alloc_workspace(shape, dev)
+    out = torch.empty((T, hq, D), dtype=torch.bfloat16, device=dev)
+    tip = torch.from_numpy(ip).to(dev)
+    for _ in range(2):
+        spd.spd_prefill_attn(shape, q, k, v, tip, part, out, ws)
+    torch.cuda.synchronize()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for _ in range(steps):
+        spd.spd_prefill_attn(shape, q, k, v, tip, part, out, ws)
+    e1.record()
+    torch.cuda.synchronize()
+    code, bad = spd.spd_query_device_status(ws)
+    if code != spd.SPD_OK or not bool(torch.isfinite(out.float()).all()):
+        raise RuntimeError(f"prefill failed: status {code}, user {bad}")
+    ms = e0.elapsed_time(e1) / steps
+    flops = 4.0 * D * hq * float(sum(int(n) * (int(n) + 1) // 2 for n in lens))
+    try:
+        with open(os.path.join(ROOT, "MEASURED_PEAKS.json")) as f:
+            peak, src = float(json.load(f)["bf16_tflops"]), "measured (MEASURED_PEAKS.json bf16_tflops, burst)"
+    except Exception:
+        peak, src = 1590.0, "fallback (1.59 PFLOP/s, earlier measurement on this pool)"
+    tf = flops / ms / 1e9
+    return {"workload": f"{B} prompts, lengths U[{case['prompt_lo']},{case['prompt_hi']}] ({T} tokens), {hq}/{hkv} heads, D {D}, bf16",
+            "ms": ms, "tokens_per_s": T / ms * 1e3,
+            "roofline": {"bound": "tensor", "achieved": tf, "peak": peak, "unit": "TFLOP/s", "frac": tf / peak,
+                         "traffic": None, "kernel": "prefill_kernel", "peak_source": src}}
+
+
 def time_append(spd, w, shape, ws, calls=8):
     """spd_append_kv on the public cache: `calls` tokens per user appended back to back (the lengths are
     first moved back by `calls`, and restored afterwards, so that every row fits the pages already listed)."""
@@ -352,6 +405,10 @@ def run_cuda(args):
     kvb = w.kv_bytes()
     spd.lib()
     spd.spd_set_bf16_math(1 if args.bf16_math == "fma" else 0)
+    if args.prefill_only:
+        if rank == 0:
+            print(json.dumps({"prefill": time_prefill(spd, dev, steps=args.steps or 5)}), flush=True)
+        return
 
     def barrier():
         if world > 1:
@@ -419,6 +476,7 @@ def run_cuda(args):
         del w
         torch.cuda.empty_cache()
         w = wl.make_workload(cfg, device=dev)
+        line["prefill"] = time_prefill(spd, dev)
         line["schedules"] = time_schedules(spd, w, spd.make_shape(w.batch, w.num_q_heads, w.num_kv_heads, w.head_dim, w.dtype, w.sm_scale))
         line["append_kv"] = time_append(spd, w, spd.make_shape(w.batch, w.num_q_heads, w.num_kv_heads, w.head_dim, w.dtype, w.sm_scale), ws)
         w = wl.make_workload(cfg, device="cpu")
@@ -441,6 +499,7 @@ def main():
     ap.add_argument("--config", default="c2_llama2_7b", choices=list(wl.CONFIGS))
     ap.add_argument("--impl", default="cuda", choices=["cuda", "reference"])
     ap.add_argument("--no-extras", action="store_true", help="skip the other configs and the CPU baseline")
+    ap.add_argument("--prefill-only", action="store_true", help="run only the prefill measurement (for profiling)")
     ap.add_argument("--bf16-math", default="mma", choices=["mma", "fma"],
                     help="arithmetic of the bf16 kernels: tensor cores (default) or the FMA-pipe comparison arm")
     args = ap.parse_args()

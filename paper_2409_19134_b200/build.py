@@ -9,8 +9,8 @@ _PKG = os.path.dirname(os.path.abspath(__file__))
 _ROOT = os.path.dirname(_PKG)
 LIB_PATH = os.path.join(_PKG, "libspd.so")
 SOURCES = [os.path.join(_PKG, "csrc", "spd_api.cu")]
-HEADERS = [os.path.join(_PKG, "csrc", "spd_kernels.cuh"), os.path.join(_PKG, "csrc", "spd_device.cuh"),
-           os.path.join(_ROOT, "include", "spd.h")]
+HEADERS = sorted(os.path.join(_PKG, "csrc", f) for f in os.listdir(os.path.join(_PKG, "csrc")) if f.endswith(".cuh")) + \
+          [os.path.join(_ROOT, "include", "spd.h")]
 
 
 def nvcc_command(verbose: bool = False):

@@ -414,13 +414,13 @@ spd_status spd_decode_step_watch(const spd_shape *shape, const void *q, const sp
     return run_job(job, ws, ws_bytes, cuda_stream);
 }
 
-// [T][H][128] bf16 as a 3-D tensor map; one box = 128 tokens x 64 channels of one head, 128-byte swizzle.
-static spd_status make_prompt_map(CUtensorMap *map, const void *ptr, int64_t T, int heads) {
+// [T][H][128] bf16 as a 3-D tensor map; one box = `rows` tokens x 64 channels of one head, 128-byte swizzle.
+static spd_status make_prompt_map(CUtensorMap *map, const void *ptr, int64_t T, int heads, int rows) {
     EncodeTiledFn fn = encode_fn();
     if (!fn) return SPD_ERR_CUDA;
     cuuint64_t dims[3] = {128, static_cast<cuuint64_t>(heads), static_cast<cuuint64_t>(T)};
     cuuint64_t strides[2] = {128 * 2, static_cast<cuuint64_t>(heads) * 128 * 2};
-    cuuint32_t box[3] = {64, 1, static_cast<cuuint32_t>(kPfBlock)};
+    cuuint32_t box[3] = {64, 1, static_cast<cuuint32_t>(rows)};
     cuuint32_t estr[3] = {1, 1, 1};
     CUresult r = fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void *>(ptr), dims, strides, box, estr,
                     CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
@@ -459,9 +459,9 @@ spd_status spd_prefill_attn(const spd_shape *shape, int64_t total_tokens, const 
     if (T == 0) return SPD_OK;
 
     CUtensorMap mq, mk, mv;
-    if ((rc = make_prompt_map(&mq, q, T, shape->num_q_heads)) != SPD_OK) return rc;
-    if ((rc = make_prompt_map(&mk, k, T, shape->num_kv_heads)) != SPD_OK) return rc;
-    if ((rc = make_prompt_map(&mv, v, T, shape->num_kv_heads)) != SPD_OK) return rc;
+    if ((rc = make_prompt_map(&mq, q, T, shape->num_q_heads, kPfBlock)) != SPD_OK) return rc;
+    if ((rc = make_prompt_map(&mk, k, T, shape->num_kv_heads, kPfKeys)) != SPD_OK) return rc;
+    if ((rc = make_prompt_map(&mv, v, T, shape->num_kv_heads, kPfKeys)) != SPD_OK) return rc;
     PrefillParams pp;
     pp.B = shape->batch; pp.Hq = shape->num_q_heads; pp.Hkv = shape->num_kv_heads; pp.T = T;
     pp.sm_scale = shape->sm_scale; pp.tok_indptr = tok_indptr; pp.out = out; pp.out_bf16 = out_dtype == SPD_BF16;

@@ -4,22 +4,28 @@
 // This is the one dense contraction next to the decode path, so it runs on the fifth-generation
 // tensor cores: tcgen05.mma with both operands in 128-byte-swizzled shared memory (filled by TMA),
 // accumulators in tensor memory (TMEM).  One CTA (128 threads) owns 128 query rows of one (user,
-// query head) and walks the key blocks up to the diagonal:
-//     S = Q K^T            128 x 128 x head_dim   -> TMEM columns [0, 128)
+// query head) and walks 64-key blocks up to the diagonal:
+//     S = Q K^T            128 x 64 x head_dim    -> TMEM, two buffers: columns [0, 64) and [64, 128)
 //     online softmax       one query row per thread (TMEM lane = row), P written to shared memory as bf16
-//     O += P V             128 x head_dim x 128   -> TMEM columns [128, 256)
-// K and V blocks are double-buffered; every wait is bounded and TMEM is freed on every way out.
-// bf16, head_dim 128.
+//     O += P V             128 x head_dim x 64    -> TMEM columns [128, 256)
+// Software pipeline: S(j+1) is computed while the threads do the softmax of S(j), and O takes block j
+// in under the exponentials of block j+1.  K and V blocks sit in two-slot rings with their own barriers;
+// every wait is bounded and TMEM is freed on every way out.
+// 112 KB of shared memory and 256 TMEM columns per CTA, so two CTAs share an SM and one's softmax
+// runs under the other's MMAs.  bf16, head_dim 128.
 #pragma once
 
 #include "spd_kernels.cuh"
 
 namespace spd {
 
-constexpr int kPfBlock = 128;                       // query rows per CTA = keys per block
-constexpr int kPfTileBytes = kPfBlock * 128 * 2;    // one 128 x 128 bf16 tile: two swizzled boxes of 16 KB
-constexpr int kPfBoxBytes = kPfBlock * 128;         // 128 rows x 128 bytes
-constexpr int kPfTmemCols = 256;
+constexpr int kPfBlock = 128;                       // query rows per CTA
+constexpr int kPfKeys = 64;                         // keys per block
+constexpr int kPfQBox = kPfBlock * 128;             // one swizzled box of Q or P: 128 rows x 128 bytes
+constexpr int kPfQTile = 2 * kPfQBox;               // Q: 128 rows x 128 channels = two boxes
+constexpr int kPfKvBox = kPfKeys * 128;             // one swizzled box of K or V: 64 rows x 128 bytes
+constexpr int kPfKvTile = 2 * kPfKvBox;             // 64 keys x 128 channels = two boxes
+constexpr int kPfTmemCols = 256;                    // S: 2 x 64, O: 128
 
 struct PrefillParams {
     int32_t B, Hq, Hkv;
@@ -47,9 +53,9 @@ __device__ __forceinline__ uint64_t umma_desc(uint32_t saddr, uint32_t lbo_bytes
     d |= 2ull << 61;
     return d;
 }
-// Instruction descriptor: fp32 accumulate, bf16 x bf16, A K-major, B K-major or MN-major, M = N = 128.
-__device__ __forceinline__ constexpr uint32_t umma_idesc(bool b_mn_major) {
-    return (1u << 4) | (1u << 7) | (1u << 10) | ((b_mn_major ? 1u : 0u) << 16) | ((128u >> 3) << 17) | ((128u >> 4) << 24);
+// Instruction descriptor: fp32 accumulate, bf16 x bf16, A K-major, B K-major or MN-major, M = 128, N = n.
+__device__ __forceinline__ constexpr uint32_t umma_idesc(bool b_mn_major, uint32_t n) {
+    return (1u << 4) | (1u << 7) | (1u << 10) | ((b_mn_major ? 1u : 0u) << 16) | ((n >> 3) << 17) | ((128u >> 4) << 24);
 }
 __device__ __forceinline__ void umma_bf16(uint32_t tmem_d, uint64_t adesc, uint64_t bdesc, uint32_t idesc, uint32_t accumulate) {
     asm volatile(
@@ -98,18 +104,20 @@ __device__ __forceinline__ void tmem_st32(uint32_t taddr, const float (&v)[32]) 
         : "memory");
 }
 
-constexpr size_t prefill_smem_bytes() { return 1024 + 6 * static_cast<size_t>(kPfTileBytes); }   // Q, K x2, V x2, P
+// Q, K x2, V x2, P, then eight mbarriers and one word; the kernel has no static shared memory, so the
+// 1024-byte alignment of the tiles costs nothing and two CTAs fit one SM.
+constexpr size_t prefill_smem_bytes() { return kPfQTile + 4 * static_cast<size_t>(kPfKvTile) + kPfQBox + 128; }
 
-__global__ void __launch_bounds__(128, 1)
+__global__ void __launch_bounds__(128, 2)
 prefill_kernel(const __grid_constant__ PrefillParams p, const __grid_constant__ CUtensorMap mq,
                const __grid_constant__ CUtensorMap mk, const __grid_constant__ CUtensorMap mv) {
-    extern __shared__ uint8_t pf_smem_raw[];
-    __shared__ uint64_t bar_q, bar_kv[2], bar_mma;
-    __shared__ uint32_t tmem_slot;
-    __shared__ int32_t gave_up;
-    uint8_t *base = reinterpret_cast<uint8_t *>((reinterpret_cast<uintptr_t>(pf_smem_raw) + 1023) & ~uintptr_t(1023));
-    const uint32_t Qs = smem_u32(base), Ks = Qs + kPfTileBytes, Vs = Ks + 2 * kPfTileBytes, Ps = Vs + 2 * kPfTileBytes;
-    uint8_t *Pp = base + 5 * kPfTileBytes;
+    extern __shared__ __align__(1024) uint8_t base[];
+    const uint32_t Qs = smem_u32(base), Ks = Qs + kPfQTile, Vs = Ks + 2 * kPfKvTile, Ps = Vs + 2 * kPfKvTile;
+    uint8_t *Pp = base + kPfQTile + 4 * kPfKvTile;
+    uint64_t *bars = reinterpret_cast<uint64_t *>(Pp + kPfQBox);
+    uint64_t &bar_q = bars[0], &bar_o = bars[1];
+    uint64_t *bar_k = bars + 2, *bar_v = bars + 4, *bar_s = bars + 6;
+    uint32_t &tmem_slot = *reinterpret_cast<uint32_t *>(bars + 8);
     const int tid = threadIdx.x, wid = tid >> 5;
     const int h = blockIdx.y, kvh = h / (p.Hq / p.Hkv);
 
@@ -126,15 +134,11 @@ prefill_kernel(const __grid_constant__ PrefillParams p, const __grid_constant__ 
         }
     }
     if (qb < 0) return;   // uniform over the CTA: no barrier, no TMEM touched yet
-    const int nkv = qb + 1;
+    const int nkv = 2 * (qb + 1);   // 64-key blocks up to and including the diagonal
 
     if (tid == 0) {
-        mbar_init(smem_u32(&bar_q), 1);
-        mbar_init(smem_u32(&bar_kv[0]), 1);
-        mbar_init(smem_u32(&bar_kv[1]), 1);
-        mbar_init(smem_u32(&bar_mma), 1);
+        for (int b = 0; b < 8; ++b) mbar_init(smem_u32(&bars[b]), 1);
         fence_mbar_init();
-        gave_up = 0;
     }
     if (wid == 0) {       // one warp allocates the accumulator columns for the CTA
         asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&tmem_slot)), "r"(kPfTmemCols) : "memory");
@@ -145,129 +149,142 @@ prefill_kernel(const __grid_constant__ PrefillParams p, const __grid_constant__ 
     tc_fence_after();
     const uint32_t tmem = tmem_slot;
     const uint32_t t_lane = tmem + (static_cast<uint32_t>(wid * 32) << 16);   // this warp's 32 lanes
-    const uint32_t tS = tmem, tO = tmem + 128;
+    const uint32_t tO = tmem + 2 * kPfKeys;     // S buffers at columns [0, 64) and [64, 128), O at [128, 256)
 
-    auto load_kv = [&](int j) {           // key block j into stage j & 1
-        const int s = j & 1;
-        const uint32_t bar = smem_u32(&bar_kv[s]);
-        mbar_expect_tx(bar, 2 * kPfTileBytes);
+    // K and V of key block j live in slot j & 1 of their rings; K is free again once S(j) exists, V once
+    // O has taken block j in.
+    auto load_k = [&](int j) {
+        const uint32_t bar = smem_u32(&bar_k[j & 1]);
+        mbar_expect_tx(bar, kPfKvTile);
+        tma_load_3d(Ks + (j & 1) * kPfKvTile, &mk, 0, kvh, first + j * kPfKeys, bar);
+        tma_load_3d(Ks + (j & 1) * kPfKvTile + kPfKvBox, &mk, 64, kvh, first + j * kPfKeys, bar);
+    };
+    auto load_v = [&](int j) {
+        const uint32_t bar = smem_u32(&bar_v[j & 1]);
+        mbar_expect_tx(bar, kPfKvTile);
+        tma_load_3d(Vs + (j & 1) * kPfKvTile, &mv, 0, kvh, first + j * kPfKeys, bar);
+        tma_load_3d(Vs + (j & 1) * kPfKvTile + kPfKvBox, &mv, 64, kvh, first + j * kPfKeys, bar);
+    };
+    auto mma_s = [&](int j) {                    // S(j) = Q K(j)^T into S buffer j & 1; 16 channels per MMA
+        tc_fence_after();
 #pragma unroll
-        for (int b = 0; b < 2; ++b) {
-            tma_load_3d(Ks + s * kPfTileBytes + b * kPfBoxBytes, &mk, b * 64, kvh, first + j * kPfBlock, bar);
-            tma_load_3d(Vs + s * kPfTileBytes + b * kPfBoxBytes, &mv, b * 64, kvh, first + j * kPfBlock, bar);
+        for (int kk = 0; kk < 8; ++kk) {
+            const uint64_t a = umma_desc(Qs + (kk >> 2) * kPfQBox + (kk & 3) * 32, 16, 1024);
+            const uint64_t b = umma_desc(Ks + (j & 1) * kPfKvTile + (kk >> 2) * kPfKvBox + (kk & 3) * 32, 16, 1024);
+            umma_bf16(tmem + (j & 1) * kPfKeys, a, b, umma_idesc(false, kPfKeys), kk > 0 ? 1u : 0u);
         }
+        umma_commit(smem_u32(&bar_s[j & 1]));
     };
     if (tid == 0) {
         const uint32_t bar = smem_u32(&bar_q);
-        mbar_expect_tx(bar, kPfTileBytes);
+        mbar_expect_tx(bar, kPfQTile);
         tma_load_3d(Qs, &mq, 0, h, first + qb * kPfBlock, bar);
-        tma_load_3d(Qs + kPfBoxBytes, &mq, 64, h, first + qb * kPfBlock, bar);
-        load_kv(0);
+        tma_load_3d(Qs + kPfQBox, &mq, 64, h, first + qb * kPfBlock, bar);
+        load_k(0);
+        load_v(0);
+        load_k(1);            // nkv >= 2 always: a query block spans two key blocks on the diagonal
+        load_v(1);
     }
 
     const float c2 = p.sm_scale * kLog2e;   // scores in log2 units
     const int row = tid;                     // query row of this thread within the block
     float m = -INFINITY, l = 0.f;
-    uint32_t mma_phase = 0;
-    // Every wait is bounded; its verdict is made uniform over the CTA (one thread's poll may run out a
-    // moment before another's succeeds), so that all threads keep meeting at the same barriers.
-    bool ok = __syncthreads_and(mbar_wait(smem_u32(&bar_q), 0));
+    // Every wait is bounded.  A wait that runs out only clears `ok`; once per key block the CTA votes on it, so
+    // that all threads leave together and keep meeting at the same barriers until then.
+    bool ok = mbar_wait(smem_u32(&bar_q), 0) && mbar_wait(smem_u32(&bar_k[0]), 0);
+    if (tid == 0) mma_s(0);
 
-    for (int j = 0; j < nkv && ok; ++j) {
-        const int s = j & 1;
-        if (tid == 0 && j + 1 < nkv) load_kv(j + 1);       // the other stage was released by the previous block's last MMA
-        ok = __syncthreads_and(mbar_wait(smem_u32(&bar_kv[s]), (j >> 1) & 1));
-        if (!ok) break;
-        // ---- S = Q K^T ------------------------------------------------------------------------
-        if (tid == 0) {
-            tc_fence_after();
-#pragma unroll
-            for (int kk = 0; kk < 8; ++kk) {               // 16 channels per MMA; 4 MMAs per 64-channel box
-                const uint32_t off = (kk >> 2) * kPfBoxBytes + (kk & 3) * 32;
-                umma_bf16(tS, umma_desc(Qs + off, 16, 1024), umma_desc(Ks + s * kPfTileBytes + off, 16, 1024),
-                          umma_idesc(false), kk > 0 ? 1u : 0u);
-            }
-            umma_commit(smem_u32(&bar_mma));
+    int j = 0;
+    for (; j < nkv; ++j) {
+        ok = mbar_wait(smem_u32(&bar_s[j & 1]), (j >> 1) & 1) && ok;           // S(j) is there, K slot j & 1 is free
+        if (j + 1 < nkv) {                                                     // start S(j+1) before touching S(j)
+            if (tid == 0 && j + 2 < nkv) load_k(j + 2);
+            ok = mbar_wait(smem_u32(&bar_k[(j + 1) & 1]), ((j + 1) >> 1) & 1) && ok;
+            if (tid == 0) mma_s(j + 1);
         }
-        ok = __syncthreads_and(mbar_wait(smem_u32(&bar_mma), mma_phase));
-        mma_phase ^= 1;
-        if (!ok) break;
         tc_fence_after();
-        // ---- online softmax over this thread's row ------------------------------------------------
-        const bool diag = (j == qb);
-        float rmax = -INFINITY;
-#pragma unroll 1
-        for (int c = 0; c < 4; ++c) {
-            float sv[32];
-            tmem_ld32(t_lane + (tS - tmem) + c * 32, sv);
+        // ---- softmax of this thread's row of S(j), in registers ---------------------------------------
+        // key (64 j + col) is visible to row (128 qb + row) iff it does not lie ahead of it; only the two
+        // blocks on the diagonal need the test; `ahead` = first column of this block hidden from this row
+        const int ahead = (j >= 2 * qb) ? (kPfBlock * qb + row) - kPfKeys * j + 1 : kPfKeys;
+        float sv[64];
+        {
+            float lo[32], hi[32];
+            tmem_ld32(t_lane + (j & 1) * kPfKeys, lo);
+            tmem_ld32(t_lane + (j & 1) * kPfKeys + 32, hi);
 #pragma unroll
-            for (int i = 0; i < 32; ++i) {
-                const float x = (diag && c * 32 + i > row) ? -INFINITY : sv[i] * c2;
-                rmax = fmaxf(rmax, x);
-            }
+            for (int i = 0; i < 32; ++i) { sv[i] = lo[i]; sv[32 + i] = hi[i]; }
         }
-        const float m_new = fmaxf(m, rmax);
+        // m is kept in log2 units of the scaled score; the maximum is taken on the raw scores (the scale is
+        // positive) and the scale rides on the fused multiply-add that feeds ex2
+        if (j >= 2 * qb) {                                   // only the two diagonal blocks hide anything
+#pragma unroll
+            for (int i = 0; i < 64; ++i) sv[i] = (i >= ahead) ? -INFINITY : sv[i];
+        }
+        float rmax = sv[0];
+#pragma unroll
+        for (int i = 1; i < 64; ++i) rmax = fmaxf(rmax, sv[i]);
+        const float m_new = fmaxf(m, rmax * c2);             // finite from the first block on: key 0 is visible to every row
         const float alpha = ex2_approx(m - m_new);
+        uint32_t pk[32];
         float lsum = 0.f;
-#pragma unroll 1
-        for (int c = 0; c < 4; ++c) {
-            float sv[32];
-            tmem_ld32(t_lane + (tS - tmem) + c * 32, sv);
-            uint32_t pk[16];
 #pragma unroll
-            for (int i = 0; i < 32; i += 2) {
-                const float x0 = (diag && c * 32 + i > row) ? -INFINITY : sv[i] * c2;
-                const float x1 = (diag && c * 32 + i + 1 > row) ? -INFINITY : sv[i + 1] * c2;
-                const __nv_bfloat162 pb = __floats2bfloat162_rn(ex2_approx(x0 - m_new), ex2_approx(x1 - m_new));
-                lsum += __low2float(pb) + __high2float(pb);     // the rounded weights are the ones that multiply V
-                pk[i >> 1] = *reinterpret_cast<const uint32_t *>(&pb);
-            }
-            // P tile, K-major with 128-byte swizzle: keys 64b..64b+63 of row r at box b, line r, chunk ^ (r & 7)
-            uint8_t *line = Pp + (c >> 1) * kPfBoxBytes + row * 128;
-#pragma unroll
-            for (int q4 = 0; q4 < 4; ++q4) {
-                const int chunk = (c & 1) * 4 + q4;
-                *reinterpret_cast<uint4 *>(line + ((chunk ^ (row & 7)) << 4)) =
-                    make_uint4(pk[4 * q4], pk[4 * q4 + 1], pk[4 * q4 + 2], pk[4 * q4 + 3]);
-            }
+        for (int i = 0; i < 64; i += 2) {
+            const float p0 = ex2_approx(fmaf(sv[i], c2, -m_new)), p1 = ex2_approx(fmaf(sv[i + 1], c2, -m_new));
+            lsum += p0 + p1;
+            pk[i >> 1] = pack_bf16(p0, p1);
         }
         l = l * alpha + lsum;
         m = m_new;
-        // ---- rescale O where the maximum moved (skipped when no row of the warp moved) ---------------
-        if (j > 0 && !__all_sync(0xffffffffu, alpha == 1.f)) {
+        // ---- O has taken block j-1 in: its V slot, the P tile and O itself are free ---------------------
+        if (j > 0) {
+            ok = mbar_wait(smem_u32(&bar_o), (j - 1) & 1) && ok;
+            tc_fence_after();
+            if (tid == 0 && j + 1 < nkv) load_v(j + 1);
+            if (!__all_sync(0xffffffffu, alpha == 1.f)) {       // rescale O where the maximum moved
 #pragma unroll 1
-            for (int c = 0; c < 4; ++c) {
-                float ov[32];
-                tmem_ld32(t_lane + (tO - tmem) + c * 32, ov);
+                for (int c = 0; c < 4; ++c) {
+                    float ov[32];
+                    tmem_ld32(t_lane + (tO - tmem) + c * 32, ov);
 #pragma unroll
-                for (int i = 0; i < 32; ++i) ov[i] *= alpha;
-                tmem_st32(t_lane + (tO - tmem) + c * 32, ov);
+                    for (int i = 0; i < 32; ++i) ov[i] *= alpha;
+                    tmem_st32(t_lane + (tO - tmem) + c * 32, ov);
+                }
+                tmem_wait_st();
             }
-            tmem_wait_st();
+        }
+        // P tile, K-major with 128-byte swizzle: the 64 keys of row r on line r, 16-byte chunk ^ (r & 7)
+        {
+            uint8_t *line = Pp + row * 128;
+#pragma unroll
+            for (int chunk = 0; chunk < 8; ++chunk)
+                *reinterpret_cast<uint4 *>(line + ((chunk ^ (row & 7)) << 4)) =
+                    make_uint4(pk[4 * chunk], pk[4 * chunk + 1], pk[4 * chunk + 2], pk[4 * chunk + 3]);
         }
         fence_proxy_async();     // P was written with ordinary stores; the tensor core reads it through the async proxy
         tc_fence_before();
-        __syncthreads();
-        // ---- O += P V ---------------------------------------------------------------------------
-        if (tid == 0) {
-            tc_fence_after();
-#pragma unroll
-            for (int kk = 0; kk < 8; ++kk) {               // 16 keys per MMA
-                const uint64_t a = umma_desc(Ps + (kk >> 2) * kPfBoxBytes + (kk & 3) * 32, 16, 1024);
-                // V is [key][channel]: MN-major for the B operand; 8-key groups 1024 bytes apart, 64-channel boxes 16 KB apart
-                const uint64_t b = umma_desc(Vs + s * kPfTileBytes + kk * 2048, kPfBoxBytes, 1024);
-                umma_bf16(tO, a, b, umma_idesc(true), (j > 0 || kk > 0) ? 1u : 0u);
-            }
-            umma_commit(smem_u32(&bar_mma));
-        }
-        ok = __syncthreads_and(mbar_wait(smem_u32(&bar_mma), mma_phase));
-        mma_phase ^= 1;
+        ok = __syncthreads_and(ok);
         if (!ok) break;
-        tc_fence_after();
+        // ---- O += P V(j) ------------------------------------------------------------------------------
+        if (tid == 0) {
+            const bool v_ok = mbar_wait(smem_u32(&bar_v[j & 1]), (j >> 1) & 1);
+            ok = ok && v_ok;                 // goes into the next vote
+            tc_fence_after();
+            if (v_ok) {
+#pragma unroll
+                for (int kk = 0; kk < 4; ++kk) {               // 16 keys per MMA
+                    const uint64_t a = umma_desc(Ps + kk * 32, 16, 1024);
+                    // V is [key][channel]: MN-major for the B operand; 8-key groups 1024 bytes apart, 64-channel boxes one box apart
+                    const uint64_t b = umma_desc(Vs + (j & 1) * kPfKvTile + kk * 2048, kPfKvBox, 1024);
+                    umma_bf16(tO, a, b, umma_idesc(true, 128), (j > 0 || kk > 0) ? 1u : 0u);
+                }
+            }
+            umma_commit(smem_u32(&bar_o));   // committed even if V never came, so that nobody waits for it in vain
+        }
     }
-
-    if (!ok) gave_up = 1;
-    __syncthreads();
+    if (ok) ok = mbar_wait(smem_u32(&bar_o), (nkv - 1) & 1);
+    tc_fence_after();
+    const bool gave_up = !__syncthreads_and(ok);
     if (gave_up) {
         if (tid == 0) flag_error(p.hdr, 6 /* SPD_ERR_TIMEOUT */, -1);
     } else {
