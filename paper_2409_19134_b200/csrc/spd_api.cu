@@ -477,7 +477,7 @@ spd_status spd_prefill_attn(const spd_shape *shape, int64_t total_tokens, const 
     if (attr_err != cudaSuccess) return SPD_ERR_CUDA;
     const int64_t max_blocks = (T + kPfBlock - 1) / kPfBlock + shape->batch;   // >= sum over users of ceil(len / 128)
     dim3 grid(static_cast<unsigned>(max_blocks), static_cast<unsigned>(shape->num_q_heads));
-    prefill_kernel<<<grid, 128, prefill_smem_bytes(), st>>>(pp, mq, mk, mv);
+    prefill_kernel<<<grid, kPfThreads, prefill_smem_bytes(), st>>>(pp, mq, mk, mv);
     ++g_launches;
     return cudaGetLastError() == cudaSuccess ? SPD_OK : SPD_ERR_CUDA;
 }

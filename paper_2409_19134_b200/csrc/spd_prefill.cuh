@@ -8,9 +8,11 @@
 //     S = Q K^T            128 x 64 x head_dim    -> TMEM, two buffers: columns [0, 64) and [64, 128)
 //     online softmax       one query row per thread (TMEM lane = row), P written to shared memory as bf16
 //     O += P V             128 x head_dim x 64    -> TMEM columns [128, 256)
-// Software pipeline: S(j+1) is computed while the threads do the softmax of S(j), and O takes block j
-// in under the exponentials of block j+1.  K and V blocks sit in two-slot rings with their own barriers;
-// every wait is bounded and TMEM is freed on every way out.
+// Warp-specialised software pipeline: four warps do the softmax (one row per thread), one thread of a
+// fifth warp issues every TMA load and every MMA.  S(j+1) is computed while the softmax warps work on
+// S(j), and O takes block j in under the exponentials of block j+1.  They hand over through mbarriers
+// only (S ready, S consumed, P ready, O updated): no CTA-wide barrier inside the loop.  K and V blocks
+// sit in two-slot rings with their own barriers; every wait is bounded and TMEM is freed on every way out.
 // 112 KB of shared memory and 256 TMEM columns per CTA, so two CTAs share an SM and one's softmax
 // runs under the other's MMAs.  bf16, head_dim 128.
 #pragma once
@@ -104,20 +106,23 @@ __device__ __forceinline__ void tmem_st32(uint32_t taddr, const float (&v)[32]) 
         : "memory");
 }
 
-// Q, K x2, V x2, P, then eight mbarriers and one word; the kernel has no static shared memory, so the
+// Q, K x2, V x2, P, then eleven mbarriers and one word; the kernel has no static shared memory, so the
 // 1024-byte alignment of the tiles costs nothing and two CTAs fit one SM.
-constexpr size_t prefill_smem_bytes() { return kPfQTile + 4 * static_cast<size_t>(kPfKvTile) + kPfQBox + 128; }
+constexpr size_t prefill_smem_bytes() { return kPfQTile + 4 * static_cast<size_t>(kPfKvTile) + kPfQBox + 128; }   // 11 x 8 + 4 <= 128
 
-__global__ void __launch_bounds__(128, 2)
+constexpr int kPfThreads = 160;   // 4 softmax warps + 1 warp that issues loads and MMAs
+
+__global__ void __launch_bounds__(kPfThreads, 2)
 prefill_kernel(const __grid_constant__ PrefillParams p, const __grid_constant__ CUtensorMap mq,
                const __grid_constant__ CUtensorMap mk, const __grid_constant__ CUtensorMap mv) {
     extern __shared__ __align__(1024) uint8_t base[];
     const uint32_t Qs = smem_u32(base), Ks = Qs + kPfQTile, Vs = Ks + 2 * kPfKvTile, Ps = Vs + 2 * kPfKvTile;
     uint8_t *Pp = base + kPfQTile + 4 * kPfKvTile;
     uint64_t *bars = reinterpret_cast<uint64_t *>(Pp + kPfQBox);
-    uint64_t &bar_q = bars[0], &bar_o = bars[1];
-    uint64_t *bar_k = bars + 2, *bar_v = bars + 4, *bar_s = bars + 6;
-    uint32_t &tmem_slot = *reinterpret_cast<uint32_t *>(bars + 8);
+    uint64_t &bar_q = bars[0], &bar_o = bars[1], &bar_p = bars[2];        // Q loaded; O updated; P written
+    uint64_t *bar_k = bars + 3, *bar_v = bars + 5, *bar_s = bars + 7;     // K / V slot loaded; S buffer ready
+    uint64_t *bar_sfree = bars + 9;                                         // S buffer read by all softmax threads
+    uint32_t &tmem_slot = *reinterpret_cast<uint32_t *>(bars + 11);
     const int tid = threadIdx.x, wid = tid >> 5;
     const int h = blockIdx.y, kvh = h / (p.Hq / p.Hkv);
 
@@ -137,7 +142,7 @@ prefill_kernel(const __grid_constant__ PrefillParams p, const __grid_constant__ 
     const int nkv = 2 * (qb + 1);   // 64-key blocks up to and including the diagonal
 
     if (tid == 0) {
-        for (int b = 0; b < 8; ++b) mbar_init(smem_u32(&bars[b]), 1);
+        for (int b = 0; b < 11; ++b) mbar_init(smem_u32(&bars[b]), (b == 2 || b >= 9) ? 128 : 1);   // P and S-consumed: every softmax thread arrives
         fence_mbar_init();
     }
     if (wid == 0) {       // one warp allocates the accumulator columns for the CTA
@@ -175,119 +180,122 @@ prefill_kernel(const __grid_constant__ PrefillParams p, const __grid_constant__ 
         }
         umma_commit(smem_u32(&bar_s[j & 1]));
     };
-    if (tid == 0) {
-        const uint32_t bar = smem_u32(&bar_q);
-        mbar_expect_tx(bar, kPfQTile);
-        tma_load_3d(Qs, &mq, 0, h, first + qb * kPfBlock, bar);
-        tma_load_3d(Qs + kPfQBox, &mq, 64, h, first + qb * kPfBlock, bar);
-        load_k(0);
-        load_v(0);
-        load_k(1);            // nkv >= 2 always: a query block spans two key blocks on the diagonal
-        load_v(1);
-    }
-
     const float c2 = p.sm_scale * kLog2e;   // scores in log2 units
-    const int row = tid;                     // query row of this thread within the block
-    float m = -INFINITY, l = 0.f;
-    // Every wait is bounded.  A wait that runs out only clears `ok`; once per key block the CTA votes on it, so
-    // that all threads leave together and keep meeting at the same barriers until then.
-    bool ok = mbar_wait(smem_u32(&bar_q), 0) && mbar_wait(smem_u32(&bar_k[0]), 0);
-    if (tid == 0) mma_s(0);
+    const int row = tid;                     // query row of a softmax thread within the block
+    float l = 0.f;
+    // Every wait is bounded.  A wait that runs out clears `ok` and the thread carries on (with garbage, but
+    // towards the same end): nothing in the loop waits for all threads, so nobody can be left behind.
+    bool ok = true;
 
-    int j = 0;
-    for (; j < nkv; ++j) {
-        ok = mbar_wait(smem_u32(&bar_s[j & 1]), (j >> 1) & 1) && ok;           // S(j) is there, K slot j & 1 is free
-        if (j + 1 < nkv) {                                                     // start S(j+1) before touching S(j)
-            if (tid == 0 && j + 2 < nkv) load_k(j + 2);
-            ok = mbar_wait(smem_u32(&bar_k[(j + 1) & 1]), ((j + 1) >> 1) & 1) && ok;
-            if (tid == 0) mma_s(j + 1);
-        }
-        tc_fence_after();
-        // ---- softmax of this thread's row of S(j), in registers ---------------------------------------
-        // key (64 j + col) is visible to row (128 qb + row) iff it does not lie ahead of it; only the two
-        // blocks on the diagonal need the test; `ahead` = first column of this block hidden from this row
-        const int ahead = (j >= 2 * qb) ? (kPfBlock * qb + row) - kPfKeys * j + 1 : kPfKeys;
-        float sv[64];
-        {
-            float lo[32], hi[32];
-            tmem_ld32(t_lane + (j & 1) * kPfKeys, lo);
-            tmem_ld32(t_lane + (j & 1) * kPfKeys + 32, hi);
-#pragma unroll
-            for (int i = 0; i < 32; ++i) { sv[i] = lo[i]; sv[32 + i] = hi[i]; }
-        }
-        // m is kept in log2 units of the scaled score; the maximum is taken on the raw scores (the scale is
-        // positive) and the scale rides on the fused multiply-add that feeds ex2
-        if (j >= 2 * qb) {                                   // only the two diagonal blocks hide anything
-#pragma unroll
-            for (int i = 0; i < 64; ++i) sv[i] = (i >= ahead) ? -INFINITY : sv[i];
-        }
-        float rmax = sv[0];
-#pragma unroll
-        for (int i = 1; i < 64; ++i) rmax = fmaxf(rmax, sv[i]);
-        const float m_new = fmaxf(m, rmax * c2);             // finite from the first block on: key 0 is visible to every row
-        const float alpha = ex2_approx(m - m_new);
-        uint32_t pk[32];
-        float lsum = 0.f;
-#pragma unroll
-        for (int i = 0; i < 64; i += 2) {
-            const float p0 = ex2_approx(fmaf(sv[i], c2, -m_new)), p1 = ex2_approx(fmaf(sv[i + 1], c2, -m_new));
-            lsum += p0 + p1;
-            pk[i >> 1] = pack_bf16(p0, p1);
-        }
-        l = l * alpha + lsum;
-        m = m_new;
-        // ---- O has taken block j-1 in: its V slot, the P tile and O itself are free ---------------------
-        if (j > 0) {
-            ok = mbar_wait(smem_u32(&bar_o), (j - 1) & 1) && ok;
-            tc_fence_after();
-            if (tid == 0 && j + 1 < nkv) load_v(j + 1);
-            if (!__all_sync(0xffffffffu, alpha == 1.f)) {       // rescale O where the maximum moved
-#pragma unroll 1
-                for (int c = 0; c < 4; ++c) {
-                    float ov[32];
-                    tmem_ld32(t_lane + (tO - tmem) + c * 32, ov);
-#pragma unroll
-                    for (int i = 0; i < 32; ++i) ov[i] *= alpha;
-                    tmem_st32(t_lane + (tO - tmem) + c * 32, ov);
+    if (wid == 4) {
+        // ---------------- the issuing thread: TMA loads and MMAs ----------------------------------------
+        if (tid == 128) {
+            const uint32_t bq = smem_u32(&bar_q);
+            mbar_expect_tx(bq, kPfQTile);
+            tma_load_3d(Qs, &mq, 0, h, first + qb * kPfBlock, bq);
+            tma_load_3d(Qs + kPfQBox, &mq, 64, h, first + qb * kPfBlock, bq);
+            load_k(0);
+            load_v(0);
+            load_k(1);            // nkv >= 2 always: a query block spans two key blocks on the diagonal
+            load_v(1);
+            ok = mbar_wait(bq, 0) && mbar_wait(smem_u32(&bar_k[0]), 0);
+            mma_s(0);
+            for (int j = 0; j < nkv; ++j) {
+                if (j + 1 < nkv) {                     // S(j+1): needs K(j+1) and the other S buffer read out (S(j-1))
+                    ok = mbar_wait(smem_u32(&bar_k[(j + 1) & 1]), ((j + 1) >> 1) & 1) && ok;
+                    if (j > 0) ok = mbar_wait(smem_u32(&bar_sfree[(j + 1) & 1]), ((j - 1) >> 1) & 1) && ok;
+                    mma_s(j + 1);
                 }
-                tmem_wait_st();
-            }
-        }
-        // P tile, K-major with 128-byte swizzle: the 64 keys of row r on line r, 16-byte chunk ^ (r & 7)
-        {
-            uint8_t *line = Pp + row * 128;
+                // P(j) is written and O rescaled: S(j) was read, so K slot j & 1 is free; and the softmax
+                // threads saw O take block j-1 in, so V slot (j-1) & 1 is free
+                ok = mbar_wait(smem_u32(&bar_p), j & 1) && ok;
+                if (j + 2 < nkv) load_k(j + 2);
+                if (j > 0 && j + 1 < nkv) load_v(j + 1);
+                ok = mbar_wait(smem_u32(&bar_v[j & 1]), (j >> 1) & 1) && ok;
+                tc_fence_after();
 #pragma unroll
-            for (int chunk = 0; chunk < 8; ++chunk)
-                *reinterpret_cast<uint4 *>(line + ((chunk ^ (row & 7)) << 4)) =
-                    make_uint4(pk[4 * chunk], pk[4 * chunk + 1], pk[4 * chunk + 2], pk[4 * chunk + 3]);
-        }
-        fence_proxy_async();     // P was written with ordinary stores; the tensor core reads it through the async proxy
-        tc_fence_before();
-        ok = __syncthreads_and(ok);
-        if (!ok) break;
-        // ---- O += P V(j) ------------------------------------------------------------------------------
-        if (tid == 0) {
-            const bool v_ok = mbar_wait(smem_u32(&bar_v[j & 1]), (j >> 1) & 1);
-            ok = ok && v_ok;                 // goes into the next vote
-            tc_fence_after();
-            if (v_ok) {
-#pragma unroll
-                for (int kk = 0; kk < 4; ++kk) {               // 16 keys per MMA
+                for (int kk = 0; kk < 4; ++kk) {       // O += P V(j), 16 keys per MMA
                     const uint64_t a = umma_desc(Ps + kk * 32, 16, 1024);
                     // V is [key][channel]: MN-major for the B operand; 8-key groups 1024 bytes apart, 64-channel boxes one box apart
                     const uint64_t b = umma_desc(Vs + (j & 1) * kPfKvTile + kk * 2048, kPfKvBox, 1024);
                     umma_bf16(tO, a, b, umma_idesc(true, 128), (j > 0 || kk > 0) ? 1u : 0u);
                 }
+                umma_commit(smem_u32(&bar_o));
             }
-            umma_commit(smem_u32(&bar_o));   // committed even if V never came, so that nobody waits for it in vain
+            ok = mbar_wait(smem_u32(&bar_o), (nkv - 1) & 1) && ok;
         }
+    } else {
+        // ---------------- softmax warps: one query row per thread -------------------------------------------
+        float m = -INFINITY;
+        for (int j = 0; j < nkv; ++j) {
+            ok = mbar_wait(smem_u32(&bar_s[j & 1]), (j >> 1) & 1) && ok;           // S(j) is there
+            tc_fence_after();
+            float sv[64];
+            {
+                float lo[32], hi[32];
+                tmem_ld32(t_lane + (j & 1) * kPfKeys, lo);
+                tmem_ld32(t_lane + (j & 1) * kPfKeys + 32, hi);
+#pragma unroll
+                for (int i = 0; i < 32; ++i) { sv[i] = lo[i]; sv[32 + i] = hi[i]; }
+            }
+            tc_fence_before();
+            mbar_arrive(smem_u32(&bar_sfree[j & 1]));                              // this S buffer may be overwritten
+            // key (64 j + col) is visible to row (128 qb + row) iff it does not lie ahead of it; only the two
+            // blocks on the diagonal hide anything; `ahead` = first column of this block hidden from this row
+            if (j >= 2 * qb) {
+                const int ahead = (kPfBlock * qb + row) - kPfKeys * j + 1;
+#pragma unroll
+                for (int i = 0; i < 64; ++i) sv[i] = (i >= ahead) ? -INFINITY : sv[i];
+            }
+            // m is kept in log2 units of the scaled score; the maximum is taken on the raw scores (the scale
+            // is positive) and the scale rides on the fused multiply-add that feeds ex2
+            float rmax = sv[0];
+#pragma unroll
+            for (int i = 1; i < 64; ++i) rmax = fmaxf(rmax, sv[i]);
+            const float m_new = fmaxf(m, rmax * c2);     // finite from the first block on: key 0 is visible to every row
+            const float alpha = ex2_approx(m - m_new);
+            uint32_t pk[32];
+            float lsum = 0.f;
+#pragma unroll
+            for (int i = 0; i < 64; i += 2) {
+                const float p0 = ex2_approx(fmaf(sv[i], c2, -m_new)), p1 = ex2_approx(fmaf(sv[i + 1], c2, -m_new));
+                lsum += p0 + p1;
+                pk[i >> 1] = pack_bf16(p0, p1);
+            }
+            l = l * alpha + lsum;
+            m = m_new;
+            if (j > 0) {                                  // O has taken block j-1 in: the P tile and O are free
+                ok = mbar_wait(smem_u32(&bar_o), (j - 1) & 1) && ok;
+                tc_fence_after();
+                if (!__all_sync(0xffffffffu, alpha == 1.f)) {       // rescale O where the maximum moved
+#pragma unroll 1
+                    for (int c = 0; c < 4; ++c) {
+                        float ov[32];
+                        tmem_ld32(t_lane + (tO - tmem) + c * 32, ov);
+#pragma unroll
+                        for (int i = 0; i < 32; ++i) ov[i] *= alpha;
+                        tmem_st32(t_lane + (tO - tmem) + c * 32, ov);
+                    }
+                    tmem_wait_st();
+                }
+            }
+            // P tile, K-major with 128-byte swizzle: the 64 keys of row r on line r, 16-byte chunk ^ (r & 7)
+            uint8_t *line = Pp + row * 128;
+#pragma unroll
+            for (int chunk = 0; chunk < 8; ++chunk)
+                *reinterpret_cast<uint4 *>(line + ((chunk ^ (row & 7)) << 4)) =
+                    make_uint4(pk[4 * chunk], pk[4 * chunk + 1], pk[4 * chunk + 2], pk[4 * chunk + 3]);
+            fence_proxy_async();     // P was written with ordinary stores; the tensor core reads it through the async proxy
+            tc_fence_before();
+            mbar_arrive(smem_u32(&bar_p));
+        }
+        ok = mbar_wait(smem_u32(&bar_o), (nkv - 1) & 1) && ok;
     }
-    if (ok) ok = mbar_wait(smem_u32(&bar_o), (nkv - 1) & 1);
     tc_fence_after();
     const bool gave_up = !__syncthreads_and(ok);
     if (gave_up) {
         if (tid == 0) flag_error(p.hdr, 6 /* SPD_ERR_TIMEOUT */, -1);
-    } else {
+    } else if (wid < 4) {
         // ---- normalise and store this thread's row (every thread reads its TMEM lane; rows past the
         //      prompt's end are not stored) --------------------------------------------------------------
         const bool live = qb * kPfBlock + row < len;
