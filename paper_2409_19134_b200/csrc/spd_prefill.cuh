@@ -28,6 +28,7 @@ constexpr int kPfQTile = 2 * kPfQBox;               // Q: 128 rows x 128 channel
 constexpr int kPfKvBox = kPfKeys * 128;             // one swizzled box of K or V: 64 rows x 128 bytes
 constexpr int kPfKvTile = 2 * kPfKvBox;             // 64 keys x 128 channels = two boxes
 constexpr int kPfTmemCols = 256;                    // S: 2 x 64, O: 128
+constexpr float kPfSlack = 8.f;                     // log2 units the running reference may lag the maximum by
 
 struct PrefillParams {
     int32_t B, Hq, Hkv;
@@ -104,6 +105,50 @@ __device__ __forceinline__ void tmem_st32(uint32_t taddr, const float (&v)[32]) 
           "r"(__float_as_uint(v[24])), "r"(__float_as_uint(v[25])), "r"(__float_as_uint(v[26])), "r"(__float_as_uint(v[27])),
           "r"(__float_as_uint(v[28])), "r"(__float_as_uint(v[29])), "r"(__float_as_uint(v[30])), "r"(__float_as_uint(v[31]))
         : "memory");
+}
+
+// 64 consecutive fp32 columns of this thread's TMEM lane, one load and one wait.
+__device__ __forceinline__ void tmem_ld64(uint32_t taddr, float (&v)[64]) {
+    uint32_t r[64];
+    asm volatile(
+        "tcgen05.ld.sync.aligned.32x32b.x64.b32 "
+        "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, %16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31, %32, %33, %34, %35, %36, %37, %38, %39, %40, %41, %42, %43, %44, %45, %46, %47, %48, %49, %50, %51, %52, %53, %54, %55, %56, %57, %58, %59, %60, %61, %62, %63}, [%64];"
+        : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]),
+          "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]),
+          "=r"(r[16]), "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]),
+          "=r"(r[24]), "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31]),
+          "=r"(r[32]), "=r"(r[33]), "=r"(r[34]), "=r"(r[35]), "=r"(r[36]), "=r"(r[37]), "=r"(r[38]), "=r"(r[39]),
+          "=r"(r[40]), "=r"(r[41]), "=r"(r[42]), "=r"(r[43]), "=r"(r[44]), "=r"(r[45]), "=r"(r[46]), "=r"(r[47]),
+          "=r"(r[48]), "=r"(r[49]), "=r"(r[50]), "=r"(r[51]), "=r"(r[52]), "=r"(r[53]), "=r"(r[54]), "=r"(r[55]),
+          "=r"(r[56]), "=r"(r[57]), "=r"(r[58]), "=r"(r[59]), "=r"(r[60]), "=r"(r[61]), "=r"(r[62]), "=r"(r[63])
+        : "r"(taddr) : "memory");
+    tmem_wait_ld();
+#pragma unroll
+    for (int i = 0; i < 64; ++i) v[i] = __uint_as_float(r[i]);
+}
+// Two fp32 lanes per instruction on the FMA pipe (halves the issue slots of the softmax arithmetic).
+__device__ __forceinline__ uint64_t pack_f32x2(float lo, float hi) {
+    uint64_t r;
+    asm("mov.b64 %0, {%1, %2};" : "=l"(r) : "f"(lo), "f"(hi));
+    return r;
+}
+__device__ __forceinline__ void unpack_f32x2(uint64_t v, float &lo, float &hi) {
+    asm("mov.b64 {%0, %1}, %2;" : "=f"(lo), "=f"(hi) : "l"(v));
+}
+__device__ __forceinline__ uint64_t fma_f32x2(uint64_t a, uint64_t b, uint64_t c) {
+    uint64_t r;
+    asm("fma.rn.ftz.f32x2 %0, %1, %2, %3;" : "=l"(r) : "l"(a), "l"(b), "l"(c));
+    return r;
+}
+__device__ __forceinline__ uint64_t add_f32x2(uint64_t a, uint64_t b) {
+    uint64_t r;
+    asm("add.rn.ftz.f32x2 %0, %1, %2;" : "=l"(r) : "l"(a), "l"(b));
+    return r;
+}
+__device__ __forceinline__ float fmax3(float a, float b, float c) {
+    float r;
+    asm("max.f32 %0, %1, %2, %3;" : "=f"(r) : "f"(a), "f"(b), "f"(c));
+    return r;
 }
 
 // Q, K x2, V x2, P, then eleven mbarriers and one word; the kernel has no static shared memory, so the
@@ -231,13 +276,7 @@ prefill_kernel(const __grid_constant__ PrefillParams p, const __grid_constant__ 
             ok = mbar_wait(smem_u32(&bar_s[j & 1]), (j >> 1) & 1) && ok;           // S(j) is there
             tc_fence_after();
             float sv[64];
-            {
-                float lo[32], hi[32];
-                tmem_ld32(t_lane + (j & 1) * kPfKeys, lo);
-                tmem_ld32(t_lane + (j & 1) * kPfKeys + 32, hi);
-#pragma unroll
-                for (int i = 0; i < 32; ++i) { sv[i] = lo[i]; sv[32 + i] = hi[i]; }
-            }
+            tmem_ld64(t_lane + (j & 1) * kPfKeys, sv);
             tc_fence_before();
             mbar_arrive(smem_u32(&bar_sfree[j & 1]));                              // this S buffer may be overwritten
             // key (64 j + col) is visible to row (128 qb + row) iff it does not lie ahead of it; only the two
@@ -248,19 +287,37 @@ prefill_kernel(const __grid_constant__ PrefillParams p, const __grid_constant__ 
                 for (int i = 0; i < 64; ++i) sv[i] = (i >= ahead) ? -INFINITY : sv[i];
             }
             // m is kept in log2 units of the scaled score; the maximum is taken on the raw scores (the scale
-            // is positive) and the scale rides on the fused multiply-add that feeds ex2
-            float rmax = sv[0];
+            // is positive) and the scale rides on the fused multiply-add that feeds ex2.  m is a reference
+            // point, not necessarily the exact maximum: it moves only when the block's maximum lies more than
+            // kPfSlack above it, so weights reach 2^kPfSlack at most (harmless in fp32 and bf16, and O and l
+            // carry the same factor, which the final division removes) and O is seldom rescaled.
+            float r4[4];                                 // four chains of three-input maxima
 #pragma unroll
-            for (int i = 1; i < 64; ++i) rmax = fmaxf(rmax, sv[i]);
-            const float m_new = fmaxf(m, rmax * c2);     // finite from the first block on: key 0 is visible to every row
+            for (int c = 0; c < 4; ++c) {
+                r4[c] = fmax3(sv[16 * c], sv[16 * c + 1], sv[16 * c + 2]);
+#pragma unroll
+                for (int i = 3; i < 15; i += 2) r4[c] = fmax3(r4[c], sv[16 * c + i], sv[16 * c + i + 1]);
+                r4[c] = fmaxf(r4[c], sv[16 * c + 15]);
+            }
+            const float rmax = fmaxf(fmax3(r4[0], r4[1], r4[2]), r4[3]) * c2;   // finite from the first block on: key 0 is visible to every row
+            const float m_new = (rmax > m + kPfSlack) ? rmax : m;
             const float alpha = ex2_approx(m - m_new);
             uint32_t pk[32];
             float lsum = 0.f;
+            const uint64_t c2x2 = pack_f32x2(c2, c2), mx2 = pack_f32x2(-m_new, -m_new);
+            uint64_t lsum2 = 0;                           // two partial row sums, (+0, +0)
 #pragma unroll
             for (int i = 0; i < 64; i += 2) {
-                const float p0 = ex2_approx(fmaf(sv[i], c2, -m_new)), p1 = ex2_approx(fmaf(sv[i + 1], c2, -m_new));
-                lsum += p0 + p1;
+                float a0, a1;
+                unpack_f32x2(fma_f32x2(pack_f32x2(sv[i], sv[i + 1]), c2x2, mx2), a0, a1);
+                const float p0 = ex2_approx(a0), p1 = ex2_approx(a1);
+                lsum2 = add_f32x2(lsum2, pack_f32x2(p0, p1));
                 pk[i >> 1] = pack_bf16(p0, p1);
+            }
+            {
+                float s0, s1;
+                unpack_f32x2(lsum2, s0, s1);
+                lsum = s0 + s1;
             }
             l = l * alpha + lsum;
             m = m_new;
