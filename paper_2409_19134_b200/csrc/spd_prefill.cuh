@@ -171,35 +171,39 @@ prefill_kernel(const __grid_constant__ PrefillParams p, const __grid_constant__ 
     const int tid = threadIdx.x, wid = tid >> 5;
     const int h = blockIdx.y, kvh = h / (p.Hq / p.Hkv);
 
-    // which (user, query block) this CTA owns; the heaviest blocks (closest to the prompt's end) come first
-    int u = 0, qb = -1, first = 0, len = 0;
+    // which (user, query block) this CTA owns; the heaviest blocks (closest to the prompt's end) come first.
+    // Every warp works it out for itself, 32 users at a time: query blocks per user, a prefix sum over the
+    // lanes, the first lane whose running total passes this CTA's index.
+    int qb = -1, first = 0, len = 0;
     {
+        const int lane = tid & 31;
         int blk = blockIdx.x;
-        for (u = 0; u < p.B; ++u) {
-            const int64_t a = p.tok_indptr[u], b = p.tok_indptr[u + 1];
-            if (a < 0 || b < a || b > p.T) { u = p.B; break; }          // inconsistent offsets: nothing to do here
-            const int nb = static_cast<int>((b - a + kPfBlock - 1) / kPfBlock);
-            if (blk < nb) { qb = nb - 1 - blk; first = static_cast<int>(a); len = static_cast<int>(b - a); break; }
-            blk -= nb;
+        for (int u0 = 0; u0 < p.B; u0 += 32) {
+            const int u = u0 + lane;
+            int64_t a = 0, b = 0;
+            if (u < p.B) { a = p.tok_indptr[u]; b = p.tok_indptr[u + 1]; }
+            const bool bad = a < 0 || b < a || b > p.T;                   // inconsistent offsets: nothing from here on
+            const int nb = bad ? 0 : static_cast<int>((b - a + kPfBlock - 1) / kPfBlock);
+            int inc = nb;
+#pragma unroll
+            for (int d = 1; d < 32; d <<= 1) {
+                const int t = __shfl_up_sync(0xffffffffu, inc, d);
+                if (lane >= d) inc += t;
+            }
+            const unsigned badmask = __ballot_sync(0xffffffffu, bad), hit = __ballot_sync(0xffffffffu, blk < inc);
+            if (hit) {
+                const int src = __ffs(hit) - 1;
+                const int nb_s = __shfl_sync(0xffffffffu, nb, src), inc_s = __shfl_sync(0xffffffffu, inc, src);
+                const int a_s = __shfl_sync(0xffffffffu, static_cast<int>(a), src), b_s = __shfl_sync(0xffffffffu, static_cast<int>(b), src);
+                if (!(badmask & ((1u << src) - 1u))) { qb = nb_s - 1 - (blk - (inc_s - nb_s)); first = a_s; len = b_s - a_s; }
+                break;
+            }
+            if (badmask) break;
+            blk -= __shfl_sync(0xffffffffu, inc, 31);
         }
     }
     if (qb < 0) return;   // uniform over the CTA: no barrier, no TMEM touched yet
     const int nkv = 2 * (qb + 1);   // 64-key blocks up to and including the diagonal
-
-    if (tid == 0) {
-        for (int b = 0; b < 11; ++b) mbar_init(smem_u32(&bars[b]), (b == 2 || b >= 9) ? 128 : 1);   // P and S-consumed: every softmax thread arrives
-        fence_mbar_init();
-    }
-    if (wid == 0) {       // one warp allocates the accumulator columns for the CTA
-        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&tmem_slot)), "r"(kPfTmemCols) : "memory");
-        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
-    }
-    tc_fence_before();
-    __syncthreads();
-    tc_fence_after();
-    const uint32_t tmem = tmem_slot;
-    const uint32_t t_lane = tmem + (static_cast<uint32_t>(wid * 32) << 16);   // this warp's 32 lanes
-    const uint32_t tO = tmem + 2 * kPfKeys;     // S buffers at columns [0, 64) and [64, 128), O at [128, 256)
 
     // K and V of key block j live in slot j & 1 of their rings; K is free again once S(j) exists, V once
     // O has taken block j in.
@@ -215,6 +219,30 @@ prefill_kernel(const __grid_constant__ PrefillParams p, const __grid_constant__ 
         tma_load_3d(Vs + (j & 1) * kPfKvTile, &mv, 0, kvh, first + j * kPfKeys, bar);
         tma_load_3d(Vs + (j & 1) * kPfKvTile + kPfKvBox, &mv, 64, kvh, first + j * kPfKeys, bar);
     };
+    if (tid == 128) {     // the issuing thread sets the barriers up and starts the first loads before anything else happens
+        for (int b = 0; b < 11; ++b) mbar_init(smem_u32(&bars[b]), (b == 2 || b >= 9) ? 128 : 1);   // P and S-consumed: every softmax thread arrives
+        fence_mbar_init();
+        fence_proxy_async();
+        const uint32_t bq = smem_u32(&bar_q);
+        mbar_expect_tx(bq, kPfQTile);
+        tma_load_3d(Qs, &mq, 0, h, first + qb * kPfBlock, bq);
+        tma_load_3d(Qs + kPfQBox, &mq, 64, h, first + qb * kPfBlock, bq);
+        load_k(0);
+        load_v(0);
+        load_k(1);            // nkv >= 2 always: a query block spans two key blocks on the diagonal
+        load_v(1);
+    }
+    if (wid == 0) {       // one warp allocates the accumulator columns for the CTA
+        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&tmem_slot)), "r"(kPfTmemCols) : "memory");
+        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+    }
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem = tmem_slot;
+    const uint32_t t_lane = tmem + (static_cast<uint32_t>(wid * 32) << 16);   // this warp's 32 lanes
+    const uint32_t tO = tmem + 2 * kPfKeys;     // S buffers at columns [0, 64) and [64, 128), O at [128, 256)
+
     auto mma_s = [&](int j) {                    // S(j) = Q K(j)^T into S buffer j & 1; 16 channels per MMA
         tc_fence_after();
 #pragma unroll
@@ -235,15 +263,7 @@ prefill_kernel(const __grid_constant__ PrefillParams p, const __grid_constant__ 
     if (wid == 4) {
         // ---------------- the issuing thread: TMA loads and MMAs ----------------------------------------
         if (tid == 128) {
-            const uint32_t bq = smem_u32(&bar_q);
-            mbar_expect_tx(bq, kPfQTile);
-            tma_load_3d(Qs, &mq, 0, h, first + qb * kPfBlock, bq);
-            tma_load_3d(Qs + kPfQBox, &mq, 64, h, first + qb * kPfBlock, bq);
-            load_k(0);
-            load_v(0);
-            load_k(1);            // nkv >= 2 always: a query block spans two key blocks on the diagonal
-            load_v(1);
-            ok = mbar_wait(bq, 0) && mbar_wait(smem_u32(&bar_k[0]), 0);
+            ok = mbar_wait(smem_u32(&bar_q), 0) && mbar_wait(smem_u32(&bar_k[0]), 0);
             mma_s(0);
             for (int j = 0; j < nkv; ++j) {
                 if (j + 1 < nkv) {                     // S(j+1): needs K(j+1) and the other S buffer read out (S(j-1))

@@ -38,7 +38,12 @@ def _case(lens, hq, hkv, seed, slack_pages=1):
     return q, k, v, ip, part
 
 
-@pytest.mark.parametrize("lens,hq,hkv", [([128], 1, 1), ([100], 2, 1), ([300, 1, 129, 0, 257], 4, 2), ([1000, 640], 8, 2)])
+# more users than a warp has lanes (the kernel finds its user 32 at a time), some without a prompt
+MANY_USERS = [int(x) for x in np.random.default_rng(70).integers(0, 200, size=70) * (np.arange(70) % 7 != 3)]
+
+
+@pytest.mark.parametrize("lens,hq,hkv", [([128], 1, 1), ([100], 2, 1), ([300, 1, 129, 0, 257], 4, 2), ([1000, 640], 8, 2),
+                                         (MANY_USERS, 2, 1)])
 def test_prefill_matches_oracle_and_hands_over(lens, hq, hkv):
     q, k, v, ip, part = _case(lens, hq, hkv, seed=sum(lens) + hq)
     B, T = len(lens), int(ip[-1])
