@@ -2,19 +2,23 @@
 // hand-over of the prompt's K/V rows to the private paged cache that decode reads.
 //
 // This is the one dense contraction next to the decode path, so it runs on the fifth-generation
-// tensor cores: tcgen05.mma with both operands in 128-byte-swizzled shared memory (filled by TMA),
-// accumulators in tensor memory (TMEM).  One CTA (128 threads) owns 128 query rows of one (user,
-// query head) and walks 64-key blocks up to the diagonal:
+// tensor cores: tcgen05.mma with operands in 128-byte-swizzled shared memory (filled by TMA) or in
+// tensor memory (TMEM), accumulators in TMEM.  One CTA owns 128 query rows of one (user, query head)
+// and walks 64-key blocks up to the diagonal:
 //     S = Q K^T            128 x 64 x head_dim    -> TMEM, two buffers: columns [0, 64) and [64, 128)
-//     online softmax       one query row per thread (TMEM lane = row), P written to shared memory as bf16
-//     O += P V             128 x head_dim x 64    -> TMEM columns [128, 256)
-// Warp-specialised software pipeline: four warps do the softmax (one row per thread), one thread of a
-// fifth warp issues every TMA load and every MMA.  S(j+1) is computed while the softmax warps work on
-// S(j), and O takes block j in under the exponentials of block j+1.  They hand over through mbarriers
-// only (S ready, S consumed, P ready, O updated): no CTA-wide barrier inside the loop.  K and V blocks
-// sit in two-slot rings with their own barriers; every wait is bounded and TMEM is freed on every way out.
-// 112 KB of shared memory and 256 TMEM columns per CTA, so two CTAs share an SM and one's softmax
-// runs under the other's MMAs.  bf16, head_dim 128.
+//     online softmax       one query row per thread (TMEM lane = row); P goes back into the first 32
+//                          columns of S's own buffer as bf16 pairs
+//     O += P V             128 x head_dim x 64    -> TMEM columns [128, 256); P is read from TMEM, V from
+//                          shared memory
+// Shared-memory bandwidth is what bounds this loop (every MMA streams its shared-memory operands again),
+// which is why P never touches shared memory.
+// Warp-specialised software pipeline: four warps do the softmax, one thread of a fifth warp issues every
+// TMA load and every MMA.  S(j+1) is computed while the softmax warps work on S(j), and O takes block j
+// in under the exponentials of block j+1.  They hand over through mbarriers only (S ready, P ready, O
+// updated): no CTA-wide barrier inside the loop.  K and V blocks sit in two-slot rings with their own
+// barriers; every wait is bounded and TMEM is freed on every way out.
+// 96 KB of shared memory and 256 TMEM columns per CTA, so two CTAs share an SM and one's softmax runs
+// under the other's MMAs.  bf16, head_dim 128.
 #pragma once
 
 #include "spd_kernels.cuh"
@@ -151,9 +155,29 @@ __device__ __forceinline__ float fmax3(float a, float b, float c) {
     return r;
 }
 
-// Q, K x2, V x2, P, then eleven mbarriers and one word; the kernel has no static shared memory, so the
+__device__ __forceinline__ void tmem_st32u(uint32_t taddr, const uint32_t (&v)[32]) {
+    asm volatile(
+        "tcgen05.st.sync.aligned.32x32b.x32.b32 [%0], "
+        "{%1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, %16, "
+        "%17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31, %32};"
+        ::"r"(taddr),
+          "r"(v[0]), "r"(v[1]), "r"(v[2]), "r"(v[3]), "r"(v[4]), "r"(v[5]), "r"(v[6]), "r"(v[7]),
+          "r"(v[8]), "r"(v[9]), "r"(v[10]), "r"(v[11]), "r"(v[12]), "r"(v[13]), "r"(v[14]), "r"(v[15]),
+          "r"(v[16]), "r"(v[17]), "r"(v[18]), "r"(v[19]), "r"(v[20]), "r"(v[21]), "r"(v[22]), "r"(v[23]),
+          "r"(v[24]), "r"(v[25]), "r"(v[26]), "r"(v[27]), "r"(v[28]), "r"(v[29]), "r"(v[30]), "r"(v[31])
+        : "memory");
+}
+// The same MMA with the A operand in TMEM (K-major: row = lane, two bf16 per column) and B in shared memory.
+__device__ __forceinline__ void umma_bf16_ta(uint32_t tmem_d, uint32_t tmem_a, uint64_t bdesc, uint32_t idesc, uint32_t accumulate) {
+    asm volatile(
+        "{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"
+        "tcgen05.mma.cta_group::1.kind::f16 [%0], [%1], %2, %3, p;\n\t}"
+        ::"r"(tmem_d), "r"(tmem_a), "l"(bdesc), "r"(idesc), "r"(accumulate) : "memory");
+}
+
+// Q, K x2, V x2, then nine mbarriers and one word; the kernel has no static shared memory, so the
 // 1024-byte alignment of the tiles costs nothing and two CTAs fit one SM.
-constexpr size_t prefill_smem_bytes() { return kPfQTile + 4 * static_cast<size_t>(kPfKvTile) + kPfQBox + 128; }   // 11 x 8 + 4 <= 128
+constexpr size_t prefill_smem_bytes() { return kPfQTile + 4 * static_cast<size_t>(kPfKvTile) + 128; }   // 9 x 8 + 4 <= 128
 
 constexpr int kPfThreads = 160;   // 4 softmax warps + 1 warp that issues loads and MMAs
 
@@ -161,13 +185,11 @@ __global__ void __launch_bounds__(kPfThreads, 2)
 prefill_kernel(const __grid_constant__ PrefillParams p, const __grid_constant__ CUtensorMap mq,
                const __grid_constant__ CUtensorMap mk, const __grid_constant__ CUtensorMap mv) {
     extern __shared__ __align__(1024) uint8_t base[];
-    const uint32_t Qs = smem_u32(base), Ks = Qs + kPfQTile, Vs = Ks + 2 * kPfKvTile, Ps = Vs + 2 * kPfKvTile;
-    uint8_t *Pp = base + kPfQTile + 4 * kPfKvTile;
-    uint64_t *bars = reinterpret_cast<uint64_t *>(Pp + kPfQBox);
+    const uint32_t Qs = smem_u32(base), Ks = Qs + kPfQTile, Vs = Ks + 2 * kPfKvTile;
+    uint64_t *bars = reinterpret_cast<uint64_t *>(base + kPfQTile + 4 * kPfKvTile);
     uint64_t &bar_q = bars[0], &bar_o = bars[1], &bar_p = bars[2];        // Q loaded; O updated; P written
     uint64_t *bar_k = bars + 3, *bar_v = bars + 5, *bar_s = bars + 7;     // K / V slot loaded; S buffer ready
-    uint64_t *bar_sfree = bars + 9;                                         // S buffer read by all softmax threads
-    uint32_t &tmem_slot = *reinterpret_cast<uint32_t *>(bars + 11);
+    uint32_t &tmem_slot = *reinterpret_cast<uint32_t *>(bars + 9);
     const int tid = threadIdx.x, wid = tid >> 5;
     const int h = blockIdx.y, kvh = h / (p.Hq / p.Hkv);
 
@@ -220,7 +242,7 @@ prefill_kernel(const __grid_constant__ PrefillParams p, const __grid_constant__ 
         tma_load_3d(Vs + (j & 1) * kPfKvTile + kPfKvBox, &mv, 64, kvh, first + j * kPfKeys, bar);
     };
     if (tid == 128) {     // the issuing thread sets the barriers up and starts the first loads before anything else happens
-        for (int b = 0; b < 11; ++b) mbar_init(smem_u32(&bars[b]), (b == 2 || b >= 9) ? 128 : 1);   // P and S-consumed: every softmax thread arrives
+        for (int b = 0; b < 9; ++b) mbar_init(smem_u32(&bars[b]), b == 2 ? 128 : 1);   // P written: every softmax thread arrives
         fence_mbar_init();
         fence_proxy_async();
         const uint32_t bq = smem_u32(&bar_q);
@@ -266,24 +288,27 @@ prefill_kernel(const __grid_constant__ PrefillParams p, const __grid_constant__ 
             ok = mbar_wait(smem_u32(&bar_q), 0) && mbar_wait(smem_u32(&bar_k[0]), 0);
             mma_s(0);
             for (int j = 0; j < nkv; ++j) {
-                if (j + 1 < nkv) {                     // S(j+1): needs K(j+1) and the other S buffer read out (S(j-1))
+                // S(j+1) goes where S(j-1) and then P(j-1) were: the softmax threads are done with both (they
+                // signalled P(j-1)), and O += P(j-1) V(j-1) was issued before, so the tensor core runs it first
+                if (j + 1 < nkv) {
                     ok = mbar_wait(smem_u32(&bar_k[(j + 1) & 1]), ((j + 1) >> 1) & 1) && ok;
-                    if (j > 0) ok = mbar_wait(smem_u32(&bar_sfree[(j + 1) & 1]), ((j - 1) >> 1) & 1) && ok;
                     mma_s(j + 1);
                 }
-                // P(j) is written and O rescaled: S(j) was read, so K slot j & 1 is free; and the softmax
-                // threads saw O take block j-1 in, so V slot (j-1) & 1 is free
+                // P(j) is written and O rescaled: S(j) was read, so K slot j & 1 is free; V slot (j+1) & 1 is
+                // free once O has taken block j-1 in (long done by now)
                 ok = mbar_wait(smem_u32(&bar_p), j & 1) && ok;
                 if (j + 2 < nkv) load_k(j + 2);
-                if (j > 0 && j + 1 < nkv) load_v(j + 1);
+                if (j > 0 && j + 1 < nkv) {
+                    ok = mbar_wait(smem_u32(&bar_o), (j - 1) & 1) && ok;
+                    load_v(j + 1);
+                }
                 ok = mbar_wait(smem_u32(&bar_v[j & 1]), (j >> 1) & 1) && ok;
                 tc_fence_after();
 #pragma unroll
-                for (int kk = 0; kk < 4; ++kk) {       // O += P V(j), 16 keys per MMA
-                    const uint64_t a = umma_desc(Ps + kk * 32, 16, 1024);
+                for (int kk = 0; kk < 4; ++kk) {       // O += P V(j), 16 keys per MMA; P comes from TMEM (8 columns per 16 keys)
                     // V is [key][channel]: MN-major for the B operand; 8-key groups 1024 bytes apart, 64-channel boxes one box apart
                     const uint64_t b = umma_desc(Vs + (j & 1) * kPfKvTile + kk * 2048, kPfKvBox, 1024);
-                    umma_bf16(tO, a, b, umma_idesc(true, 128), (j > 0 || kk > 0) ? 1u : 0u);
+                    umma_bf16_ta(tO, tmem + (j & 1) * kPfKeys + kk * 8, b, umma_idesc(true, 128), (j > 0 || kk > 0) ? 1u : 0u);
                 }
                 umma_commit(smem_u32(&bar_o));
             }
@@ -297,8 +322,6 @@ prefill_kernel(const __grid_constant__ PrefillParams p, const __grid_constant__ 
             tc_fence_after();
             float sv[64];
             tmem_ld64(t_lane + (j & 1) * kPfKeys, sv);
-            tc_fence_before();
-            mbar_arrive(smem_u32(&bar_sfree[j & 1]));                              // this S buffer may be overwritten
             // key (64 j + col) is visible to row (128 qb + row) iff it does not lie ahead of it; only the two
             // blocks on the diagonal hide anything; `ahead` = first column of this block hidden from this row
             if (j >= 2 * qb) {
@@ -341,28 +364,23 @@ prefill_kernel(const __grid_constant__ PrefillParams p, const __grid_constant__ 
             }
             l = l * alpha + lsum;
             m = m_new;
-            if (j > 0) {                                  // O has taken block j-1 in: the P tile and O are free
+            // rescale O where the reference moved (rare): only then must O += P(j-1) V(j-1) have finished
+            if (j > 0 && !__all_sync(0xffffffffu, alpha == 1.f)) {
                 ok = mbar_wait(smem_u32(&bar_o), (j - 1) & 1) && ok;
                 tc_fence_after();
-                if (!__all_sync(0xffffffffu, alpha == 1.f)) {       // rescale O where the maximum moved
 #pragma unroll 1
-                    for (int c = 0; c < 4; ++c) {
-                        float ov[32];
-                        tmem_ld32(t_lane + (tO - tmem) + c * 32, ov);
+                for (int c = 0; c < 4; ++c) {
+                    float ov[32];
+                    tmem_ld32(t_lane + (tO - tmem) + c * 32, ov);
 #pragma unroll
-                        for (int i = 0; i < 32; ++i) ov[i] *= alpha;
-                        tmem_st32(t_lane + (tO - tmem) + c * 32, ov);
-                    }
-                    tmem_wait_st();
+                    for (int i = 0; i < 32; ++i) ov[i] *= alpha;
+                    tmem_st32(t_lane + (tO - tmem) + c * 32, ov);
                 }
             }
-            // P tile, K-major with 128-byte swizzle: the 64 keys of row r on line r, 16-byte chunk ^ (r & 7)
-            uint8_t *line = Pp + row * 128;
-#pragma unroll
-            for (int chunk = 0; chunk < 8; ++chunk)
-                *reinterpret_cast<uint4 *>(line + ((chunk ^ (row & 7)) << 4)) =
-                    make_uint4(pk[4 * chunk], pk[4 * chunk + 1], pk[4 * chunk + 2], pk[4 * chunk + 3]);
-            fence_proxy_async();     // P was written with ordinary stores; the tensor core reads it through the async proxy
+            // P(j) as bf16 pairs over the first 32 columns of S(j)'s buffer: the A operand of O += P V, read
+            // by the tensor core straight from TMEM (row = lane, two keys per column)
+            tmem_st32u(t_lane + (j & 1) * kPfKeys, pk);
+            tmem_wait_st();
             tc_fence_before();
             mbar_arrive(smem_u32(&bar_p));
         }
@@ -373,28 +391,49 @@ prefill_kernel(const __grid_constant__ PrefillParams p, const __grid_constant__ 
     if (gave_up) {
         if (tid == 0) flag_error(p.hdr, 6 /* SPD_ERR_TIMEOUT */, -1);
     } else if (wid < 4) {
-        // ---- normalise and store this thread's row (every thread reads its TMEM lane; rows past the
-        //      prompt's end are not stored) --------------------------------------------------------------
-        const bool live = qb * kPfBlock + row < len;
+        // ---- normalise this thread's row into shared memory (the Q and K tiles are free by now), then each
+        //      warp stores its own 32 rows with whole rows per instruction; 16-byte chunks are XOR-swizzled
+        //      by the row so that neither side meets bank conflicts; rows past the prompt's end are not stored
         const float inv = 1.f / l;
-        const int64_t tok = static_cast<int64_t>(first) + qb * kPfBlock + row;
+        const int lane = tid & 31;
+        uint8_t *stage = base;
 #pragma unroll 1
         for (int c = 0; c < 4; ++c) {
             float ov[32];
-            __syncwarp();        // the TMEM load is warp-wide: rows that skipped the stores rejoin here
             tmem_ld32(t_lane + (tO - tmem) + c * 32, ov);
-            if (!live) continue;
             if (p.out_bf16) {
-                uint4 *dst = reinterpret_cast<uint4 *>(reinterpret_cast<__nv_bfloat16 *>(p.out) + (tok * p.Hq + h) * 128 + c * 32);
 #pragma unroll
                 for (int q4 = 0; q4 < 4; ++q4)
-                    dst[q4] = make_uint4(pack_bf16(ov[8 * q4] * inv, ov[8 * q4 + 1] * inv), pack_bf16(ov[8 * q4 + 2] * inv, ov[8 * q4 + 3] * inv),
-                                         pack_bf16(ov[8 * q4 + 4] * inv, ov[8 * q4 + 5] * inv), pack_bf16(ov[8 * q4 + 6] * inv, ov[8 * q4 + 7] * inv));
+                    *reinterpret_cast<uint4 *>(stage + row * 256 + (((c * 4 + q4) ^ (row & 7)) << 4)) =
+                        make_uint4(pack_bf16(ov[8 * q4] * inv, ov[8 * q4 + 1] * inv), pack_bf16(ov[8 * q4 + 2] * inv, ov[8 * q4 + 3] * inv),
+                                   pack_bf16(ov[8 * q4 + 4] * inv, ov[8 * q4 + 5] * inv), pack_bf16(ov[8 * q4 + 6] * inv, ov[8 * q4 + 7] * inv));
             } else {
-                float4 *dst = reinterpret_cast<float4 *>(reinterpret_cast<float *>(p.out) + (tok * p.Hq + h) * 128 + c * 32);
 #pragma unroll
                 for (int q4 = 0; q4 < 8; ++q4)
-                    dst[q4] = make_float4(ov[4 * q4] * inv, ov[4 * q4 + 1] * inv, ov[4 * q4 + 2] * inv, ov[4 * q4 + 3] * inv);
+                    *reinterpret_cast<float4 *>(stage + row * 512 + (((c * 8 + q4) ^ (row & 7)) << 4)) =
+                        make_float4(ov[4 * q4] * inv, ov[4 * q4 + 1] * inv, ov[4 * q4 + 2] * inv, ov[4 * q4 + 3] * inv);
+            }
+        }
+        __syncwarp();
+        const int rows_live = len - (qb * kPfBlock + wid * 32);            // rows of this warp that belong to the prompt
+        const int64_t tok0 = static_cast<int64_t>(first) + qb * kPfBlock + wid * 32;
+        if (p.out_bf16) {
+            uint8_t *dst = reinterpret_cast<uint8_t *>(p.out);
+#pragma unroll 4
+            for (int it = 0; it < 16; ++it) {
+                const int r = 2 * it + (lane >> 4), ch = lane & 15, rr = wid * 32 + r;
+                if (r < rows_live)
+                    *reinterpret_cast<uint4 *>(dst + ((tok0 + r) * p.Hq + h) * 256 + ch * 16) =
+                        *reinterpret_cast<const uint4 *>(stage + rr * 256 + ((ch ^ (rr & 7)) << 4));
+            }
+        } else {
+            uint8_t *dst = reinterpret_cast<uint8_t *>(p.out);
+#pragma unroll 4
+            for (int r = 0; r < 32; ++r) {
+                const int rr = wid * 32 + r;
+                if (r < rows_live)
+                    *reinterpret_cast<uint4 *>(dst + ((tok0 + r) * p.Hq + h) * 512 + lane * 16) =
+                        *reinterpret_cast<const uint4 *>(stage + rr * 512 + ((lane ^ (rr & 7)) << 4));
             }
         }
     }
