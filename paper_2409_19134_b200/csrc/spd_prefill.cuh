@@ -175,9 +175,9 @@ __device__ __forceinline__ void umma_bf16_ta(uint32_t tmem_d, uint32_t tmem_a, u
         ::"r"(tmem_d), "r"(tmem_a), "l"(bdesc), "r"(idesc), "r"(accumulate) : "memory");
 }
 
-// Q, K x2, V x2, then nine mbarriers and one word; the kernel has no static shared memory, so the
+// Q, K x2, V x2, then ten mbarriers and one word; the kernel has no static shared memory, so the
 // 1024-byte alignment of the tiles costs nothing and two CTAs fit one SM.
-constexpr size_t prefill_smem_bytes() { return kPfQTile + 4 * static_cast<size_t>(kPfKvTile) + 128; }   // 9 x 8 + 4 <= 128
+constexpr size_t prefill_smem_bytes() { return kPfQTile + 4 * static_cast<size_t>(kPfKvTile) + 128; }   // 10 x 8 + 4 <= 128
 
 constexpr int kPfThreads = 160;   // 4 softmax warps + 1 warp that issues loads and MMAs
 
@@ -187,9 +187,10 @@ prefill_kernel(const __grid_constant__ PrefillParams p, const __grid_constant__ 
     extern __shared__ __align__(1024) uint8_t base[];
     const uint32_t Qs = smem_u32(base), Ks = Qs + kPfQTile, Vs = Ks + 2 * kPfKvTile;
     uint64_t *bars = reinterpret_cast<uint64_t *>(base + kPfQTile + 4 * kPfKvTile);
-    uint64_t &bar_q = bars[0], &bar_o = bars[1], &bar_p = bars[2];        // Q loaded; O updated; P written
-    uint64_t *bar_k = bars + 3, *bar_v = bars + 5, *bar_s = bars + 7;     // K / V slot loaded; S buffer ready
-    uint32_t &tmem_slot = *reinterpret_cast<uint32_t *>(bars + 9);
+    uint64_t &bar_q = bars[0], &bar_o = bars[1];                          // Q loaded; O updated
+    uint64_t *bar_p = bars + 2;                                            // P written into S buffer 0 / 1
+    uint64_t *bar_k = bars + 4, *bar_v = bars + 6, *bar_s = bars + 8;     // K / V slot loaded; S buffer ready
+    uint32_t &tmem_slot = *reinterpret_cast<uint32_t *>(bars + 10);
     const int tid = threadIdx.x, wid = tid >> 5;
     const int h = blockIdx.y, kvh = h / (p.Hq / p.Hkv);
 
@@ -242,7 +243,7 @@ prefill_kernel(const __grid_constant__ PrefillParams p, const __grid_constant__ 
         tma_load_3d(Vs + (j & 1) * kPfKvTile + kPfKvBox, &mv, 64, kvh, first + j * kPfKeys, bar);
     };
     if (tid == 128) {     // the issuing thread sets the barriers up and starts the first loads before anything else happens
-        for (int b = 0; b < 9; ++b) mbar_init(smem_u32(&bars[b]), b == 2 ? 128 : 1);   // P written: every softmax thread arrives
+        for (int b = 0; b < 10; ++b) mbar_init(smem_u32(&bars[b]), (b == 2 || b == 3) ? 128 : 1);   // P written: every softmax thread arrives
         fence_mbar_init();
         fence_proxy_async();
         const uint32_t bq = smem_u32(&bar_q);
@@ -295,8 +296,10 @@ prefill_kernel(const __grid_constant__ PrefillParams p, const __grid_constant__ 
                     mma_s(j + 1);
                 }
                 // P(j) is written and O rescaled: S(j) was read, so K slot j & 1 is free; V slot (j+1) & 1 is
-                // free once O has taken block j-1 in (long done by now)
-                ok = mbar_wait(smem_u32(&bar_p), j & 1) && ok;
+                // free once O has taken block j-1 in (long done by now).  The softmax threads may already be
+                // a block ahead (S(j+1) exists), hence one P barrier per S buffer: S(j+2) is not issued before
+                // this wait returns, so they can never be two phases ahead on either.
+                ok = mbar_wait(smem_u32(&bar_p[j & 1]), (j >> 1) & 1) && ok;
                 if (j + 2 < nkv) load_k(j + 2);
                 if (j > 0 && j + 1 < nkv) {
                     ok = mbar_wait(smem_u32(&bar_o), (j - 1) & 1) && ok;
@@ -382,7 +385,7 @@ prefill_kernel(const __grid_constant__ PrefillParams p, const __grid_constant__ 
             tmem_st32u(t_lane + (j & 1) * kPfKeys, pk);
             tmem_wait_st();
             tc_fence_before();
-            mbar_arrive(smem_u32(&bar_p));
+            mbar_arrive(smem_u32(&bar_p[j & 1]));
         }
         ok = mbar_wait(smem_u32(&bar_o), (nkv - 1) & 1) && ok;
     }
