@@ -42,14 +42,22 @@ def _case(lens, hq, hkv, seed, slack_pages=1):
 MANY_USERS = [int(x) for x in np.random.default_rng(70).integers(0, 200, size=70) * (np.arange(70) % 7 != 3)]
 
 
+@pytest.fixture(params=[128, 256], ids=["rows128", "rows256"])
+def tile(request):
+    """Both prefill kernels (128 and 256 query rows per CTA) must pass every case; the default picks by length."""
+    spd.spd_set_prefill_tile(request.param)
+    yield request.param
+    spd.spd_set_prefill_tile(0)
+
+
 @pytest.mark.parametrize("lens,hq,hkv", [([128], 1, 1), ([100], 2, 1), ([300, 1, 129, 0, 257], 4, 2), ([1000, 640], 8, 2),
-                                         (MANY_USERS, 2, 1)])
-def test_prefill_matches_oracle_and_hands_over(lens, hq, hkv):
+                                         (MANY_USERS, 2, 1), ([2500, 256, 385], 4, 1)])
+def test_prefill_matches_oracle_and_hands_over(lens, hq, hkv, tile):
     q, k, v, ip, part = _case(lens, hq, hkv, seed=sum(lens) + hq)
     B, T = len(lens), int(ip[-1])
     scale = 1.0 / np.sqrt(128.0)
     rows = np.arange(T) if T <= 700 else np.unique(np.concatenate([np.arange(0, T, 37), ip[1:] - 1, ip[:-1],
-                                                                   np.array([127, 128, 255, 256, 999, 1000, 1127, 1128])]))
+                                                                   np.array([127, 128, 255, 256, 999, 1000, 1127, 1128, 2303, 2304, 2431, 2432, 2499])]))
     rows = rows[(rows >= 0) & (rows < T)]
     ref = orc.prefill(orc.q_from_torch(q), orc.q_from_torch(k), orc.q_from_torch(v), ip, scale, rows)
     shape = spd.make_shape(B, hq, hkv, 128, torch.bfloat16, scale)
@@ -79,7 +87,7 @@ def test_prefill_matches_oracle_and_hands_over(lens, hq, hkv):
     assert np.max(np.abs(yd.cpu().numpy() - refd)) <= 2e-3
 
 
-def test_prefill_bf16_output_and_full_cache_is_flagged():
+def test_prefill_bf16_output_and_full_cache_is_flagged(tile):
     q, k, v, ip, part = _case([200, 90], 2, 2, seed=9, slack_pages=0)
     part.page_indptr = torch.tensor([0, 13, 18], dtype=torch.int32)        # user 1 needs 6 pages, gets 5
     scale = 0.09
