@@ -13,7 +13,7 @@
 // Shared-memory bandwidth is what bounds this loop (every MMA streams its shared-memory operands again),
 // which is why P never touches shared memory.
 // Warp-specialised software pipeline: four warps do the softmax, one thread of a fifth warp issues every
-// TMA load and every MMA.  S(j+1) is computed while the softmax warps work on S(j), and O takes block j
+// TMA load and the S products, one thread of a sixth the P V products.  S(j+1) is computed while the softmax warps work on S(j), and O takes block j
 // in under the exponentials of block j+1.  They hand over through mbarriers only (S ready, P ready, O
 // updated): no CTA-wide barrier inside the loop.  K and V blocks sit in two-slot rings with their own
 // barriers; every wait is bounded and TMEM is freed on every way out.
@@ -175,11 +175,11 @@ __device__ __forceinline__ void umma_bf16_ta(uint32_t tmem_d, uint32_t tmem_a, u
         ::"r"(tmem_d), "r"(tmem_a), "l"(bdesc), "r"(idesc), "r"(accumulate) : "memory");
 }
 
-// Q, K x2, V x2, then ten mbarriers and one word; the kernel has no static shared memory, so the
+// Q, K x2, V x2, then eleven mbarriers and one word; the kernel has no static shared memory, so the
 // 1024-byte alignment of the tiles costs nothing and two CTAs fit one SM.
-constexpr size_t prefill_smem_bytes() { return kPfQTile + 4 * static_cast<size_t>(kPfKvTile) + 128; }   // 10 x 8 + 4 <= 128
+constexpr size_t prefill_smem_bytes() { return kPfQTile + 4 * static_cast<size_t>(kPfKvTile) + 128; }   // 11 x 8 + 4 <= 128
 
-constexpr int kPfThreads = 160;   // 4 softmax warps + 1 warp that issues loads and MMAs
+constexpr int kPfThreads = 192;   // 4 softmax warps + 2 warps with one issuing thread each
 
 __global__ void __launch_bounds__(kPfThreads, 2)
 prefill_kernel(const __grid_constant__ PrefillParams p, const __grid_constant__ CUtensorMap mq,
@@ -187,10 +187,11 @@ prefill_kernel(const __grid_constant__ PrefillParams p, const __grid_constant__ 
     extern __shared__ __align__(1024) uint8_t base[];
     const uint32_t Qs = smem_u32(base), Ks = Qs + kPfQTile, Vs = Ks + 2 * kPfKvTile;
     uint64_t *bars = reinterpret_cast<uint64_t *>(base + kPfQTile + 4 * kPfKvTile);
-    uint64_t &bar_q = bars[0], &bar_o = bars[1];                          // Q loaded; O updated
-    uint64_t *bar_p = bars + 2;                                            // P written into S buffer 0 / 1
-    uint64_t *bar_k = bars + 4, *bar_v = bars + 6, *bar_s = bars + 8;     // K / V slot loaded; S buffer ready
-    uint32_t &tmem_slot = *reinterpret_cast<uint32_t *>(bars + 10);
+    uint64_t &bar_q = bars[0];                                             // Q loaded
+    uint64_t *bar_o = bars + 1;                                            // O has taken in the block whose P was in S buffer 0 / 1
+    uint64_t *bar_p = bars + 3;                                            // P written into S buffer 0 / 1
+    uint64_t *bar_k = bars + 5, *bar_v = bars + 7, *bar_s = bars + 9;     // K / V slot loaded; S buffer ready
+    uint32_t &tmem_slot = *reinterpret_cast<uint32_t *>(bars + 11);
     const int tid = threadIdx.x, wid = tid >> 5;
     const int h = blockIdx.y, kvh = h / (p.Hq / p.Hkv);
 
@@ -243,7 +244,7 @@ prefill_kernel(const __grid_constant__ PrefillParams p, const __grid_constant__ 
         tma_load_3d(Vs + (j & 1) * kPfKvTile + kPfKvBox, &mv, 64, kvh, first + j * kPfKeys, bar);
     };
     if (tid == 128) {     // the issuing thread sets the barriers up and starts the first loads before anything else happens
-        for (int b = 0; b < 10; ++b) mbar_init(smem_u32(&bars[b]), (b == 2 || b == 3) ? 128 : 1);   // P written: every softmax thread arrives
+        for (int b = 0; b < 11; ++b) mbar_init(smem_u32(&bars[b]), (b == 3 || b == 4) ? 128 : 1);   // P written: every softmax thread arrives
         fence_mbar_init();
         fence_proxy_async();
         const uint32_t bq = smem_u32(&bar_q);
@@ -283,39 +284,48 @@ prefill_kernel(const __grid_constant__ PrefillParams p, const __grid_constant__ 
     // towards the same end): nothing in the loop waits for all threads, so nobody can be left behind.
     bool ok = true;
 
+    // One thread cannot issue MMAs faster than about one per hundred cycles, whatever their size, while the
+    // tensor core takes them from two threads at nearly twice that rate: so two threads issue, one the
+    // S = Q K^T products (and the TMA loads), the other the O += P V products.  MMAs of different threads are
+    // not ordered by issue, so where one's operands or accumulator depend on the other's work it waits for the
+    // commit barrier, never for the issue.  All barriers that a thread may find two phases ahead exist twice
+    // (per S buffer), so that parity never aliases.
     if (wid == 4) {
-        // ---------------- the issuing thread: TMA loads and MMAs ----------------------------------------
+        // ---------------- first issuing thread: TMA loads and S = Q K^T -------------------------------------
         if (tid == 128) {
             ok = mbar_wait(smem_u32(&bar_q), 0) && mbar_wait(smem_u32(&bar_k[0]), 0);
             mma_s(0);
             for (int j = 0; j < nkv; ++j) {
-                // S(j+1) goes where S(j-1) and then P(j-1) were: the softmax threads are done with both (they
-                // signalled P(j-1)), and O += P(j-1) V(j-1) was issued before, so the tensor core runs it first
                 if (j + 1 < nkv) {
                     ok = mbar_wait(smem_u32(&bar_k[(j + 1) & 1]), ((j + 1) >> 1) & 1) && ok;
+                    // S(j+1) goes where S(j-1) and then P(j-1) were, and V(j+1) where V(j-1) was: both are free
+                    // once O has taken block j-1 in
+                    if (j > 0) ok = mbar_wait(smem_u32(&bar_o[(j - 1) & 1]), ((j - 1) >> 1) & 1) && ok;
                     mma_s(j + 1);
+                    if (j > 0) load_v(j + 1);
                 }
-                // P(j) is written and O rescaled: S(j) was read, so K slot j & 1 is free; V slot (j+1) & 1 is
-                // free once O has taken block j-1 in (long done by now).  The softmax threads may already be
-                // a block ahead (S(j+1) exists), hence one P barrier per S buffer: S(j+2) is not issued before
-                // this wait returns, so they can never be two phases ahead on either.
-                ok = mbar_wait(smem_u32(&bar_p[j & 1]), (j >> 1) & 1) && ok;
-                if (j + 2 < nkv) load_k(j + 2);
-                if (j > 0 && j + 1 < nkv) {
-                    ok = mbar_wait(smem_u32(&bar_o), (j - 1) & 1) && ok;
-                    load_v(j + 1);
+                if (j + 2 < nkv) {                     // K slot j & 1 is free once S(j) exists (issued a round ago)
+                    ok = mbar_wait(smem_u32(&bar_s[j & 1]), (j >> 1) & 1) && ok;
+                    load_k(j + 2);
                 }
+            }
+        }
+    } else if (wid == 5) {
+        // ---------------- second issuing thread: O += P V -----------------------------------------------------
+        if (tid == 160) {
+            for (int j = 0; j < nkv; ++j) {
+                ok = mbar_wait(smem_u32(&bar_p[j & 1]), (j >> 1) & 1) && ok;       // P(j) is written and O rescaled
                 ok = mbar_wait(smem_u32(&bar_v[j & 1]), (j >> 1) & 1) && ok;
                 tc_fence_after();
 #pragma unroll
-                for (int kk = 0; kk < 4; ++kk) {       // O += P V(j), 16 keys per MMA; P comes from TMEM (8 columns per 16 keys)
+                for (int kk = 0; kk < 4; ++kk) {       // 16 keys per MMA; P comes from TMEM (8 columns per 16 keys)
                     // V is [key][channel]: MN-major for the B operand; 8-key groups 1024 bytes apart, 64-channel boxes one box apart
                     const uint64_t b = umma_desc(Vs + (j & 1) * kPfKvTile + kk * 2048, kPfKvBox, 1024);
                     umma_bf16_ta(tO, tmem + (j & 1) * kPfKeys + kk * 8, b, umma_idesc(true, 128), (j > 0 || kk > 0) ? 1u : 0u);
                 }
-                umma_commit(smem_u32(&bar_o));
+                umma_commit(smem_u32(&bar_o[j & 1]));
             }
-            ok = mbar_wait(smem_u32(&bar_o), (nkv - 1) & 1) && ok;
+            ok = mbar_wait(smem_u32(&bar_o[(nkv - 1) & 1]), ((nkv - 1) >> 1) & 1) && ok;
         }
     } else {
         // ---------------- softmax warps: one query row per thread -------------------------------------------
@@ -369,7 +379,7 @@ prefill_kernel(const __grid_constant__ PrefillParams p, const __grid_constant__ 
             m = m_new;
             // rescale O where the reference moved (rare): only then must O += P(j-1) V(j-1) have finished
             if (j > 0 && !__all_sync(0xffffffffu, alpha == 1.f)) {
-                ok = mbar_wait(smem_u32(&bar_o), (j - 1) & 1) && ok;
+                ok = mbar_wait(smem_u32(&bar_o[(j - 1) & 1]), ((j - 1) >> 1) & 1) && ok;
                 tc_fence_after();
 #pragma unroll 1
                 for (int c = 0; c < 4; ++c) {
@@ -387,7 +397,7 @@ prefill_kernel(const __grid_constant__ PrefillParams p, const __grid_constant__ 
             tc_fence_before();
             mbar_arrive(smem_u32(&bar_p[j & 1]));
         }
-        ok = mbar_wait(smem_u32(&bar_o), (nkv - 1) & 1) && ok;
+        ok = mbar_wait(smem_u32(&bar_o[(nkv - 1) & 1]), ((nkv - 1) >> 1) & 1) && ok;
     }
     tc_fence_after();
     const bool gave_up = !__syncthreads_and(ok);
