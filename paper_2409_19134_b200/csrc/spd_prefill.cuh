@@ -244,7 +244,7 @@ prefill_kernel(const __grid_constant__ PrefillParams p, const __grid_constant__ 
         tma_load_3d(Vs + (j & 1) * kPfKvTile + kPfKvBox, &mv, 64, kvh, first + j * kPfKeys, bar);
     };
     if (tid == 128) {     // the issuing thread sets the barriers up and starts the first loads before anything else happens
-        for (int b = 0; b < 11; ++b) mbar_init(smem_u32(&bars[b]), (b == 3 || b == 4) ? 128 : 1);   // P written: every softmax thread arrives
+        for (int b = 0; b < 11; ++b) mbar_init(smem_u32(&bars[b]), (b == 3 || b == 4) ? 4 : 1);   // P written: every softmax thread arrives
         fence_mbar_init();
         fence_proxy_async();
         const uint32_t bq = smem_u32(&bar_q);
@@ -395,7 +395,8 @@ prefill_kernel(const __grid_constant__ PrefillParams p, const __grid_constant__ 
             tmem_st32u(t_lane + (j & 1) * kPfKeys, pk);
             tmem_wait_st();
             tc_fence_before();
-            mbar_arrive(smem_u32(&bar_p[j & 1]));
+            __syncwarp();                                 // one arrival per warp: arrivals on one barrier word queue up
+            if ((tid & 31) == 0) mbar_arrive(smem_u32(&bar_p[j & 1]));
         }
         ok = mbar_wait(smem_u32(&bar_o[(nkv - 1) & 1]), ((nkv - 1) >> 1) & 1) && ok;
     }
