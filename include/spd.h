@@ -280,11 +280,12 @@ spd_status spd_decode_step_static(const spd_shape *shape, const void *q, const s
 spd_status spd_set_bf16_math(int32_t path);
 
 /*
- * Tuning and test aid (no counterpart in the paper): keys per block of spd_prefill_attn from now on,
- * process-wide.  0 (default) = chosen per call from the mean prompt length (128 keys from 1024 tokens
- * on, else 64); 64 or 128 force one kernel.  Both compute the same thing within tolerance.
+ * Tuning and test aid (no counterpart in the paper): query rows per CTA of spd_prefill_attn from now on,
+ * process-wide.  0 (default) = chosen per call from the mean prompt length (256 rows, two tiles sharing
+ * their K/V loads, from 256 tokens on, else 128); 128 or 256 force one kernel.  Both compute the same
+ * thing within tolerance.
  */
-spd_status spd_set_prefill_keys(int32_t keys);
+spd_status spd_set_prefill_rows(int32_t rows);
 
 /* Static text for a status code. */
 const char *spd_status_string(spd_status status);

@@ -23,7 +23,7 @@ EXPORTS = ["spd_workspace_size", "spd_partial_attn", "spd_service_attn_merge", "
            "spd_kernel_launch_count", "spd_status_string", "spd_profile_begin", "spd_profile_end",
            "spd_decode_step_static", "spd_append_kv",
            "spd_partial_attn_watch", "spd_decode_step_watch", "spd_set_bf16_math", "spd_merge_partials", "spd_prefill_attn",
-           "spd_set_prefill_keys"]
+           "spd_set_prefill_rows"]
 
 
 class SpdError(RuntimeError):
@@ -88,7 +88,7 @@ def lib() -> C.CDLL:
         L.spd_decode_step_watch.argtypes = [C.POINTER(Shape), vp, C.POINTER(PagedKV), C.POINTER(PagedKV), vp, C.c_int,
                                             C.POINTER(Watch), vp, sz, vp]
         L.spd_set_bf16_math.argtypes = [C.c_int32]
-        L.spd_set_prefill_keys.argtypes = [C.c_int32]
+        L.spd_set_prefill_rows.argtypes = [C.c_int32]
         L.spd_merge_partials.argtypes = [C.POINTER(Shape), C.c_int32, C.POINTER(Partial), vp, C.c_int, vp]
         L.spd_prefill_attn.argtypes = [C.POINTER(Shape), C.c_int64, vp, vp, vp, vp, vp, vp, C.c_int32, vp, vp, vp, vp,
                                        C.c_int, vp, sz, vp]
@@ -311,9 +311,9 @@ def spd_set_bf16_math(path: int) -> None:
     _check(lib().spd_set_bf16_math(int(path)), "spd_set_bf16_math")
 
 
-def spd_set_prefill_keys(keys: int) -> None:
-    """Keys per prefill block: 0 = chosen per call from the mean prompt length (default), 64 or 128; process-wide."""
-    _check(lib().spd_set_prefill_keys(int(keys)), "spd_set_prefill_keys")
+def spd_set_prefill_rows(rows: int) -> None:
+    """Query rows per prefill CTA: 0 = chosen per call from the mean prompt length (default), 128 or 256; process-wide."""
+    _check(lib().spd_set_prefill_rows(int(rows)), "spd_set_prefill_rows")
 
 
 def spd_merge_partials(shape, parts, out, stream=None) -> None:

@@ -11,7 +11,7 @@
 
 #include "spd_kernels.cuh"
 #include "spd_prefill.cuh"
-#include "spd_prefill_wide.cuh"
+#include "spd_prefill_pair.cuh"
 
 namespace {
 
@@ -33,8 +33,8 @@ void prof_mark(int job, int k, cudaStream_t st) {
 
 std::atomic<uint32_t> g_epoch{0};
 std::atomic<int> g_bf16_math{0};   // 0 = tensor cores (default), 1 = FMA pipes (comparison arm)
-std::atomic<int> g_prefill_keys{0};   // keys per prefill block: 0 = by mean prompt length, 64, 128
-constexpr int64_t kPrefillWideFrom = 1024;   // mean prompt length from which the 128-key kernel is used
+std::atomic<int> g_prefill_rows{0};   // query rows per prefill CTA: 0 = by mean prompt length, 128, 256
+constexpr int64_t kPrefillPairFrom = 256;    // mean prompt length from which the 256-row kernel is used
 
 // Ids of calls: non-zero, so that a zeroed workspace matches none.
 int32_t next_epoch() {
@@ -461,16 +461,15 @@ spd_status spd_prefill_attn(const spd_shape *shape, int64_t total_tokens, const 
     if (cudaGetLastError() != cudaSuccess) return SPD_ERR_CUDA;
     if (T == 0) return SPD_OK;
 
-    // Long prompts go to the kernel with 128-key blocks (one CTA per SM, MMAs of twice the size); short ones
-    // to the 64-key kernel, whose two CTAs per SM hide each other's start and end.  Only the mean length is
+    // Long prompts go to the kernel with two 128-row tiles per CTA (each K/V block crosses from L2 once for
+    // 256 rows); short ones to the one-tile kernel, whose CTAs are finer grained.  Only the mean length is
     // known on the host.
-    const int keys_pref = g_prefill_keys.load();
-    const bool wide = keys_pref == 128 || (keys_pref == 0 && T / shape->batch >= kPrefillWideFrom);
-    const int krows = wide ? kPwKeys : kPfKeys;
+    const int rows_pref = g_prefill_rows.load();
+    const bool pair = rows_pref == 256 || (rows_pref == 0 && T / shape->batch >= kPrefillPairFrom);
     CUtensorMap mq, mk, mv;
     if ((rc = make_prompt_map(&mq, q, T, shape->num_q_heads, kPfBlock)) != SPD_OK) return rc;
-    if ((rc = make_prompt_map(&mk, k, T, shape->num_kv_heads, krows)) != SPD_OK) return rc;
-    if ((rc = make_prompt_map(&mv, v, T, shape->num_kv_heads, krows)) != SPD_OK) return rc;
+    if ((rc = make_prompt_map(&mk, k, T, shape->num_kv_heads, kPfKeys)) != SPD_OK) return rc;
+    if ((rc = make_prompt_map(&mv, v, T, shape->num_kv_heads, kPfKeys)) != SPD_OK) return rc;
     PrefillParams pp;
     pp.B = shape->batch; pp.Hq = shape->num_q_heads; pp.Hkv = shape->num_kv_heads; pp.T = T;
     pp.sm_scale = shape->sm_scale; pp.tok_indptr = tok_indptr; pp.out = out; pp.out_bf16 = out_dtype == SPD_BF16;
@@ -483,13 +482,14 @@ spd_status spd_prefill_attn(const spd_shape *shape, int64_t total_tokens, const 
         attr_err = cudaFuncSetAttribute(prefill_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                         static_cast<int>(prefill_smem_bytes()));
         if (attr_err == cudaSuccess)
-            attr_err = cudaFuncSetAttribute(prefill_wide_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                            static_cast<int>(prefill_wide_smem_bytes()));
+            attr_err = cudaFuncSetAttribute(prefill_pair_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                            static_cast<int>(prefill_pair_smem_bytes()));
     });
     if (attr_err != cudaSuccess) return SPD_ERR_CUDA;
-    const int64_t max_blocks = (T + kPfBlock - 1) / kPfBlock + shape->batch;   // >= sum over users of ceil(len / 128)
+    const int rows = pair ? kPpRows : kPfBlock;
+    const int64_t max_blocks = (T + rows - 1) / rows + shape->batch;   // >= sum over users of ceil(len / rows)
     dim3 grid(static_cast<unsigned>(max_blocks), static_cast<unsigned>(shape->num_q_heads));
-    if (wide) prefill_wide_kernel<<<grid, kPwThreads, prefill_wide_smem_bytes(), st>>>(pp, mq, mk, mv);
+    if (pair) prefill_pair_kernel<<<grid, kPpThreads, prefill_pair_smem_bytes(), st>>>(pp, mq, mk, mv);
     else prefill_kernel<<<grid, kPfThreads, prefill_smem_bytes(), st>>>(pp, mq, mk, mv);
     ++g_launches;
     return cudaGetLastError() == cudaSuccess ? SPD_OK : SPD_ERR_CUDA;
@@ -652,9 +652,9 @@ spd_status spd_set_bf16_math(int32_t path) {
     return SPD_OK;
 }
 
-spd_status spd_set_prefill_keys(int32_t keys) {
-    if (keys != 0 && keys != 64 && keys != 128) return SPD_ERR_INVALID_ARG;
-    g_prefill_keys.store(keys);
+spd_status spd_set_prefill_rows(int32_t rows) {
+    if (rows != 0 && rows != 128 && rows != 256) return SPD_ERR_INVALID_ARG;
+    g_prefill_rows.store(rows);
     return SPD_OK;
 }
 

@@ -42,12 +42,12 @@ def _case(lens, hq, hkv, seed, slack_pages=1):
 MANY_USERS = [int(x) for x in np.random.default_rng(70).integers(0, 200, size=70) * (np.arange(70) % 7 != 3)]
 
 
-@pytest.fixture(params=[64, 128], ids=["keys64", "keys128"])
+@pytest.fixture(params=[128, 256], ids=["rows128", "rows256"])
 def tile(request):
-    """Both prefill kernels (64-key and 128-key blocks) must pass every case; the default picks by length."""
-    spd.spd_set_prefill_keys(request.param)
+    """Both prefill kernels (one or two 128-row tiles per CTA) must pass every case; the default picks by length."""
+    spd.spd_set_prefill_rows(request.param)
     yield request.param
-    spd.spd_set_prefill_keys(0)
+    spd.spd_set_prefill_rows(0)
 
 
 @pytest.mark.parametrize("lens,hq,hkv", [([128], 1, 1), ([100], 2, 1), ([300, 1, 129, 0, 257], 4, 2), ([1000, 640], 8, 2),
