@@ -355,7 +355,7 @@ def time_prefill(spd, dev, steps=5, case=PREFILL_CASE):
     return {"workload": f"{B} prompts, lengths U[{case['prompt_lo']},{case['prompt_hi']}] ({T} tokens), {hq}/{hkv} heads, D {D}, bf16",
             "ms": ms, "tokens_per_s": T / ms * 1e3,
             "roofline": {"bound": "tensor", "achieved": tf, "peak": peak, "unit": "TFLOP/s", "frac": tf / peak,
-                         "traffic": None, "kernel": "prefill_kernel", "peak_source": src}}
+                         "traffic": None, "kernel": "prefill_pair_kernel", "peak_source": src}}
 
 
 def time_append(spd, w, shape, ws, calls=8):
