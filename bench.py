@@ -388,6 +388,55 @@ def time_append(spd, w, shape, ws, calls=8):
     return {"us_per_call": min(ms) * 1e3, "bytes_written_per_call": nbytes, "note": "latency-bound: one small kernel"}
 
 
+def time_token_step(spd, w, shape, ws, n_layers=8, replays=4):
+    """spd_token_step: the append plus the fused decode step for each of `n_layers` layers (every layer with its
+    own copy of the caches), run eagerly and replayed from one CUDA graph; microseconds per token step.  Every
+    run appends a token per user and layer, so the lengths are first moved back by the number of runs."""
+    if int(w.pub.seq_lens.min()) < 1:
+        return None
+    dev = w.q.device
+    runs = 2 * (replays + 2)
+    gen = torch.Generator(device=dev)
+    gen.manual_seed(101)
+    layers = []
+    for i in range(n_layers):
+        priv = wl.PagedKV(w.priv.k_pool.clone(), w.priv.v_pool.clone(), w.priv.page_indptr, w.priv.page_indices, w.priv.seq_lens)
+        pub = wl.PagedKV(w.pub.k_pool.clone(), w.pub.v_pool.clone(), w.pub.page_indptr, w.pub.page_indices,
+                         torch.clamp(w.pub.seq_lens - runs, min=0))
+        k_new = torch.randn((w.batch, w.num_kv_heads, w.head_dim), generator=gen, device=dev).to(w.dtype)
+        v_new = torch.randn((w.batch, w.num_kv_heads, w.head_dim), generator=gen, device=dev).to(w.dtype)
+        out = torch.empty((w.batch, w.num_q_heads, w.head_dim), dtype=torch.float32, device=dev)
+        layers.append((w.q, k_new, v_new, priv, pub, out))
+    if any(int((p[4].seq_lens + runs > (p[4].page_indptr[1:] - p[4].page_indptr[:-1]) * 16).sum()) for p in layers[:1]):
+        return None                                    # some user's listed pages cannot take that many tokens
+    sa = torch.cuda.Stream()
+
+    def timed(fn, n):
+        for _ in range(2):
+            fn()
+        torch.cuda.synchronize()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record(sa)
+        for _ in range(n):
+            fn()
+        e1.record(sa)
+        torch.cuda.synchronize()
+        return e0.elapsed_time(e1) / n * 1e3
+
+    with torch.cuda.stream(sa):
+        eager = timed(lambda: spd.spd_token_step(shape, layers, ws, stream=sa), replays)
+        graph = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(graph, stream=sa):
+            spd.spd_token_step(shape, layers, ws, stream=sa)
+        replay = timed(graph.replay, replays)
+    code, bad = spd.spd_query_device_status(ws, stream=sa)
+    if code != spd.SPD_OK:
+        raise RuntimeError(f"token step failed: status {code}, user {bad}")
+    kv = sum(int(p[3].seq_lens.sum()) + int(p[4].seq_lens.sum()) for p in layers) * 2 * w.num_kv_heads * w.head_dim * w.elem_size
+    return {"layers": n_layers, "eager_us": eager, "graph_us": replay, "kernels_per_step": 2 * n_layers,
+            "kv_gbs_graph": kv / replay / 1e3}
+
+
 def run_cuda(args):
     from paper_2409_19134_b200 import binding as spd
     rank, local_rank, world = dist_env()
@@ -479,6 +528,7 @@ def run_cuda(args):
         line["prefill"] = time_prefill(spd, dev)
         line["schedules"] = time_schedules(spd, w, spd.make_shape(w.batch, w.num_q_heads, w.num_kv_heads, w.head_dim, w.dtype, w.sm_scale))
         line["append_kv"] = time_append(spd, w, spd.make_shape(w.batch, w.num_q_heads, w.num_kv_heads, w.head_dim, w.dtype, w.sm_scale), ws)
+        line["token_step"] = time_token_step(spd, w, spd.make_shape(w.batch, w.num_q_heads, w.num_kv_heads, w.head_dim, w.dtype, w.sm_scale), ws)
         w = wl.make_workload(cfg, device="cpu")
         line["cpu_baseline"] = cpu_baseline(w)
     print(json.dumps(line), flush=True)

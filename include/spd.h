@@ -188,6 +188,29 @@ spd_status spd_append_kv(const spd_shape *shape, const void *k_new, const void *
                          void *cuda_stream);
 
 /*
+ * One token step over `num_layers` layers (protocol step 3 for every layer of the model; Fig. 3 steps 2 to
+ * 5): for each layer in order, the new token's K and V rows are appended to that layer's public cache
+ * (spd_append_kv) and the layer's decode step runs fused (spd_decode_step).  `layers` is a HOST array;
+ * every pointer inside it is a device pointer that the caller owns.  Each layer brings its own caches,
+ * page tables and lengths (layers[i].pub's pools and seq_lens are written by the append), its own q and
+ * its own output.  In a model q of layer i+1 depends on layer i's output through the weights; those are
+ * not this library's, so all inputs are taken as given and the driver only fixes the order and the launch
+ * structure: 2 * num_layers kernels on `cuda_stream`, nothing else, so that a caller can capture the whole
+ * token step in one CUDA graph and replay it (what the call id and the share table do under replay is
+ * described with spd_decode_step).  The workspace is shared by the layers.  Stops at the first host-side
+ * error; device-side mistakes are reported through spd_query_device_status as for the single calls.
+ */
+typedef struct {
+    const void *q;             /* [batch][num_q_heads][head_dim]                                  */
+    const void *k_new, *v_new; /* [batch][num_kv_heads][head_dim]: this layer's new token         */
+    spd_paged_kv priv;         /* this layer's private (prompt) cache                             */
+    spd_paged_kv pub;          /* this layer's public cache; pools and seq_lens are written       */
+    void *out;                 /* [batch][num_q_heads][head_dim] in out_dtype                     */
+} spd_layer;
+spd_status spd_token_step(const spd_shape *shape, int32_t num_layers, const spd_layer *layers,
+                          spd_dtype out_dtype, void *ws, size_t ws_bytes, void *cuda_stream);
+
+/*
  * spd_decode_step (fused) for a caller whose per-step data lives in HOST memory (no counterpart in
  * the paper, whose two processes exchange these arrays through the host on every layer).
  *

@@ -23,7 +23,7 @@ EXPORTS = ["spd_workspace_size", "spd_partial_attn", "spd_service_attn_merge", "
            "spd_kernel_launch_count", "spd_status_string", "spd_profile_begin", "spd_profile_end",
            "spd_decode_step_static", "spd_append_kv",
            "spd_partial_attn_watch", "spd_decode_step_watch", "spd_set_bf16_math", "spd_merge_partials", "spd_prefill_attn",
-           "spd_set_prefill_rows"]
+           "spd_set_prefill_rows", "spd_token_step"]
 
 
 class SpdError(RuntimeError):
@@ -40,6 +40,11 @@ class Shape(C.Structure):
 class PagedKV(C.Structure):
     _fields_ = [("k_pool", C.c_void_p), ("v_pool", C.c_void_p), ("num_pages", C.c_int32),
                 ("page_indptr", C.c_void_p), ("page_indices", C.c_void_p), ("seq_lens", C.c_void_p)]
+
+
+class Layer(C.Structure):
+    _fields_ = [("q", C.c_void_p), ("k_new", C.c_void_p), ("v_new", C.c_void_p), ("priv", PagedKV), ("pub", PagedKV),
+                ("out", C.c_void_p)]
 
 
 class StepBlob(C.Structure):
@@ -89,6 +94,7 @@ def lib() -> C.CDLL:
                                             C.POINTER(Watch), vp, sz, vp]
         L.spd_set_bf16_math.argtypes = [C.c_int32]
         L.spd_set_prefill_rows.argtypes = [C.c_int32]
+        L.spd_token_step.argtypes = [C.POINTER(Shape), C.c_int32, C.POINTER(Layer), C.c_int, vp, sz, vp]
         L.spd_merge_partials.argtypes = [C.POINTER(Shape), C.c_int32, C.POINTER(Partial), vp, C.c_int, vp]
         L.spd_prefill_attn.argtypes = [C.POINTER(Shape), C.c_int64, vp, vp, vp, vp, vp, vp, C.c_int32, vp, vp, vp, vp,
                                        C.c_int, vp, sz, vp]
@@ -285,6 +291,16 @@ def spd_append_kv(shape, k_new, v_new, part, ws, stream=None) -> None:
                                part.v_pool.data_ptr(), int(part.k_pool.shape[0]), part.page_indptr.data_ptr(),
                                _ptr(part.page_indices), part.seq_lens.data_ptr(), ws.data_ptr(), ws.numel(),
                                _stream_ptr(stream)), "spd_append_kv")
+
+
+def spd_token_step(shape, layers, ws, stream=None) -> None:
+    """layers: a sequence of (q, k_new, v_new, priv, pub, out) per layer; appends to each pub and runs each decode step."""
+    arr = (Layer * len(layers))()
+    for i, (q, k_new, v_new, priv, pub, out) in enumerate(layers):
+        assert q.is_contiguous() and k_new.is_contiguous() and v_new.is_contiguous() and out.is_contiguous()
+        arr[i] = Layer(q.data_ptr(), k_new.data_ptr(), v_new.data_ptr(), paged_kv(priv), paged_kv(pub), out.data_ptr())
+    _check(lib().spd_token_step(C.byref(shape), len(layers), arr, _dtype_code(layers[0][5].dtype), ws.data_ptr(),
+                                ws.numel(), _stream_ptr(stream)), "spd_token_step")
 
 
 def _watch(tok_lo, tok_hi, out) -> Watch:

@@ -542,6 +542,23 @@ spd_status spd_append_kv(const spd_shape *shape, const void *k_new, const void *
     return cudaGetLastError() == cudaSuccess ? SPD_OK : SPD_ERR_CUDA;
 }
 
+spd_status spd_token_step(const spd_shape *shape, int32_t num_layers, const spd_layer *layers, spd_dtype out_dtype,
+                          void *ws, size_t ws_bytes, void *cuda_stream) {
+    if (!layers || num_layers <= 0) return SPD_ERR_INVALID_ARG;
+    for (int32_t i = 0; i < num_layers; ++i) {
+        const spd_layer &ly = layers[i];
+        // the append writes through pointers that spd_paged_kv declares const for the readers
+        spd_status rc = spd_append_kv(shape, ly.k_new, ly.v_new, const_cast<void *>(ly.pub.k_pool),
+                                      const_cast<void *>(ly.pub.v_pool), ly.pub.num_pages, ly.pub.page_indptr,
+                                      ly.pub.page_indices, const_cast<int32_t *>(ly.pub.seq_lens), ws, ws_bytes,
+                                      cuda_stream);
+        if (rc != SPD_OK) return rc;
+        rc = spd_decode_step(shape, ly.q, &ly.priv, &ly.pub, ly.out, out_dtype, 1, ws, ws_bytes, cuda_stream);
+        if (rc != SPD_OK) return rc;
+    }
+    return SPD_OK;
+}
+
 spd_status spd_step_blob_layout(const spd_shape *shape, int64_t priv_pages_listed, int64_t pub_pages_listed,
                                 spd_dtype out_dtype, spd_step_blob *layout) {
     spd_status rc = check_shape(shape);

@@ -89,3 +89,55 @@ def test_cuda_graph_replay(name):
     torch.cuda.synchronize()
     assert spd.spd_query_device_status(ws) == (spd.SPD_OK, -1)
     assert_close(out.cpu().numpy(), ref2, w.dtype, f"{name} graph replay with new q")
+
+
+@pytest.mark.parametrize("dtype", ["bf16", "f32"])
+def test_token_step_over_layers_eager_and_as_one_graph(dtype):
+    """Step 3 for every layer of a model in one call: per layer the append, then the fused decode step.  Run once
+    eagerly, then captured in a CUDA graph and replayed twice; after every run each layer's output, cache and
+    lengths must be what the oracle gets from the same number of appends."""
+    n_layers, B, hq, hkv, d = 3, 5, 8, 2, 128
+    rng = np.random.default_rng(61)
+    layers_cpu, layers_gpu, oracles = [], [], []
+    shape = None
+    for i in range(n_layers):
+        lin, lout = rng.integers(1, 400, size=B), rng.integers(1, 90, size=B)
+        cfg = dict(name=f"layer{i}", batch=B, hq=hq, hkv=hkv, d=d, dtype=dtype, lin=("const", 0), lout=("const", 0), seed=62 + i)
+        w = wl.make_workload(cfg, lengths=(lin, lout))
+        w.pub.seq_lens = torch.clamp(w.pub.seq_lens - 3, min=0)          # room for three more tokens in the listed pages
+        gen = torch.Generator().manual_seed(70 + i)
+        k_new = torch.randn((B, hkv, d), generator=gen).to(w.dtype)
+        v_new = torch.randn((B, hkv, d), generator=gen).to(w.dtype)
+        wg = w.to("cuda")
+        out = torch.full((B, hq, d), float("nan"), dtype=torch.float32, device="cuda")
+        layers_cpu.append((w, k_new, v_new))
+        layers_gpu.append((wg.q, k_new.cuda(), v_new.cuda(), wg.priv, wg.pub, out))
+        oracles.append(oracle_inputs(w))
+        shape = spd.make_shape(B, hq, hkv, d, w.dtype, w.sm_scale)
+    ws = spd.alloc_workspace(shape)
+
+    def bits(t):
+        return t.cpu().view(torch.int16 if t.dtype == torch.bfloat16 else torch.int32).numpy()
+
+    def check(what):
+        torch.cuda.synchronize()
+        assert spd.spd_query_device_status(ws) == (spd.SPD_OK, -1)
+        for i, ((w, k_new, v_new), (q, kin, kout), lg) in enumerate(zip(layers_cpu, oracles, layers_gpu)):
+            assert orc.append(kout, orc.q_from_torch(k_new), orc.q_from_torch(v_new)).all()
+            pub, out = lg[4], lg[5]
+            assert np.array_equal(pub.seq_lens.cpu().numpy(), kout.seq_lens), f"{what}: lengths of layer {i}"
+            assert np.array_equal(bits(pub.k_pool), kout.k_pool.view(bits(pub.k_pool).dtype)), f"{what}: K cache of layer {i}"
+            assert np.array_equal(bits(pub.v_pool), kout.v_pool.view(bits(pub.v_pool).dtype)), f"{what}: V cache of layer {i}"
+            assert_close(out.cpu().numpy(), orc.full(q, kin, kout, w.sm_scale), w.dtype, f"{what}: layer {i}")
+            out.fill_(float("nan"))
+
+    launches = spd.spd_kernel_launch_count()
+    spd.spd_token_step(shape, layers_gpu, ws)
+    assert spd.spd_kernel_launch_count() - launches == 2 * n_layers
+    check("eager")
+    graph = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(graph):
+        spd.spd_token_step(shape, layers_gpu, ws)
+    for r in range(2):
+        graph.replay()
+        check(f"graph replay {r}")
