@@ -258,7 +258,7 @@ def time_e2e(spd, w, shape, ws, steps, warmup):
 def time_schedules(spd, w, shape, steps=200):
     """The same step scheduled four ways, microseconds per step by CUDA events: the two halves chained on one
     stream, the halves on two streams followed by the stand-alone merge, the fused step, and the fused
-    step replayed from a CUDA graph (20 steps per graph)."""
+    step replayed from a CUDA graph (20 steps per graph); then each half alone, and the spread of single steps."""
     dev = w.q.device
     out = torch.empty((w.batch, w.num_q_heads, w.head_dim), dtype=torch.float32, device=dev)
     ws_a, ws_b = spd.alloc_workspace(shape), spd.alloc_workspace(shape)
@@ -291,6 +291,19 @@ def time_schedules(spd, w, shape, steps=200):
         return e0.elapsed_time(e1) / n * 1e3
 
     res = {"chained_us": timed(chained, steps), "two_streams_us": timed(two_streams, steps), "fused_us": timed(fused, steps)}
+    # the two halves of the protocol on their own: the per-user call (private partial) and the service call
+    # (public partial + merge of a given private partial)
+    res["partial_attn_us"] = timed(lambda: spd.spd_partial_attn(shape, w.q, w.priv, pa, ws_a, stream=sa), steps)
+    res["service_attn_merge_us"] = timed(lambda: spd.spd_service_attn_merge(shape, w.q, w.pub, pa, out, ws_a, stream=sa), steps)
+    # spread of single fused steps: an event between every two calls
+    evs = [torch.cuda.Event(enable_timing=True) for _ in range(steps + 1)]
+    evs[0].record(sa)
+    for i in range(steps):
+        fused()
+        evs[i + 1].record(sa)
+    torch.cuda.synchronize()
+    per = np.array([evs[i].elapsed_time(evs[i + 1]) for i in range(steps)]) * 1e3
+    res["fused_step_us"] = {"median": float(np.median(per)), "best": float(per.min()), "p95": float(np.percentile(per, 95))}
     per_graph = 20
     graph = torch.cuda.CUDAGraph()
     with torch.cuda.stream(sa):
