@@ -162,7 +162,7 @@ spd_status spd_decode_step_watch(const spd_shape *shape, const void *q, const sp
  *   page_indices[page_indptr[u] + t / page_size], slot t % page_size, and seq_lens[u] is set to the
  *   prompt's length.  A user whose listed pages cannot hold its prompt, or whose offsets are inconsistent,
  *   is skipped and raises SPD_ERR_BAD_PAGE in the status words at the start of `ws`.
- * Supported: BF16, head_dim 128.  Two kernels on `cuda_stream`: the copy into the cache and the attention
+ * Supported: BF16, head_dim 128, sm_scale > 0 (else SPD_ERR_UNSUPPORTED).  Two kernels on `cuda_stream`: the copy into the cache and the attention
  * (tcgen05 tensor-core MMAs with accumulators in tensor memory).
  */
 spd_status spd_prefill_attn(const spd_shape *shape, int64_t total_tokens, const void *q, const void *k,

@@ -438,6 +438,7 @@ spd_status spd_prefill_attn(const spd_shape *shape, int64_t total_tokens, const 
     spd_status rc = check_shape(shape);
     if (rc != SPD_OK) return rc;
     if (shape->dtype != SPD_BF16 || shape->head_dim != 128) return SPD_ERR_UNSUPPORTED;
+    if (!(shape->sm_scale > 0.f)) return SPD_ERR_UNSUPPORTED;   // the kernels take row maxima before scaling
     if (out_dtype != SPD_F32 && out_dtype != SPD_BF16) return SPD_ERR_UNSUPPORTED;
     if (total_tokens < 0 || total_tokens >= (1ll << 31) - kPfBlock) return SPD_ERR_INVALID_ARG;
     if (!tok_indptr || !page_indptr || !seq_lens || !ws || misaligned(ws, 256)) return SPD_ERR_INVALID_ARG;
