@@ -29,6 +29,10 @@ MUTANTS = [
     ("merge forgets the weight on l", "L += w * parts_l[c * rows + r];", "L += parts_l[c * rows + r];", 0),
     ("merge forgets the weight on O", "o_out[r * D + d] += w * parts_o", "o_out[r * D + d] += parts_o", 0),
     ("alpha applied the wrong way", "(l_in[r] + alpha * l_out[r])", "(l_in[r] + l_out[r] / alpha)", 0),
+    ("prefill: first token sees nothing", "n = i - first + 1;", "n = i - first;", 0),
+    ("prefill: user boundary off by one", "tok_indptr[u + 1] <= i) ++u;", "tok_indptr[u + 1] < i) ++u;", 0),
+    ("prefill: scale dropped", "sc[j] = s->sm_scale * acc;", "sc[j] = acc;", 0),
+    ("prefill: values in reverse order", "widen(v, ((first + j) * Hkv + kvh) * D + d, s->dtype);", "widen(v, ((first + n - 1 - j) * Hkv + kvh) * D + d, s->dtype);", 0),
     ("range lower bound ignored", "for (int64_t t = tok_lo; t < hi; ++t) {\n                double p", "for (int64_t t = 0; t < hi; ++t) {\n                double p", 0),
 ]
 
@@ -44,6 +48,7 @@ BATTERY = [
     pins.test_gqa_head_map_is_contiguous_groups,
     pins.test_indexing_probe_one_hot_query,
     pins.test_bf16_bits_are_widened_exactly_and_page_shuffle_is_invisible,
+    pins.test_prefill_is_causal_softmax_and_hands_over_to_decode,
 ]
 
 
