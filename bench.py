@@ -504,7 +504,8 @@ def run_cuda(args):
         "config": {"workload": cfg, "users": w.batch, "q_heads": w.num_q_heads, "kv_heads": w.num_kv_heads,
                    "head_dim": w.head_dim, "page_size": w.page_size, "kv_bytes_per_step": kvb,
                    "parallelism": "replicas only" if world > 1 else "single GPU", "call": "spd_decode_step(fused=1)", "bf16_math": args.bf16_math,
-                   "l2": "inputs larger than L2 (KV bytes per step >> 126 MB); no flush"},
+                   "l2": ("inputs larger than L2 (KV bytes per step >> 126 MB); no flush" if w.kv_bytes() > 4 * 126e6 else
+                          "inputs FIT in L2 and are not flushed: a latency figure, not comparable with the HBM roofline")},
         "user_tokens_per_s": world * w.batch / ms_max * 1e3,
         "pct_of_nominal_hbm_8000": 100.0 * value / world / NOMINAL_HBM_GBS,
         "pct_of_measured_hbm": 100.0 * value / world / peak,
