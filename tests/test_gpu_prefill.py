@@ -101,3 +101,41 @@ def test_prefill_bf16_output_and_full_cache_is_flagged(tile):
     ref = orc.prefill(orc.q_from_torch(q), orc.q_from_torch(k), orc.q_from_torch(v), ip, scale)
     got = out.float().cpu().numpy()
     assert np.max(np.abs(got - ref)) <= TOL_ABS + 2.0 ** -8 * np.max(np.abs(ref))   # attention itself is still computed
+
+
+@pytest.mark.parametrize("seed", range(8))
+def test_prefill_random_shapes(seed, tile):
+    """Seeded random batches (users with no prompt, prompts that end just before, on and just after a block edge,
+    every head grouping): sampled rows against the oracle, cache hand-over bit for bit."""
+    rng = np.random.default_rng(1000 + seed)
+    B = int(rng.integers(1, 7))
+    hq, hkv = [(1, 1), (2, 1), (4, 2), (8, 8), (8, 1), (4, 4)][int(rng.integers(0, 6))]
+    edges = np.array([0, 1, 63, 64, 65, 127, 128, 129, 191, 192, 193, 255, 256, 257, 383, 384, 385, 511, 512, 513])
+    lens = [int(edges[rng.integers(0, len(edges))]) if rng.random() < 0.5 else int(rng.integers(0, 900)) for _ in range(B)]
+    if sum(lens) == 0:
+        lens[0] = 130
+    q, k, v, ip, part = _case(lens, hq, hkv, seed=2000 + seed)
+    T = int(ip[-1])
+    scale = float(rng.choice([1.0 / np.sqrt(128.0), 0.05, 0.2]))
+    rows = np.unique(np.concatenate([rng.integers(0, T, size=min(T, 150)), ip[1:] - 1, ip[:-1]]))
+    rows = rows[(rows >= 0) & (rows < T)]
+    ref = orc.prefill(orc.q_from_torch(q), orc.q_from_torch(k), orc.q_from_torch(v), ip, scale, rows)
+    shape = spd.make_shape(B, hq, hkv, 128, torch.bfloat16, scale)
+    ws = spd.alloc_workspace(shape)
+    pg = part.to("cuda")
+    out = torch.full((T, hq, 128), float("nan"), dtype=torch.float32, device="cuda")
+    spd.spd_prefill_attn(shape, q.cuda(), k.cuda(), v.cuda(), torch.from_numpy(ip).cuda(), pg, out, ws)
+    assert spd.spd_query_device_status(ws) == (spd.SPD_OK, -1)
+    full = out.cpu().numpy().astype(np.float64)
+    assert np.all(np.isfinite(full)), "a row of some prompt was not written"
+    got = full[rows]
+    # scales up to 0.2 make rows on which one or two keys take nearly all the weight; there the bf16 rounding of P
+    # (relative 2^-9 per weight, so at most 2^-9 max|v| on an output) is the whole error and TOL_ABS, derived for
+    # the diffuse rows of scale 1/sqrt(D), is too tight: the bound itself is used
+    tol_abs = max(TOL_ABS, 2.0 ** -9 * float(v.float().abs().max()) + 5e-4)
+    assert np.abs(got - ref).max() <= tol_abs and np.linalg.norm(got - ref) / np.linalg.norm(ref) <= TOL_REL, (lens, hq, hkv, scale)
+    okv = orc.kv_from_torch(part)
+    orc.write_prompt_kv(okv, orc.q_from_torch(k), orc.q_from_torch(v), ip)
+    assert np.array_equal(pg.seq_lens.cpu().numpy(), okv.seq_lens)
+    assert np.array_equal(pg.k_pool.cpu().view(torch.int16).numpy().view(np.uint16), okv.k_pool)
+    assert np.array_equal(pg.v_pool.cpu().view(torch.int16).numpy().view(np.uint16), okv.v_pool)
