@@ -321,9 +321,8 @@ def time_schedules(spd, w, shape, steps=200):
 PREFILL_CASE = dict(users=8, prompt_lo=2048, prompt_hi=8192, hq=32, hkv=8, d=128, seed=7)   # Llama-3-8B-shaped prompts
 
 
-def time_prefill(spd, dev, steps=5, case=PREFILL_CASE):
-    """spd_prefill_attn on seeded ragged prompts: causal attention (tensor-bound) plus the K/V hand-over.
-    Flops counted: 4 * D * Hq * sum over users of L (L + 1) / 2 (the causal half only)."""
+def prefill_inputs(spd, dev, case=PREFILL_CASE):
+    """Seeded ragged prompts and an empty private cache with room for them (values drawn on `dev`)."""
     rng = np.random.default_rng(case["seed"])
     lens = rng.integers(case["prompt_lo"], case["prompt_hi"] + 1, size=case["users"])
     B, hq, hkv, D = case["users"], case["hq"], case["hkv"], case["d"]
@@ -342,6 +341,15 @@ def time_prefill(spd, dev, steps=5, case=PREFILL_CASE):
                       torch.zeros((pages, hkv, 16, D), dtype=torch.bfloat16, device=dev),
                       torch.from_numpy(pidx).to(dev), perm, torch.zeros(B, dtype=torch.int32, device=dev))
     shape = spd.make_shape(B, hq, hkv, D, torch.bfloat16, 1.0 / np.sqrt(D))
+    return lens, ip, q, k, v, part, shape
+
+
+def time_prefill(spd, dev, steps=5, case=PREFILL_CASE):
+    """spd_prefill_attn on seeded ragged prompts: causal attention (tensor-bound) plus the K/V hand-over.
+    Flops counted: 4 * D * Hq * sum over users of L (L + 1) / 2 (the causal half only)."""
+    lens, ip, q, k, v, part, shape = prefill_inputs(spd, dev, case)
+    B, hq, hkv, D = case["users"], case["hq"], case["hkv"], case["d"]
+    T = int(ip[-1])
     ws = spd.alloc_workspace(shape, dev)
     out = torch.empty((T, hq, D), dtype=torch.bfloat16, device=dev)
     tip = torch.from_numpy(ip).to(dev)

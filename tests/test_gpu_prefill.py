@@ -139,3 +139,30 @@ def test_prefill_random_shapes(seed, tile):
     assert np.array_equal(pg.seq_lens.cpu().numpy(), okv.seq_lens)
     assert np.array_equal(pg.k_pool.cpu().view(torch.int16).numpy().view(np.uint16), okv.k_pool)
     assert np.array_equal(pg.v_pool.cpu().view(torch.int16).numpy().view(np.uint16), okv.v_pool)
+
+
+def test_prefill_at_the_benchmark_size_on_sampled_rows():
+    """The workload bench.py times (8 prompts of 2 to 8 K tokens, 32/8 heads), in the launch configuration it times
+    (default kernel choice, bf16 output): sampled rows against the oracle, and the cache hand-over bit for bit."""
+    import bench
+    lens, ip, q, k, v, part, shape = bench.prefill_inputs(spd, torch.device("cuda"))
+    T = int(ip[-1])
+    ws = spd.alloc_workspace(shape)
+    out = torch.full((T, 32, 128), float("nan"), dtype=torch.bfloat16, device="cuda")
+    spd.spd_prefill_attn(shape, q, k, v, torch.from_numpy(ip).cuda(), part, out, ws)
+    assert spd.spd_query_device_status(ws) == (spd.SPD_OK, -1)
+    assert bool(torch.isfinite(out.float()).all())
+    rng = np.random.default_rng(5)
+    rows = np.unique(np.concatenate([rng.integers(0, T, size=40), ip[1:] - 1, ip[:-1], ip[:-1] + 255, ip[:-1] + 256]))
+    qh, kh, vh = (orc.q_from_torch(t.cpu()) for t in (q, k, v))
+    ref = orc.prefill(qh, kh, vh, ip, shape.sm_scale, rows)
+    got = out[torch.from_numpy(rows).cuda()].float().cpu().numpy().astype(np.float64)
+    err = np.abs(got - ref)
+    assert err.max() <= TOL_ABS + 2.0 ** -8 * np.abs(ref).max() and np.linalg.norm(got - ref) / np.linalg.norm(ref) <= 3e-3   # bf16 output adds half an ulp
+    pc = wl.PagedKV(part.k_pool.cpu(), part.v_pool.cpu(), part.page_indptr.cpu(), part.page_indices.cpu(), torch.zeros(len(lens), dtype=torch.int32))
+    pc.k_pool.zero_(), pc.v_pool.zero_()
+    okv = orc.kv_from_torch(pc)
+    orc.write_prompt_kv(okv, kh, vh, ip)
+    assert np.array_equal(part.seq_lens.cpu().numpy(), okv.seq_lens)
+    assert np.array_equal(part.k_pool.cpu().view(torch.int16).numpy().view(np.uint16), okv.k_pool)
+    assert np.array_equal(part.v_pool.cpu().view(torch.int16).numpy().view(np.uint16), okv.v_pool)
