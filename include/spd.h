@@ -305,7 +305,7 @@ spd_status spd_set_bf16_math(int32_t path);
 /*
  * Tuning and test aid (no counterpart in the paper): query rows per CTA of spd_prefill_attn from now on,
  * process-wide.  0 (default) = chosen per call from the mean prompt length (256 rows, two tiles sharing
- * their K/V loads, from 256 tokens on, else 128); 128 or 256 force one kernel.  Both compute the same
+ * their K/V loads, from 768 tokens on, else 128); 128 or 256 force one kernel.  Both compute the same
  * thing within tolerance.
  */
 spd_status spd_set_prefill_rows(int32_t rows);

@@ -34,7 +34,7 @@ void prof_mark(int job, int k, cudaStream_t st) {
 std::atomic<uint32_t> g_epoch{0};
 std::atomic<int> g_bf16_math{0};   // 0 = tensor cores (default), 1 = FMA pipes (comparison arm)
 std::atomic<int> g_prefill_rows{0};   // query rows per prefill CTA: 0 = by mean prompt length, 128, 256
-constexpr int64_t kPrefillPairFrom = 256;    // mean prompt length from which the 256-row kernel is used
+constexpr int64_t kPrefillPairFrom = 768;    // mean prompt length from which the 256-row kernel is used
 
 // Ids of calls: non-zero, so that a zeroed workspace matches none.
 int32_t next_epoch() {

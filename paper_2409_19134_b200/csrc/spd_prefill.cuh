@@ -175,6 +175,49 @@ __device__ __forceinline__ void umma_bf16_ta(uint32_t tmem_d, uint32_t tmem_a, u
         ::"r"(tmem_d), "r"(tmem_a), "l"(bdesc), "r"(idesc), "r"(accumulate) : "memory");
 }
 
+// Which (user, query block) a CTA owns: blocks of `rows` query rows are numbered user by user, and within a
+// user from the prompt's end backwards (the heaviest first).  Every warp works it out for itself: lane l sums
+// the blocks of users [l C, (l + 1) C) (independent loads, no early exit), a prefix sum over the lanes finds the
+// chunk that holds block `blk`, and that lane walks its chunk once more (cache hits now).  A user whose offsets
+// are inconsistent ends the list: blocks of earlier users are served, nothing from there on.  qb < 0: no block.
+__device__ __forceinline__ void prefill_find_block(const PrefillParams &p, int rows, int blk, int lane, int &qb, int &first, int &len) {
+    qb = -1; first = 0; len = 0;
+    const int C = (p.B + 31) / 32;
+    const int u0 = lane * C, u1 = min(p.B, u0 + C);
+    int sum = 0;
+    bool bad = false;
+#pragma unroll 4
+    for (int u = u0; u < u1; ++u) {
+        const int64_t a = p.tok_indptr[u], b = p.tok_indptr[u + 1];
+        bad = bad || a < 0 || b < a || b > p.T;
+        if (!bad) sum += static_cast<int>((b - a + rows - 1) / rows);
+    }
+    int inc = sum;
+#pragma unroll
+    for (int d = 1; d < 32; d <<= 1) {
+        const int up = __shfl_up_sync(0xffffffffu, inc, d);
+        if (lane >= d) inc += up;
+    }
+    const unsigned badmask = __ballot_sync(0xffffffffu, bad), hit = __ballot_sync(0xffffffffu, blk < inc);
+    if (!hit) return;
+    const int src = __ffs(hit) - 1;
+    if (badmask & ((1u << src) - 1u)) return;          // an inconsistent user in an earlier chunk
+    int r_qb = -1, r_first = 0, r_len = 0;
+    if (lane == src) {
+        int rem = blk - (inc - sum);
+        for (int u = u0; u < u1; ++u) {
+            const int64_t a = p.tok_indptr[u], b = p.tok_indptr[u + 1];
+            if (a < 0 || b < a || b > p.T) break;     // the sum stopped here too, so rem was used up before
+            const int nb = static_cast<int>((b - a + rows - 1) / rows);
+            if (rem < nb) { r_qb = nb - 1 - rem; r_first = static_cast<int>(a); r_len = static_cast<int>(b - a); break; }
+            rem -= nb;
+        }
+    }
+    qb = __shfl_sync(0xffffffffu, r_qb, src);
+    first = __shfl_sync(0xffffffffu, r_first, src);
+    len = __shfl_sync(0xffffffffu, r_len, src);
+}
+
 // Q, K x2, V x2, then eleven mbarriers and one word; the kernel has no static shared memory, so the
 // 1024-byte alignment of the tiles costs nothing and two CTAs fit one SM.
 constexpr size_t prefill_smem_bytes() { return kPfQTile + 4 * static_cast<size_t>(kPfKvTile) + 128; }   // 11 x 8 + 4 <= 128
@@ -195,37 +238,8 @@ prefill_kernel(const __grid_constant__ PrefillParams p, const __grid_constant__ 
     const int tid = threadIdx.x, wid = tid >> 5;
     const int h = blockIdx.y, kvh = h / (p.Hq / p.Hkv);
 
-    // which (user, query block) this CTA owns; the heaviest blocks (closest to the prompt's end) come first.
-    // Every warp works it out for itself, 32 users at a time: query blocks per user, a prefix sum over the
-    // lanes, the first lane whose running total passes this CTA's index.
-    int qb = -1, first = 0, len = 0;
-    {
-        const int lane = tid & 31;
-        int blk = blockIdx.x;
-        for (int u0 = 0; u0 < p.B; u0 += 32) {
-            const int u = u0 + lane;
-            int64_t a = 0, b = 0;
-            if (u < p.B) { a = p.tok_indptr[u]; b = p.tok_indptr[u + 1]; }
-            const bool bad = a < 0 || b < a || b > p.T;                   // inconsistent offsets: nothing from here on
-            const int nb = bad ? 0 : static_cast<int>((b - a + kPfBlock - 1) / kPfBlock);
-            int inc = nb;
-#pragma unroll
-            for (int d = 1; d < 32; d <<= 1) {
-                const int t = __shfl_up_sync(0xffffffffu, inc, d);
-                if (lane >= d) inc += t;
-            }
-            const unsigned badmask = __ballot_sync(0xffffffffu, bad), hit = __ballot_sync(0xffffffffu, blk < inc);
-            if (hit) {
-                const int src = __ffs(hit) - 1;
-                const int nb_s = __shfl_sync(0xffffffffu, nb, src), inc_s = __shfl_sync(0xffffffffu, inc, src);
-                const int a_s = __shfl_sync(0xffffffffu, static_cast<int>(a), src), b_s = __shfl_sync(0xffffffffu, static_cast<int>(b), src);
-                if (!(badmask & ((1u << src) - 1u))) { qb = nb_s - 1 - (blk - (inc_s - nb_s)); first = a_s; len = b_s - a_s; }
-                break;
-            }
-            if (badmask) break;
-            blk -= __shfl_sync(0xffffffffu, inc, 31);
-        }
-    }
+    int qb, first, len;
+    prefill_find_block(p, kPfBlock, blockIdx.x, tid & 31, qb, first, len);
     if (qb < 0) return;   // uniform over the CTA: no barrier, no TMEM touched yet
     const int nkv = 2 * (qb + 1);   // 64-key blocks up to and including the diagonal
 

@@ -42,34 +42,8 @@ prefill_pair_kernel(const __grid_constant__ PrefillParams p, const __grid_consta
     const int tid = threadIdx.x, wid = tid >> 5, lane = tid & 31;
     const int h = blockIdx.y, kvh = h / (p.Hq / p.Hkv);
 
-    // which (user, 256-row query block) this CTA owns; heaviest blocks first.  Every warp finds it for itself.
-    int qb = -1, first = 0, len = 0;
-    {
-        int blk = blockIdx.x;
-        for (int u0 = 0; u0 < p.B; u0 += 32) {
-            const int u = u0 + lane;
-            int64_t a = 0, b = 0;
-            if (u < p.B) { a = p.tok_indptr[u]; b = p.tok_indptr[u + 1]; }
-            const bool bad = a < 0 || b < a || b > p.T;                   // inconsistent offsets: nothing from here on
-            const int nb = bad ? 0 : static_cast<int>((b - a + kPpRows - 1) / kPpRows);
-            int inc = nb;
-#pragma unroll
-            for (int d = 1; d < 32; d <<= 1) {
-                const int up = __shfl_up_sync(0xffffffffu, inc, d);
-                if (lane >= d) inc += up;
-            }
-            const unsigned badmask = __ballot_sync(0xffffffffu, bad), hit = __ballot_sync(0xffffffffu, blk < inc);
-            if (hit) {
-                const int src = __ffs(hit) - 1;
-                const int nb_s = __shfl_sync(0xffffffffu, nb, src), inc_s = __shfl_sync(0xffffffffu, inc, src);
-                const int a_s = __shfl_sync(0xffffffffu, static_cast<int>(a), src), b_s = __shfl_sync(0xffffffffu, static_cast<int>(b), src);
-                if (!(badmask & ((1u << src) - 1u))) { qb = nb_s - 1 - (blk - (inc_s - nb_s)); first = a_s; len = b_s - a_s; }
-                break;
-            }
-            if (badmask) break;
-            blk -= __shfl_sync(0xffffffffu, inc, 31);
-        }
-    }
+    int qb, first, len;
+    prefill_find_block(p, kPpRows, blockIdx.x, lane, qb, first, len);
     if (qb < 0) return;   // uniform over the CTA: no barrier, no TMEM touched yet
     // Tile t holds rows [256 qb + 128 t, + 128) and needs the 64-key blocks 0 .. 4 qb + 2 t + 1 (the last two
     // straddle its diagonal).  The second tile may lie wholly past the prompt's end: then it is left out.
