@@ -160,10 +160,13 @@ spd_status spd_decode_step_watch(const spd_shape *shape, const void *q, const sp
  *   the same prompt (softmax of sm_scale * q.k, as in the decode calls).
  *   k_pool / v_pool / page tables: the private partition; token t of user u is stored in page
  *   page_indices[page_indptr[u] + t / page_size], slot t % page_size, and seq_lens[u] is set to the
- *   prompt's length.  A user whose listed pages cannot hold its prompt, or whose offsets are inconsistent,
- *   is skipped and raises SPD_ERR_BAD_PAGE in the status words at the start of `ws`.
- * Supported: BF16, head_dim 128, sm_scale > 0 (else SPD_ERR_UNSUPPORTED).  Two kernels on `cuda_stream`: the copy into the cache and the attention
- * (tcgen05 tensor-core MMAs with accumulators in tensor memory).
+ *   prompt's length.  A user whose listed pages cannot hold its prompt is skipped by the hand-over (its
+ *   attention is still computed) and raises SPD_ERR_BAD_PAGE in the status words at the start of `ws`.
+ *   tok_indptr must be non-decreasing and end at total_tokens; where it is not, the users before the first
+ *   inconsistent one are served, the rows of that user and of all later ones are left unwritten, and the
+ *   same status is raised.  Nothing is read or written out of bounds either way.
+ * Supported: BF16, head_dim 128, sm_scale > 0 (else SPD_ERR_UNSUPPORTED).  Two kernels on `cuda_stream`:
+ * the copy into the cache and the attention (tcgen05 tensor-core MMAs with accumulators in tensor memory).
  */
 spd_status spd_prefill_attn(const spd_shape *shape, int64_t total_tokens, const void *q, const void *k,
                             const void *v, const int32_t *tok_indptr, void *k_pool, void *v_pool,

@@ -166,3 +166,27 @@ def test_prefill_at_the_benchmark_size_on_sampled_rows():
     assert np.array_equal(part.seq_lens.cpu().numpy(), okv.seq_lens)
     assert np.array_equal(part.k_pool.cpu().view(torch.int16).numpy().view(np.uint16), okv.k_pool)
     assert np.array_equal(part.v_pool.cpu().view(torch.int16).numpy().view(np.uint16), okv.v_pool)
+
+
+def test_prefill_with_inconsistent_offsets_serves_the_users_before_them(tile):
+    """A user whose token offsets run backwards ends the list: users before it are computed as usual, its own rows
+    and those of later users are not written, and the call reports the mistake instead of faulting."""
+    lens = [200, 150, 100, 120]
+    q, k, v, ip, part = _case(lens, 4, 2, seed=77)
+    T = int(ip[-1])
+    bad_ip = ip.copy()
+    bad_ip[3] = bad_ip[2] - 10                     # user 2 now ends before it begins
+    scale = 1.0 / np.sqrt(128.0)
+    good = int(ip[2])                               # rows of users 0 and 1
+    ref = orc.prefill(orc.q_from_torch(q[:good]), orc.q_from_torch(k[:good]), orc.q_from_torch(v[:good]), ip[:3], scale)
+    shape = spd.make_shape(4, 4, 2, 128, torch.bfloat16, scale)
+    ws = spd.alloc_workspace(shape)
+    pg = part.to("cuda")
+    out = torch.full((T, 4, 128), float("nan"), dtype=torch.float32, device="cuda")
+    spd.spd_prefill_attn(shape, q.cuda(), k.cuda(), v.cuda(), torch.from_numpy(bad_ip).cuda(), pg, out, ws)
+    code, bad = spd.spd_query_device_status(ws)
+    assert code == 4 and bad >= 2
+    got = out.cpu().numpy().astype(np.float64)
+    assert np.abs(got[:good] - ref).max() <= TOL_ABS
+    assert np.all(np.isnan(got[good:]))
+    assert pg.seq_lens.cpu().tolist()[:2] == lens[:2]
