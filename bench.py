@@ -458,6 +458,45 @@ def time_token_step(spd, w, shape, ws, n_layers=8, replays=4):
             "kv_gbs_graph": kv / replay / 1e3}
 
 
+PAPER_SCALE = dict(batch=8, hq=32, hkv=8, d=128, dtype="bf16", lin=("const", 512), lout=("uniform", 1, 128), seed=11)
+
+
+def time_paper_scale(spd, dev, steps=300):
+    """The scale of the paper's own runs (a handful of users, prompts of 64 to 512 tokens, a Llama-3-8B-shaped
+    layer): latency of one fused decode step, of the per-user call alone (one user per call, as the paper's
+    per-user processes issue it) and of the prefill of the same prompts.  Latency-bound: microseconds, no roofline."""
+    w = wl.make_workload(dict(PAPER_SCALE, name="paper_scale"), device=dev)
+    shape = spd.make_shape(w.batch, w.num_q_heads, w.num_kv_heads, w.head_dim, w.dtype, w.sm_scale)
+    ws = spd.alloc_workspace(shape, dev)
+    out = torch.empty((w.batch, w.num_q_heads, w.head_dim), dtype=torch.float32, device=dev)
+
+    def timed(fn, n):
+        for _ in range(10):
+            fn()
+        torch.cuda.synchronize()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        for _ in range(n):
+            fn()
+        e1.record()
+        torch.cuda.synchronize()
+        return e0.elapsed_time(e1) / n * 1e3
+
+    res = {"workload": "8 users, 512-token prompts, 1-128 generated tokens, 32/8 heads, D 128, bf16",
+           "decode_step_us": timed(lambda: spd.spd_decode_step(shape, w.q, w.priv, w.pub, out, ws, fused=True), steps)}
+    one = wl.make_workload(dict(PAPER_SCALE, name="one_user", batch=1), device=dev)
+    shape1 = spd.make_shape(1, w.num_q_heads, w.num_kv_heads, w.head_dim, w.dtype, w.sm_scale)
+    ws1, part1 = spd.alloc_workspace(shape1, dev), spd.alloc_partial(shape1)
+    res["per_user_partial_us"] = timed(lambda: spd.spd_partial_attn(shape1, one.q, one.priv, part1, ws1), steps)
+    case = dict(users=8, prompt_lo=512, prompt_hi=512, hq=32, hkv=8, d=128, seed=11)
+    res["prefill_us"] = time_prefill(spd, dev, steps=20, case=case)["ms"] * 1e3
+    for x in (ws, ws1):
+        code, bad = spd.spd_query_device_status(x)
+        if code != spd.SPD_OK:
+            raise RuntimeError(f"paper-scale run failed: status {code}, user {bad}")
+    return res
+
+
 def run_cuda(args):
     from paper_2409_19134_b200 import binding as spd
     rank, local_rank, world = dist_env()
@@ -550,6 +589,7 @@ def run_cuda(args):
         line["prefill"] = time_prefill(spd, dev)
         line["schedules"] = time_schedules(spd, w, spd.make_shape(w.batch, w.num_q_heads, w.num_kv_heads, w.head_dim, w.dtype, w.sm_scale))
         line["append_kv"] = time_append(spd, w, spd.make_shape(w.batch, w.num_q_heads, w.num_kv_heads, w.head_dim, w.dtype, w.sm_scale), ws)
+        line["paper_scale"] = time_paper_scale(spd, dev)
         line["token_step"] = time_token_step(spd, w, spd.make_shape(w.batch, w.num_q_heads, w.num_kv_heads, w.head_dim, w.dtype, w.sm_scale), ws)
         w = wl.make_workload(cfg, device="cpu")
         line["cpu_baseline"] = cpu_baseline(w)
