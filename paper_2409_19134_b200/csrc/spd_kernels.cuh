@@ -785,10 +785,12 @@ attn_kernel(const __grid_constant__ Params p, const __grid_constant__ CUtensorMa
     static_assert(2 * TB >= (kHeadsPerItem * (D + 4) + 3 * kHeadsPerItem) * 4, "a stage must hold the epilogue staging");
     static_assert(attn_smem_bytes<Math>(kMaxGrid) + 16384 <= 227 * 1024, "ring does not fit shared memory");
     static_assert(Math::kWarps <= 16 && Math::kStages >= 2, "CTA shape");
+    static_assert(2 * Math::kWarps * 32 >= kMaxGrid, "every thread looks after at most two entries of the rate table");
     extern __shared__ uint8_t smem_raw[];
     __shared__ int32_t chunk_pfx[NT + 1];
     __shared__ int32_t warp_tot[Math::kWarps];
-    __shared__ float sh_w[kMaxGrid], sh_r[kMaxGrid];
+    __shared__ float red_w[Math::kWarps], red_r[Math::kWarps];
+    __shared__ int32_t red_ok[Math::kWarps];
     __shared__ int32_t sh_wq[kMaxGrid], sh_pc[kMaxGrid + 1];
     __shared__ int2 sh_np[kUserCache];
     __shared__ long long cta_clock0;
@@ -803,6 +805,10 @@ attn_kernel(const __grid_constant__ Params p, const __grid_constant__ CUtensorMa
     uint8_t *extra = tail + attn_extra_offset<Math>() + static_cast<size_t>(wid) * Math::kExtraBytes;
 
     griddep_launch_dependents();   // the next kernel on the stream may begin its own read-only preamble
+    // the four tensor maps are needed ~7 us from now: fetch them meanwhile (when no partition owns a page they
+    // are never used and hold nothing)
+    if (wid == 0 && lane < 4 && (p.part[0].num_pages > 0 || p.part[1].num_pages > 0))
+        prefetch_tensormap(lane == 0 ? &mk0 : lane == 1 ? &mv0 : lane == 2 ? &mk1 : &mv1);
 
     // ---- plan: every CTA computes the same thing from the inputs alone -------------------------
     // Thread t sums the tiles of users [t*C, (t+1)*C); a block scan gives chunk prefixes.
@@ -813,11 +819,12 @@ attn_kernel(const __grid_constant__ Params p, const __grid_constant__ CUtensorMa
     float2 *rate_wr = p.rates + (p.rate_sel % 3) * kMaxGrid;
     {
         if (threadIdx.x == 0) cta_exits = 0;
-        for (int i = threadIdx.x; i < G; i += NT) {     // the rate table travels together with the lengths
-            const float2 v = __ldcg(rate_rd + i);
-            sh_w[i] = v.x;
-            sh_r[i] = (v.x > 0.f && v.y > 0.f) ? v.x / v.y : 0.f;
-        }
+        // the rate table travels together with the lengths: its loads are issued first and used last, so that
+        // the two round trips to memory overlap (G <= 2 NT)
+        const int i0 = threadIdx.x, i1 = threadIdx.x + NT;
+        float2 v0 = make_float2(0.f, 0.f), v1 = make_float2(0.f, 0.f);
+        if (i0 < G) v0 = __ldcg(rate_rd + i0);
+        if (i1 < G) v1 = __ldcg(rate_rd + i1);
         int sum = 0;
         const int ub = threadIdx.x * C, ue = min(p.B, ub + C);
         for (int u = ub; u < ue; ++u) {
@@ -826,6 +833,18 @@ attn_kernel(const __grid_constant__ Params p, const __grid_constant__ CUtensorMa
             if (u < kUserCache) sh_np[u] = make_int2(n0, n1);
             sum += n0 + n1;
         }
+        // rate = weight / cycles of the entries this thread looks after; their sums over the table by one
+        // fixed tree (butterfly inside a warp, warps in order), so that every thread of every CTA gets the same bits
+        const float r0 = (v0.x > 0.f && v0.y > 0.f) ? v0.x / v0.y : 0.f, r1 = (v1.x > 0.f && v1.y > 0.f) ? v1.x / v1.y : 0.f;
+        float sw = (i0 < G ? v0.x : 0.f) + (i1 < G ? v1.x : 0.f), sr = r0 + r1;
+        const bool ok_mine = (i0 >= G || r0 > 0.f) && (i1 >= G || r1 > 0.f);
+#pragma unroll
+        for (int d = 16; d >= 1; d >>= 1) {
+            sw += __shfl_xor_sync(0xffffffffu, sw, d);
+            sr += __shfl_xor_sync(0xffffffffu, sr, d);
+        }
+        const bool ok_warp = __all_sync(0xffffffffu, ok_mine);
+        if (lane == 0) { red_w[wid] = sw; red_r[wid] = sr; red_ok[wid] = ok_warp; }
         int inc = sum;
 #pragma unroll
         for (int d = 1; d < 32; d <<= 1) {
@@ -838,42 +857,35 @@ attn_kernel(const __grid_constant__ Params p, const __grid_constant__ CUtensorMa
         for (int w = 0; w < wid; ++w) before += warp_tot[w];
         chunk_pfx[threadIdx.x] = before + inc - sum;
         if (threadIdx.x == NT - 1) chunk_pfx[NT] = before + inc;
+        // ---- shares, first half: CTAs do not all stream at the same rate (some SMs sit behind busier
+        // ports), so shares are sized by the rates measured on an earlier call that used this workspace: each
+        // CTA left its (weight, cycles) in the rate table.  New weight = old weight moved towards the measured
+        // rate (both relative to the mean): most of the way when they disagree by more than 4 % (a real
+        // difference between SMs), a quarter of the way otherwise (so that run-to-run noise is averaged out
+        // instead of chased); quantised to integers so that all CTAs cut alike.
+        float tw = 0.f, tr = 0.f;
+        bool ok = true;
+        for (int w = 0; w < Math::kWarps; ++w) { tw += red_w[w]; tr += red_r[w]; ok = ok && red_ok[w] != 0; }
+        const float nw = ok ? G / tw : 0.f, nr = ok ? G / tr : 0.f;
+        auto quantise = [&](float w_old, float r) {
+            const float wn = w_old * nw, rn = r * nr;
+            const float gain = fabsf(rn - wn) > 0.04f * wn ? 0.75f : 0.25f;
+            const float m = ok ? wn + gain * (rn - wn) : 1.f;
+            const int q = static_cast<int>(m * 1024.f + 0.5f);
+            return q < 512 ? 512 : (q > 2048 ? 2048 : q);
+        };
+        if (i0 < G) sh_wq[i0] = quantise(v0.x, r0);
+        if (i1 < G) sh_wq[i1] = quantise(v1.x, r1);
         __syncthreads();
     }
     const int64_t T64 = static_cast<int64_t>(chunk_pfx[NT]) * p.S;
     const int T = T64 >= (1ll << 31) ? 0 : static_cast<int>(T64);
 
-    // ---- shares: warp w of the grid owns tiles [bnd[w], bnd[w+1]) ------------------------------
-    // CTAs do not all stream at the same rate (some SMs sit behind busier ports), so shares are
-    // sized by the rates measured on the previous call that used this workspace: each CTA left its
-    // (weight, cycles) in one half of a double-buffered table; this call reads that half and writes
-    // the other, so every CTA sees the same numbers however late it starts.
-    if (wid == 0) {                  // one fixed reduction tree, so that every CTA rounds alike
-        float sw = 0.f, sr = 0.f;
-        bool ok = true;
-        for (int i = lane; i < G; i += 32) { sw += sh_w[i]; sr += sh_r[i]; ok = ok && sh_r[i] > 0.f; }
-#pragma unroll
-        for (int d = 16; d >= 1; d >>= 1) {
-            sw += __shfl_xor_sync(0xffffffffu, sw, d);
-            sr += __shfl_xor_sync(0xffffffffu, sr, d);
-        }
-        ok = __all_sync(0xffffffffu, ok);
-        const float nw = ok ? G / sw : 0.f, nr = ok ? G / sr : 0.f;
-        // lane l looks after CTAs [l*cpl, (l+1)*cpl)
-        const int cpl = (G + 31) / 32;
+    // ---- shares, second half: warp w of the grid owns tiles [bnd[w], bnd[w+1]); prefix sums of the CTA weights
+    if (wid == 0) {
+        const int cpl = (G + 31) / 32;      // lane l looks after CTAs [l*cpl, (l+1)*cpl)
         int mysum = 0;
-        for (int i = lane * cpl; i < min(G, (lane + 1) * cpl); ++i) {
-            // new weight = old weight moved towards the measured rate (both relative to the mean): most of
-            // the way when they disagree by more than 4 % (a real difference between SMs), a quarter of
-            // the way otherwise (so that run-to-run noise is averaged out instead of chased)
-            const float wn = sh_w[i] * nw, rn = sh_r[i] * nr;
-            const float gain = fabsf(rn - wn) > 0.04f * wn ? 0.75f : 0.25f;
-            const float m = ok ? wn + gain * (rn - wn) : 1.f;
-            int q = static_cast<int>(m * 1024.f + 0.5f);
-            q = q < 512 ? 512 : (q > 2048 ? 2048 : q);
-            sh_wq[i] = q;
-            mysum += q;
-        }
+        for (int i = lane * cpl; i < min(G, (lane + 1) * cpl); ++i) mysum += sh_wq[i];
         int inc = mysum;
 #pragma unroll
         for (int d = 1; d < 32; d <<= 1) {
@@ -893,8 +905,12 @@ attn_kernel(const __grid_constant__ Params p, const __grid_constant__ CUtensorMa
             const int c = w / Math::kWarps;
             return static_cast<int64_t>(Math::kWarps) * sh_pc[c] + static_cast<int64_t>(w - c * Math::kWarps) * (c < G ? sh_wq[c] : 0);
         };
-        const int64_t total = A > 0 ? wsum(A) : 1;
-        for (int w = threadIdx.x; w <= A; w += NT) bnd[w] = static_cast<int32_t>(static_cast<int64_t>(T) * wsum(w) / total);
+        // T * wsum(w) / total in double: the product is an integer below 2^53, hence exact; the quotient may
+        // land one tile off where it is within an ulp of an integer, which moves a cut by a tile and nothing else
+        // (every CTA computes the same bits; wsum is monotone; w = A gives T exactly)
+        const double total = A > 0 ? static_cast<double>(wsum(A)) : 1.0;
+        for (int w = threadIdx.x; w <= A; w += NT)
+            bnd[w] = static_cast<int32_t>(static_cast<double>(T) * static_cast<double>(wsum(w)) / total);
     }
     __syncthreads();
 

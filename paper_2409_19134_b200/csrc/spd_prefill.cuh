@@ -238,6 +238,7 @@ prefill_kernel(const __grid_constant__ PrefillParams p, const __grid_constant__ 
     const int tid = threadIdx.x, wid = tid >> 5;
     const int h = blockIdx.y, kvh = h / (p.Hq / p.Hkv);
 
+    if (tid == 128) { prefetch_tensormap(&mq); prefetch_tensormap(&mk); prefetch_tensormap(&mv); }   // needed right after the search below
     int qb, first, len;
     prefill_find_block(p, kPfBlock, blockIdx.x, tid & 31, qb, first, len);
     if (qb < 0) return;   // uniform over the CTA: no barrier, no TMEM touched yet

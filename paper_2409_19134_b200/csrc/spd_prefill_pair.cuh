@@ -42,6 +42,7 @@ prefill_pair_kernel(const __grid_constant__ PrefillParams p, const __grid_consta
     const int tid = threadIdx.x, wid = tid >> 5, lane = tid & 31;
     const int h = blockIdx.y, kvh = h / (p.Hq / p.Hkv);
 
+    if (tid == 384) { prefetch_tensormap(&mq); prefetch_tensormap(&mk); prefetch_tensormap(&mv); }   // needed right after the search below
     int qb, first, len;
     prefill_find_block(p, kPpRows, blockIdx.x, lane, qb, first, len);
     if (qb < 0) return;   // uniform over the CTA: no barrier, no TMEM touched yet
