@@ -8,6 +8,12 @@ time) of spd_decode_step (fused) with every input resident in HBM; `e2e` is the 
 spd_decode_step_host, whose per-step inputs (q, page tables, lengths) start in one pinned host buffer and
 whose output is read back inside the timed region.  The KV pools are the resident cache in both.
 
+The headline workload is the largest single-GPU configuration (c5_many_user); the GQA configuration
+(c3_llama3_8b_gqa) is measured the same way beside it (`co_headline`), the other two more briefly
+(`other_configs`).  A timed region is `--steps` back-to-back steps between two CUDA events; it is repeated
+until at least a second of GPU time has gone by, and the MEDIAN repeat is reported (the best one beside it),
+so that the figure is the sustained, power-capped one.
+
 With N > 1 (torchrun) every rank runs an independent replica on its own GPU (the path has no exchange
 step) and `value` sums the replicas over the slowest rank's time.
 
@@ -32,7 +38,9 @@ from paper_2409_19134_b200 import workloads as wl  # noqa: E402
 
 METRIC = "decode-attention KV GB/s"
 NOMINAL_HBM_GBS = 8000.0
-OTHER_CONFIGS = ["c3_llama3_8b_gqa", "c4_long_prompt", "c5_many_user"]
+CO_HEADLINE = {"c5_many_user": "c3_llama3_8b_gqa", "c3_llama3_8b_gqa": "c5_many_user"}
+BRIEF_CONFIGS = ["c2_llama2_7b", "c4_long_prompt", "c3_llama3_8b_gqa", "c5_many_user"]
+MIN_GPU_SECONDS = 1.0
 
 
 def measured_peak():
@@ -155,15 +163,27 @@ def oracle_sample(w_cpu, budget_s):
     return run, nb, n_users, n_kvh, cores
 
 
-def cpu_baseline(w_cpu, budget_s=12.0):
+def cpu_baseline(w_cpu, full_batch, budget_s=12.0):
     run, nb, n_users, n_kvh, cores = oracle_sample(w_cpu, budget_s)
     ts = [run()]
-    while sum(ts) < 3.0 and len(ts) < 20:     # a short pass is repeated so that the clock has something to hold
+    while sum(ts) < 10.0 and len(ts) < 40:    # a short pass is repeated: about ten seconds of CPU work in all
         ts.append(run())
     dt = float(np.mean(ts))
     return {"value": nb / dt / 1e9, "unit": "GB/s", "cores": cores, "kind": "oracle",
-            "sample": f"first {n_users} of {w_cpu.batch} users x first {n_kvh} of {w_cpu.num_kv_heads} KV heads, "
+            "sample": f"first {n_users} of {full_batch} users x first {n_kvh} of {w_cpu.num_kv_heads} KV heads, "
                       f"mean of {len(ts)} passes of {dt:.2f} s", "user_tokens_per_s": n_users * n_kvh / w_cpu.num_kv_heads / dt}
+
+
+def sample_workload_cpu(cfg_name, max_users=48, users=None):
+    """The first users of a config, generated on the CPU: same seeded length draw as the full workload (so these
+    are its first users' lengths), values from the CPU generator.  Keeps the oracle legs from building 5 GB pools."""
+    cfg = wl.CONFIGS[cfg_name]
+    lin, lout = wl.make_lengths(cfg)
+    full = cfg["batch"] if users is None else min(users, cfg["batch"])
+    n = min(full, max_users)
+    w = wl.make_workload(dict(cfg, name=cfg_name, batch=n), lengths=(lin[:n], lout[:n]), device="cpu")
+    w.full_kv_bytes = int(lin[:full].sum() + lout[:full].sum()) * 2 * cfg["hkv"] * cfg["d"] * w.elem_size
+    return w, full
 
 
 def run_reference(args):
@@ -171,7 +191,7 @@ def run_reference(args):
     if rank != 0:
         return
     cfg = args.config
-    w = wl.make_workload(cfg, device="cpu")
+    w, full_batch = sample_workload_cpu(cfg, users=args.users)
     steps, warmup = args.steps or 5, args.warmup if args.warmup is not None else 1
     budget = min(15.0, 150.0 / (steps + warmup))
     run, nb, n_users, n_kvh, cores = oracle_sample(w, budget)
@@ -180,44 +200,72 @@ def run_reference(args):
     ts = [run() for _ in range(steps)]
     dt = float(np.mean(ts))
     val = nb / dt / 1e9
-    sample = (f"each step: first {n_users} of {w.batch} users x first {n_kvh} of {w.num_kv_heads} KV heads "
+    sample = (f"each step: first {n_users} of {full_batch} users x first {n_kvh} of {w.num_kv_heads} KV heads "
               f"({nb / 1e6:.1f} MB of KV)")
     line = {"impl": "reference", "metric": METRIC, "value": val, "unit": "GB/s", "n_gpus": args.gpus, "steps": steps,
             "warmup": warmup, "ms_per_step": dt * 1e3, "higher_is_better": True, "scaling": "weak",
             "vs_baseline": None, "dtype": "f64", "data": "synthetic",
-            "config": {"workload": cfg, "sample": sample},
+            "config": workload_config(cfg, w, full_batch, world, args, kv_bytes_per_step=w.full_kv_bytes, sample=sample),
             "cpu_baseline": {"value": val, "unit": "GB/s", "cores": cores, "kind": "oracle", "sample": sample},
             "e2e": {"value": val, "unit": "GB/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
             "gpu_launches": 0}
     print(json.dumps(line), flush=True)
 
 
+def workload_config(cfg, w, users, world, args, **extra):
+    """The `config` object of the JSON line: the same keys for both arms."""
+    c = {"workload": cfg, "users": users, "q_heads": w.num_q_heads, "kv_heads": w.num_kv_heads,
+         "head_dim": w.head_dim, "page_size": w.page_size,
+         "parallelism": "replicas only" if world > 1 else "single GPU", "call": "spd_decode_step(fused=1)",
+         "bf16_math": args.bf16_math}
+    c.update(extra)
+    return c
+
+
 # ------------------------------------------------------------------------------------------------ CUDA arm
-def time_config(spd, w, steps, warmup, fused=True):
-    """Device time of `steps` back-to-back decode steps, by CUDA events on the launching stream."""
+def time_config(spd, w, steps, warmup, fused=True, plan=None, min_seconds=MIN_GPU_SECONDS, max_repeats=400):
+    """Device time of `steps` back-to-back decode steps between two CUDA events on the launching stream, repeated
+    until `min_seconds` of GPU time have gone by.  Returns the median repeat (ms per step), all repeats, and the
+    objects the other measurements reuse.  plan: None = the plain call; 'reuse' = one storing call, then every
+    timed call loads the stored plan."""
     shape = spd.make_shape(w.batch, w.num_q_heads, w.num_kv_heads, w.head_dim, w.dtype, w.sm_scale)
     ws = spd.alloc_workspace(shape)
     out = torch.empty((w.batch, w.num_q_heads, w.head_dim), dtype=torch.float32, device=w.q.device)
+    mode = None
+    if plan == "reuse":
+        spd.spd_decode_step(shape, w.q, w.priv, w.pub, out, ws, fused=fused, plan=spd.SPD_PLAN_STORE)
+        mode = spd.SPD_PLAN_REUSE
+
+    def step():
+        spd.spd_decode_step(shape, w.q, w.priv, w.pub, out, ws, fused=fused, plan=mode)
     for _ in range(warmup):
-        spd.spd_decode_step(shape, w.q, w.priv, w.pub, out, ws, fused=fused)
+        step()
     torch.cuda.synchronize()
-    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     n0 = spd.spd_kernel_launch_count()
-    e0.record()
-    for _ in range(steps):
-        spd.spd_decode_step(shape, w.q, w.priv, w.pub, out, ws, fused=fused)
-    e1.record()
-    torch.cuda.synchronize()
+    per_step, total = [], 0.0
+    while total < min_seconds * 1e3 and len(per_step) < max_repeats:
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        for _ in range(steps):
+            step()
+        e1.record()
+        e1.synchronize()
+        ms = e0.elapsed_time(e1)
+        per_step.append(ms / steps)
+        total += ms
     launches = spd.spd_kernel_launch_count() - n0
     code, bad = spd.spd_query_device_status(ws)
     if code != spd.SPD_OK or not bool(torch.isfinite(out).all()):
         raise RuntimeError(f"decode step failed: status {code}, first bad user {bad}")
-    return e0.elapsed_time(e1) / steps, launches, shape, ws, out
+    timing = {"repeats": len(per_step), "steps_per_repeat": steps, "median_ms_per_step": float(np.median(per_step)),
+              "best_ms_per_step": float(np.min(per_step)), "worst_ms_per_step": float(np.max(per_step)),
+              "gpu_seconds": total / 1e3}
+    return timing["median_ms_per_step"], launches, shape, ws, out, timing
 
 
 def kernel_split(spd, w, shape, ws, out, steps):
     """Average device time of the attention kernel alone, events recorded inside the library."""
-    steps = min(steps, 2000)
+    steps = max(1, min(steps, 2000))
     spd.spd_profile_begin(steps)
     for _ in range(steps):
         spd.spd_decode_step(shape, w.q, w.priv, w.pub, out, ws, fused=True)
@@ -445,17 +493,17 @@ def time_token_step(spd, w, shape, ws, n_layers=8, replays=4):
         return e0.elapsed_time(e1) / n * 1e3
 
     with torch.cuda.stream(sa):
-        eager = timed(lambda: spd.spd_token_step(shape, layers, ws, stream=sa), replays)
+        eager = timed(lambda: spd.spd_token_step(shape, layers, ws, stream=sa, same_lengths=True), replays)
         graph = torch.cuda.CUDAGraph()
         with torch.cuda.graph(graph, stream=sa):
-            spd.spd_token_step(shape, layers, ws, stream=sa)
+            spd.spd_token_step(shape, layers, ws, stream=sa, same_lengths=True)
         replay = timed(graph.replay, replays)
     code, bad = spd.spd_query_device_status(ws, stream=sa)
     if code != spd.SPD_OK:
         raise RuntimeError(f"token step failed: status {code}, user {bad}")
     kv = sum(int(p[3].seq_lens.sum()) + int(p[4].seq_lens.sum()) for p in layers) * 2 * w.num_kv_heads * w.head_dim * w.elem_size
     return {"layers": n_layers, "eager_us": eager, "graph_us": replay, "kernels_per_step": 2 * n_layers,
-            "kv_gbs_graph": kv / replay / 1e3}
+            "kv_gbs_graph": kv / replay / 1e3, "plan": "derived by layer 0, loaded by the other layers"}
 
 
 PAPER_SCALE = dict(batch=8, hq=32, hkv=8, d=128, dtype="bf16", lin=("const", 512), lout=("uniform", 1, 128), seed=11)
@@ -484,10 +532,19 @@ def time_paper_scale(spd, dev, steps=300):
 
     res = {"workload": "8 users, 512-token prompts, 1-128 generated tokens, 32/8 heads, D 128, bf16",
            "decode_step_us": timed(lambda: spd.spd_decode_step(shape, w.q, w.priv, w.pub, out, ws, fused=True), steps)}
+    spd.spd_decode_step(shape, w.q, w.priv, w.pub, out, ws, fused=True, plan=spd.SPD_PLAN_STORE)
+    res["decode_step_plan_cached_us"] = timed(
+        lambda: spd.spd_decode_step(shape, w.q, w.priv, w.pub, out, ws, fused=True, plan=spd.SPD_PLAN_REUSE), steps)
     one = wl.make_workload(dict(PAPER_SCALE, name="one_user", batch=1), device=dev)
     shape1 = spd.make_shape(1, w.num_q_heads, w.num_kv_heads, w.head_dim, w.dtype, w.sm_scale)
     ws1, part1 = spd.alloc_workspace(shape1, dev), spd.alloc_partial(shape1)
     res["per_user_partial_us"] = timed(lambda: spd.spd_partial_attn(shape1, one.q, one.priv, part1, ws1), steps)
+    spd.spd_partial_attn(shape1, one.q, one.priv, part1, ws1, plan=spd.SPD_PLAN_STORE)
+    res["per_user_partial_plan_cached_us"] = timed(
+        lambda: spd.spd_partial_attn(shape1, one.q, one.priv, part1, ws1, plan=spd.SPD_PLAN_REUSE), steps)
+    ts = time_token_step(spd, w, shape, ws, n_layers=8, replays=4)
+    if ts is not None:
+        res["token_step_8_layers"] = dict(ts, per_layer_graph_us=ts["graph_us"] / ts["layers"])
     case = dict(users=8, prompt_lo=512, prompt_hi=512, hq=32, hkv=8, d=128, seed=11)
     res["prefill_us"] = time_prefill(spd, dev, steps=20, case=case)["ms"] * 1e3
     for x in (ws, ws1):
@@ -495,6 +552,59 @@ def time_paper_scale(spd, dev, steps=300):
         if code != spd.SPD_OK:
             raise RuntimeError(f"paper-scale run failed: status {code}, user {bad}")
     return res
+
+
+def make_gpu_workload(cfg, dev, users=None):
+    """The named workload on `dev`; with `users`, its first users only (for profiler captures that must stay small)."""
+    if users is None or users >= wl.CONFIGS[cfg]["batch"]:
+        return wl.make_workload(cfg, device=dev)
+    lin, lout = wl.make_lengths(wl.CONFIGS[cfg])
+    return wl.make_workload(dict(wl.CONFIGS[cfg], name=cfg, batch=users), lengths=(lin[:users], lout[:users]), device=dev)
+
+
+def roofline_block(kvb, attn_ms, cfg, users):
+    peak, peak_src = measured_peak()
+    achieved = kvb / attn_ms / 1e6
+    traffic = TRAFFIC_BYTES.get(cfg) if users is None else None
+    return {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
+            "traffic": traffic, "kernel": "attn_kernel", "peak_source": peak_src, "kernel_ms": attn_ms,
+            "algorithmic_bytes": kvb, "frac_of_nominal_8000": achieved / NOMINAL_HBM_GBS,
+            "timing": "separate pass, CUDA events around each kernel on the launch stream"}
+
+
+def measure_config(spd, cfg, dev, steps, warmup, local_rank, users=None, seconds=MIN_GPU_SECONDS, extras=True):
+    """One configuration measured on its own: the fused step (median repeat of a >= `seconds` region, clocks
+    sampled meanwhile), the attention kernel alone against the roofline, and -- with extras -- the step through
+    host buffers, the chained step, the step on a stored plan and the step with the measured rates ignored."""
+    w = make_gpu_workload(cfg, dev, users)
+    kvb = w.kv_bytes()
+    with ClockSampler(local_rank) as clocks:
+        ms, launches, shape, ws, out, timing = time_config(spd, w, steps, warmup, min_seconds=seconds)
+    res = {"workload": cfg, "users": w.batch, "kv_bytes_per_step": kvb, "ms_per_step": ms, "gbs": kvb / ms / 1e6,
+           "best_gbs": kvb / timing["best_ms_per_step"] / 1e6, "timing": timing, "clocks": clocks.summary(),
+           "user_tokens_per_s": w.batch / ms * 1e3, "pct_of_nominal_hbm_8000": 100.0 * kvb / ms / 1e6 / NOMINAL_HBM_GBS,
+           "pct_of_measured_hbm": 100.0 * kvb / ms / 1e6 / measured_peak()[0], "gpu_launches": launches}
+    split = kernel_split(spd, w, shape, ws, out, min(2000, max(steps, int(seconds * 1e3 / ms))))
+    res["roofline"] = roofline_block(kvb, split["attn_ms"], cfg, users)
+    res["sm_moves"] = dict(zip(("launches_compared", "ctas_on_another_sm"), spd.spd_debug_sm_moves(ws)))
+    if extras:
+        e2e_ms, h2d, d2h, outh = time_e2e(spd, w, shape, ws, min(500, max(steps, int(0.3 * seconds * 1e3 / ms))), warmup)
+        if not torch.allclose(outh, out.cpu(), atol=2e-3, rtol=0):   # share sizes adapt, so rounding order may differ
+            raise RuntimeError("host-buffer path and device path disagree")
+        res["e2e"] = {"value": kvb / e2e_ms / 1e6, "unit": "GB/s", "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
+                      "ms_per_step": e2e_ms, "call": "spd_decode_step_host"}
+        brief = 0.25 * seconds
+        m, *_ = time_config(spd, w, steps, warmup, fused=False, min_seconds=brief)
+        res["chained"] = {"ms_per_step": m, "gbs": kvb / m / 1e6}
+        m, *_ = time_config(spd, w, steps, warmup, plan="reuse", min_seconds=brief)
+        res["plan_cached"] = {"ms_per_step": m, "gbs": kvb / m / 1e6, "note": "every timed call loads the plan stored by one call before the region; the headline derives it inside every call (plan included)"}
+        spd.spd_set_split(0, True)
+        try:
+            m, *_ = time_config(spd, w, steps, warmup, min_seconds=brief)
+        finally:
+            spd.spd_set_split(0, False)
+        res["uniform_shares"] = {"ms_per_step": m, "gbs": kvb / m / 1e6, "note": "measured streaming rates ignored: what the rate-weighted shares are worth"}
+    return res, w
 
 
 def run_cuda(args):
@@ -505,13 +615,11 @@ def run_cuda(args):
     if world > 1:
         import torch.distributed as dist
         dist.init_process_group("nccl", device_id=dev)
-    steps = args.steps or 2000
+    steps = args.steps or 100
     warmup = args.warmup if args.warmup is not None else 20
     if warmup < 3:
         warmup = 3
     cfg = args.config
-    w = wl.make_workload(cfg, device=dev)     # every rank: its own replica of the same seeded workload
-    kvb = w.kv_bytes()
     spd.lib()
     spd.spd_set_bf16_math(1 if args.bf16_math == "fma" else 0)
     if args.prefill_only:
@@ -525,82 +633,78 @@ def run_cuda(args):
         torch.cuda.synchronize()
 
     barrier()
-    with ClockSampler(local_rank) as clocks:
-        ms, launches, shape, ws, out = time_config(spd, w, steps, warmup)
+    head, w = measure_config(spd, cfg, dev, steps, warmup, local_rank, users=args.users, extras=not args.kernel_only)
     barrier()
-    ms_max = max_over_ranks(ms, dev)
+    kvb = head["kv_bytes_per_step"]
+    ms_max = max_over_ranks(head["ms_per_step"], dev)     # every rank: its own replica of the same seeded workload
     value = replica_throughput(kvb, ms_max, world)
-
-    split = kernel_split(spd, w, shape, ws, out, steps)
-    e2e_ms, h2d, d2h, outh = time_e2e(spd, w, shape, ws, min(steps, 500), warmup)
-    if not torch.allclose(outh, out.cpu(), atol=2e-3, rtol=0):   # share sizes adapt, so rounding order may differ
-        raise RuntimeError("host-buffer path and device path disagree")
-    e2e_ms = max_over_ranks(e2e_ms, dev)
-    e2e_val = replica_throughput(kvb, e2e_ms, world)
-
+    e2e = head.get("e2e")
+    if e2e is not None:
+        e2e_ms = max_over_ranks(e2e["ms_per_step"], dev)
+        e2e = dict(e2e, value=replica_throughput(kvb, e2e_ms, world), ms_per_step=e2e_ms)
     if rank != 0:
         if world > 1:
             dist.destroy_process_group()
         return
-    peak, peak_src = measured_peak()
-    achieved = kvb / split["attn_ms"] / 1e6
+    peak = measured_peak()[0]
     line = {
         "metric": METRIC, "value": value, "unit": "GB/s", "n_gpus": world, "steps": steps, "warmup": warmup,
         "ms_per_step": ms_max, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
         "dtype": "bf16" if w.dtype == torch.bfloat16 else "f32", "data": "synthetic",
-        "config": {"workload": cfg, "users": w.batch, "q_heads": w.num_q_heads, "kv_heads": w.num_kv_heads,
-                   "head_dim": w.head_dim, "page_size": w.page_size, "kv_bytes_per_step": kvb,
-                   "parallelism": "replicas only" if world > 1 else "single GPU", "call": "spd_decode_step(fused=1)", "bf16_math": args.bf16_math,
-                   "l2": ("inputs larger than L2 (KV bytes per step >> 126 MB); no flush" if w.kv_bytes() > 4 * 126e6 else
-                          "inputs FIT in L2 and are not flushed: a latency figure, not comparable with the HBM roofline")},
+        "config": workload_config(cfg, w, w.batch, world, args, kv_bytes_per_step=kvb,
+                                  l2=("inputs larger than L2 (KV bytes per step >> 126 MB); no flush" if kvb > 4 * 126e6 else
+                                      "inputs FIT in L2 and are not flushed: a latency figure, not comparable with the HBM roofline"),
+                                  timed_region=f"{steps} back-to-back steps between two CUDA events, repeated {head['timing']['repeats']} "
+                                               f"times ({head['timing']['gpu_seconds']:.2f} s of GPU time); value = median repeat"),
+        "timing": head["timing"], "best_repeat_gbs": head["best_gbs"] * world,
         "user_tokens_per_s": world * w.batch / ms_max * 1e3,
         "pct_of_nominal_hbm_8000": 100.0 * value / world / NOMINAL_HBM_GBS,
         "pct_of_measured_hbm": 100.0 * value / world / peak,
-        "e2e": {"value": e2e_val, "unit": "GB/s", "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
-                "ms_per_step": e2e_ms, "call": "spd_decode_step_host"},
-        "gpu_launches": launches,
-        "roofline": {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
-                     "traffic": TRAFFIC_BYTES.get(cfg), "kernel": "attn_kernel", "peak_source": peak_src,
-                     "kernel_ms": split, "timing": "separate pass, CUDA events around each kernel on the launch stream"},
-        "clocks": clocks.summary(),
+        "e2e": e2e, "gpu_launches": head["gpu_launches"], "roofline": head["roofline"], "clocks": head["clocks"],
+        "sm_moves": head["sm_moves"],
     }
-    if world == 1 and not args.no_extras:
-        others = {}
-        for name in OTHER_CONFIGS:
-            if name == cfg:
-                continue
-            del w
-            torch.cuda.empty_cache()
-            w = wl.make_workload(name, device=dev)
-            n = max(50, min(steps, int(300.0 / 1.0)))
-            o = {}
-            for fused in (True, False):
-                m, _, sh, wsx, ox = time_config(spd, w, n, 5, fused=fused)
-                o["fused" if fused else "chained"] = {"ms_per_step": m, "gbs": w.kv_bytes() / m / 1e6}
-            sp = kernel_split(spd, w, sh, wsx, ox, n)
-            o["attn_kernel_gbs"] = w.kv_bytes() / sp["attn_ms"] / 1e6
-            o["pct_of_nominal_hbm_8000"] = 100.0 * o["fused"]["gbs"] / NOMINAL_HBM_GBS
-            o["kv_bytes_per_step"] = w.kv_bytes()
-            others[name] = o
-        line["other_configs"] = others
+    for k in ("chained", "plan_cached", "uniform_shares"):
+        if k in head:
+            line[k] = head[k]
+    if world == 1 and not args.no_extras and not args.kernel_only and args.users is None:
         del w
         torch.cuda.empty_cache()
-        w = wl.make_workload(cfg, device=dev)
+        co = CO_HEADLINE.get(cfg)
+        if co:
+            line["co_headline"], w = measure_config(spd, co, dev, steps, warmup, local_rank)
+            del w
+            torch.cuda.empty_cache()
+        others = {}
+        for name in BRIEF_CONFIGS:
+            if name in (cfg, co):
+                continue
+            others[name], w = measure_config(spd, name, dev, steps, warmup, local_rank, seconds=0.4)
+            if name != "c2_llama2_7b":
+                del w
+                torch.cuda.empty_cache()
+        line["other_configs"] = others
+        # the studies around the path run on the Llama-2-7B-shaped layer (the smallest bf16 configuration)
+        if "c2_llama2_7b" not in others:
+            w = wl.make_workload("c2_llama2_7b", device=dev)
+        shape2 = spd.make_shape(w.batch, w.num_q_heads, w.num_kv_heads, w.head_dim, w.dtype, w.sm_scale)
+        ws2 = spd.alloc_workspace(shape2)
         line["prefill"] = time_prefill(spd, dev)
-        line["schedules"] = time_schedules(spd, w, spd.make_shape(w.batch, w.num_q_heads, w.num_kv_heads, w.head_dim, w.dtype, w.sm_scale))
-        line["append_kv"] = time_append(spd, w, spd.make_shape(w.batch, w.num_q_heads, w.num_kv_heads, w.head_dim, w.dtype, w.sm_scale), ws)
+        line["schedules"] = dict(time_schedules(spd, w, shape2), workload="c2_llama2_7b")
+        line["append_kv"] = time_append(spd, w, shape2, ws2)
         line["paper_scale"] = time_paper_scale(spd, dev)
-        line["token_step"] = time_token_step(spd, w, spd.make_shape(w.batch, w.num_q_heads, w.num_kv_heads, w.head_dim, w.dtype, w.sm_scale), ws)
-        w = wl.make_workload(cfg, device="cpu")
-        line["cpu_baseline"] = cpu_baseline(w)
+        line["token_step"] = time_token_step(spd, w, shape2, ws2)
+        del w
+        torch.cuda.empty_cache()
+        w_cpu, full_batch = sample_workload_cpu(cfg)
+        line["cpu_baseline"] = cpu_baseline(w_cpu, full_batch)
     print(json.dumps(line), flush=True)
     if world > 1:
         dist.destroy_process_group()
 
 
 # DRAM traffic (dram__bytes_read.sum + dram__bytes_write.sum) of one attn_kernel launch, from the ncu
-# capture summarised under profiles/; configs without a capture of the current kernel report None.
-TRAFFIC_BYTES = {"c2_llama2_7b": 1341912320}
+# captures summarised under profiles/; configs without a capture of the current kernel report None.
+TRAFFIC_BYTES = {}
 
 
 def main():
@@ -608,7 +712,11 @@ def main():
     ap.add_argument("--gpus", type=int, default=1)
     ap.add_argument("--steps", type=int, default=None)
     ap.add_argument("--warmup", type=int, default=None)
-    ap.add_argument("--config", default="c2_llama2_7b", choices=list(wl.CONFIGS))
+    ap.add_argument("--config", default="c5_many_user", choices=list(wl.CONFIGS))
+    ap.add_argument("--users", type=int, default=None,
+                    help="only the first N users of the config (for profiler captures that must hold little memory)")
+    ap.add_argument("--kernel-only", action="store_true",
+                    help="only the fused step and the kernel-alone pass of the chosen config (for profiler captures)")
     ap.add_argument("--impl", default="cuda", choices=["cuda", "reference"])
     ap.add_argument("--no-extras", action="store_true", help="skip the other configs and the CPU baseline")
     ap.add_argument("--prefill-only", action="store_true", help="run only the prefill measurement (for profiling)")

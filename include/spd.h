@@ -26,6 +26,21 @@
  *     call (or process) to another as is.  An empty partition gives O = 0, m = -inf, l = 0.
  *   - Supported: head_dim 64 or 128, page_size 16, dtype F32 or BF16 (q and KV alike),
  *     num_q_heads a multiple of num_kv_heads with a group size of 1, 2, 4, 8 or a multiple of 8.
+ *   - Stream order.  The attention kernel is launched with programmatic stream serialisation: the part of it
+ *     that only READS the lengths, the page tables and the KV pools may start while the previous kernel on the
+ *     stream is still finishing; q, an incoming partial, the workspace and the outputs are touched only after
+ *     that kernel has completed.  If a kernel of yours on the same stream writes lengths, page tables or KV rows
+ *     immediately before a call, launch in plain stream order: spd_set_programmatic_launch(0), or SPD_NO_PDL=1
+ *     in the environment.  The library's own append is followed by a plain-order launch inside spd_token_step.
+ *   - Threads.  Calls may come from several host threads; calls that share a workspace must be ordered by the
+ *     caller (one stream at a time per workspace).  Each workspace keeps a small table of streaming rates that
+ *     sizes the next call's shares; it is rotated by a per-workspace launch count held on the host, so calls on
+ *     other workspaces or streams never disturb it.
+ *   - CUDA graphs.  Every call may be captured.  What is decided on the host at call time is then frozen into
+ *     the graph: the call id (a user flagged in one replay stays flagged in later replays until the workspace's
+ *     flags are cleared by spd_query_device_status), which third of the rate table a launch reads and writes
+ *     (replays keep rotating correctly among the launches of one graph; shares keep following the rates that
+ *     those launches leave), and the plan mode of the *_planned calls.
  */
 #ifndef SPD_H_
 #define SPD_H_
@@ -44,7 +59,8 @@ typedef enum {
     SPD_ERR_WORKSPACE = 3,     /* workspace smaller than spd_workspace_size() reports          */
     SPD_ERR_BAD_PAGE = 4,      /* device saw a page index or length out of range (sticky flag) */
     SPD_ERR_CUDA = 5,          /* a CUDA runtime or driver call failed                         */
-    SPD_ERR_TIMEOUT = 6        /* a bounded wait inside a kernel ran out (sticky flag)         */
+    SPD_ERR_TIMEOUT = 6,       /* a bounded wait inside a kernel ran out (sticky flag)         */
+    SPD_ERR_PLAN = 7           /* a call told to reuse a stored plan found none that fits (sticky flag) */
 } spd_status;
 
 typedef enum { SPD_F32 = 0, SPD_BF16 = 1 } spd_dtype;
@@ -127,6 +143,31 @@ spd_status spd_decode_step(const spd_shape *shape, const void *q, const spd_page
                            void *ws, size_t ws_bytes, void *cuda_stream);
 
 /*
+ * The same three calls with the plan under the caller's control (the paper has no counterpart; the plan -- tiles
+ * per user, their prefix sums, the share of the tile stream that each warp owns -- depends only on the two
+ * seq_lens arrays, the shape and the GPU):
+ *   SPD_PLAN_PER_CALL : derive the plan inside the kernel (what the plain calls do);
+ *   SPD_PLAN_STORE    : derive it and leave it in the workspace;
+ *   SPD_PLAN_REUSE    : load what the last SPD_PLAN_STORE call of the same kind (private only, public only, both
+ *                       partitions) on this workspace and stream left, instead of deriving it.  The caller
+ *                       states thereby that shape and every length are what they were at that call (page tables,
+ *                       pools, q may differ).  A plan that was never stored, or was stored for another shape,
+ *                       raises SPD_ERR_PLAN and the call writes nothing; lengths that changed silently give
+ *                       wrong results for the users concerned (never a fault: every index is still checked).
+ * Reuse pays for small calls, where deriving the plan is most of the time; large calls hide it anyway.
+ */
+typedef enum { SPD_PLAN_PER_CALL = 0, SPD_PLAN_STORE = 1, SPD_PLAN_REUSE = 2 } spd_plan_mode;
+spd_status spd_partial_attn_planned(const spd_shape *shape, const void *q, const spd_paged_kv *priv,
+                                    spd_partial out, spd_plan_mode plan, void *ws, size_t ws_bytes,
+                                    void *cuda_stream);
+spd_status spd_service_attn_merge_planned(const spd_shape *shape, const void *q, const spd_paged_kv *pub,
+                                          spd_partial in, void *out, spd_dtype out_dtype, spd_plan_mode plan,
+                                          void *ws, size_t ws_bytes, void *cuda_stream);
+spd_status spd_decode_step_planned(const spd_shape *shape, const void *q, const spd_paged_kv *priv,
+                                   const spd_paged_kv *pub, void *out, spd_dtype out_dtype, int32_t fused,
+                                   spd_plan_mode plan, void *ws, size_t ws_bytes, void *cuda_stream);
+
+/*
  * Input-attention monitor (Sec. 2.4.4 and Sec. 7.1.1: watching how much attention the query pays to
  * the user's original instruction, inside the per-user process, to notice an instruction injected by
  * the service).  For every user, tokens [tok_lo[u], tok_hi[u]) of the PRIVATE partition are watched
@@ -199,9 +240,12 @@ spd_status spd_append_kv(const spd_shape *shape, const void *k_new, const void *
  * its own output.  In a model q of layer i+1 depends on layer i's output through the weights; those are
  * not this library's, so all inputs are taken as given and the driver only fixes the order and the launch
  * structure: 2 * num_layers kernels on `cuda_stream`, nothing else, so that a caller can capture the whole
- * token step in one CUDA graph and replay it (what the call id and the share table do under replay is
- * described with spd_decode_step).  The workspace is shared by the layers.  Stops at the first host-side
- * error; device-side mistakes are reported through spd_query_device_status as for the single calls.
+ * token step in one CUDA graph and replay it (what is frozen into a graph is listed under "CUDA graphs" at the
+ * top of this file).  The workspace is shared by the layers.  same_lengths != 0 states that every layer's
+ * private and public seq_lens hold the same values as layer 0's (as in a model, whose layers all cache the same
+ * tokens): the plan is then derived once, by layer 0, and loaded by the other layers (SPD_PLAN_STORE /
+ * SPD_PLAN_REUSE above).  Stops at the first host-side error; device-side mistakes are reported through
+ * spd_query_device_status as for the single calls.
  */
 typedef struct {
     const void *q;             /* [batch][num_q_heads][head_dim]                                  */
@@ -211,7 +255,8 @@ typedef struct {
     void *out;                 /* [batch][num_q_heads][head_dim] in out_dtype                     */
 } spd_layer;
 spd_status spd_token_step(const spd_shape *shape, int32_t num_layers, const spd_layer *layers,
-                          spd_dtype out_dtype, void *ws, size_t ws_bytes, void *cuda_stream);
+                          spd_dtype out_dtype, int32_t same_lengths, void *ws, size_t ws_bytes,
+                          void *cuda_stream);
 
 /*
  * spd_decode_step (fused) for a caller whose per-step data lives in HOST memory (no counterpart in
@@ -249,8 +294,9 @@ spd_status spd_decode_step_host(const spd_shape *shape, const spd_step_blob *lay
 
 /*
  * Waits for `cuda_stream`, then reads and clears the workspace's sticky status.  Returns SPD_OK,
- * SPD_ERR_BAD_PAGE or SPD_ERR_TIMEOUT; *first_bad_user (may be NULL) receives the lowest user
- * index that was flagged, or -1.
+ * SPD_ERR_BAD_PAGE, SPD_ERR_TIMEOUT or SPD_ERR_PLAN; *first_bad_user (may be NULL) receives the lowest user
+ * index that was flagged, or -1.  After a status other than SPD_OK the per-user flags and the merge tickets of
+ * the workspace are cleared too, so the next call starts clean.
  */
 spd_status spd_query_device_status(void *ws, void *cuda_stream, int32_t *first_bad_user);
 
@@ -284,9 +330,11 @@ spd_status spd_profile_end(int32_t *calls, double *kernel_ms);
  *     batch * num_q_heads <= 13000 at head_dim 128.
  *   - The first call on each device looks up the array's device address (with that device current).
  *     Make that first call outside any stream capture.
- *   - All calls share the one array, and it keeps what the previous call left.  The call itself
- *     clears the words that must start at zero (the sticky status and the per-user flags), so a
- *     flag raised by an earlier call never leaks into this one.  Two calls that overlap on the GPU
+ *   - All calls share the one array, and it keeps what the previous call left, laid out for the
+ *     previous call's shape.  The call itself clears what must start at zero (the sticky status, the
+ *     per-user flags and the merge tickets), so neither a flag raised by an earlier call nor tickets
+ *     that an earlier call left drawn (a call that timed out, or one of another shape whose scratch lay
+ *     where this call's tickets lie) leak into this one.  Two calls that overlap on the GPU
  *     (different streams, or different host threads without ordering) race on the array: order them.
  *   - The call allocates and frees nothing, on the device or through any library.
  *   - wait_and_check = 0: returns once the work is enqueued.  Non-zero: waits for the stream and
@@ -312,6 +360,36 @@ spd_status spd_set_bf16_math(int32_t path);
  * thing within tolerance.
  */
 spd_status spd_set_prefill_rows(int32_t rows);
+
+/*
+ * Test and tuning aid (no counterpart in the paper): how the tile stream is cut into shares from now on,
+ * process-wide.  min_tiles_per_share: fewest page tiles (16 tokens each) a share may hold; 0 restores the default
+ * (4); 1 lets every page become a piece of its own when the batch is small enough; a value at or above the
+ * batch's tile count leaves one share, hence no second-level merge at all.  uniform_shares = 1 gives every CTA the
+ * same weight and ignores the measured streaming rates: the cut points then depend on the lengths alone, and a
+ * call repeated on the same inputs gives bit-identical results.
+ */
+spd_status spd_set_split(int32_t min_tiles_per_share, int32_t uniform_shares);
+
+/*
+ * Process-wide switch for programmatic stream serialisation of the attention kernel (see "Stream order" at the
+ * top): 1 = on (default unless SPD_NO_PDL is set in the environment), 0 = plain stream order.
+ */
+spd_status spd_set_programmatic_launch(int32_t on);
+
+/*
+ * Debugging aids (no counterpart in the paper).  Both wait for `cuda_stream`.
+ *   spd_debug_read_plan : the plan of the last call of kind `which` (0 = private partition only, 1 = public only,
+ *     2 = both) on this workspace that derived its plan: *tiles = page tiles in the stream, *shares = warps that own a
+ *     share, bnd[w] = first tile of share w for w in [0, *shares] (bnd[*shares] = *tiles); at most bnd_capacity
+ *     entries are written.  Any of the three outputs may be NULL.
+ *   spd_debug_sm_moves  : the rate table is indexed by CTA while the rates belong to SMs; *launches counts the
+ *     attention launches on this workspace that could compare, *moves the CTAs among them that ran on another SM
+ *     than the same CTA index did one launch earlier.
+ */
+spd_status spd_debug_read_plan(void *ws, int32_t which, void *cuda_stream, int32_t *tiles, int32_t *shares,
+                               int32_t *bnd, int32_t bnd_capacity);
+spd_status spd_debug_sm_moves(void *ws, void *cuda_stream, int64_t *launches, int64_t *moves);
 
 /* Static text for a status code. */
 const char *spd_status_string(spd_status status);

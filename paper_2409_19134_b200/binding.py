@@ -15,15 +15,19 @@ from .build import LIB_PATH
 
 SPD_OK = 0
 SPD_F32, SPD_BF16 = 0, 1
+SPD_PLAN_PER_CALL, SPD_PLAN_STORE, SPD_PLAN_REUSE = 0, 1, 2
 _STATUS_NAMES = {0: "SPD_OK", 1: "SPD_ERR_INVALID_ARG", 2: "SPD_ERR_UNSUPPORTED", 3: "SPD_ERR_WORKSPACE",
-                 4: "SPD_ERR_BAD_PAGE", 5: "SPD_ERR_CUDA", 6: "SPD_ERR_TIMEOUT"}
+                 4: "SPD_ERR_BAD_PAGE", 5: "SPD_ERR_CUDA", 6: "SPD_ERR_TIMEOUT", 7: "SPD_ERR_PLAN"}
+_DEVICE_CODES = (SPD_OK, 4, 6, 7)     # what a call that waits for the device may report without raising
 
 EXPORTS = ["spd_workspace_size", "spd_partial_attn", "spd_service_attn_merge", "spd_decode_step",
            "spd_step_blob_layout", "spd_decode_step_host", "spd_query_device_status",
            "spd_kernel_launch_count", "spd_status_string", "spd_profile_begin", "spd_profile_end",
            "spd_decode_step_static", "spd_append_kv",
            "spd_partial_attn_watch", "spd_decode_step_watch", "spd_set_bf16_math", "spd_merge_partials", "spd_prefill_attn",
-           "spd_set_prefill_rows", "spd_token_step"]
+           "spd_set_prefill_rows", "spd_token_step", "spd_partial_attn_planned", "spd_service_attn_merge_planned",
+           "spd_decode_step_planned", "spd_set_split", "spd_set_programmatic_launch", "spd_debug_read_plan",
+           "spd_debug_sm_moves"]
 
 
 class SpdError(RuntimeError):
@@ -94,7 +98,17 @@ def lib() -> C.CDLL:
                                             C.POINTER(Watch), vp, sz, vp]
         L.spd_set_bf16_math.argtypes = [C.c_int32]
         L.spd_set_prefill_rows.argtypes = [C.c_int32]
-        L.spd_token_step.argtypes = [C.POINTER(Shape), C.c_int32, C.POINTER(Layer), C.c_int, vp, sz, vp]
+        L.spd_token_step.argtypes = [C.POINTER(Shape), C.c_int32, C.POINTER(Layer), C.c_int, C.c_int32, vp, sz, vp]
+        L.spd_partial_attn_planned.argtypes = [C.POINTER(Shape), vp, C.POINTER(PagedKV), Partial, C.c_int, vp, sz, vp]
+        L.spd_service_attn_merge_planned.argtypes = [C.POINTER(Shape), vp, C.POINTER(PagedKV), Partial, vp, C.c_int, C.c_int,
+                                                     vp, sz, vp]
+        L.spd_decode_step_planned.argtypes = [C.POINTER(Shape), vp, C.POINTER(PagedKV), C.POINTER(PagedKV), vp, C.c_int,
+                                              C.c_int32, C.c_int, vp, sz, vp]
+        L.spd_set_split.argtypes = [C.c_int32, C.c_int32]
+        L.spd_set_programmatic_launch.argtypes = [C.c_int32]
+        L.spd_debug_read_plan.argtypes = [vp, C.c_int32, vp, C.POINTER(C.c_int32), C.POINTER(C.c_int32),
+                                          C.POINTER(C.c_int32), C.c_int32]
+        L.spd_debug_sm_moves.argtypes = [vp, vp, C.POINTER(C.c_int64), C.POINTER(C.c_int64)]
         L.spd_merge_partials.argtypes = [C.POINTER(Shape), C.c_int32, C.POINTER(Partial), vp, C.c_int, vp]
         L.spd_prefill_attn.argtypes = [C.POINTER(Shape), C.c_int64, vp, vp, vp, vp, vp, vp, C.c_int32, vp, vp, vp, vp,
                                        C.c_int, vp, sz, vp]
@@ -163,26 +177,41 @@ def alloc_partial(shape: Shape, device="cuda") -> Tuple[torch.Tensor, torch.Tens
             torch.empty((B, H), dtype=torch.float32, device=device))
 
 
-def spd_partial_attn(shape, q, priv, out, ws, stream=None) -> None:
+def spd_partial_attn(shape, q, priv, out, ws, stream=None, plan=None) -> None:
+    """plan=None calls spd_partial_attn; SPD_PLAN_* calls spd_partial_attn_planned with that mode."""
     kv = paged_kv(priv)
     part = Partial(out[0].data_ptr(), out[1].data_ptr(), out[2].data_ptr())
-    _check(lib().spd_partial_attn(C.byref(shape), q.data_ptr(), C.byref(kv), part, ws.data_ptr(), ws.numel(),
-                                  _stream_ptr(stream)), "spd_partial_attn")
+    if plan is None:
+        _check(lib().spd_partial_attn(C.byref(shape), q.data_ptr(), C.byref(kv), part, ws.data_ptr(), ws.numel(),
+                                      _stream_ptr(stream)), "spd_partial_attn")
+    else:
+        _check(lib().spd_partial_attn_planned(C.byref(shape), q.data_ptr(), C.byref(kv), part, int(plan), ws.data_ptr(),
+                                              ws.numel(), _stream_ptr(stream)), "spd_partial_attn_planned")
 
 
-def spd_service_attn_merge(shape, q, pub, partial_in, out, ws, stream=None) -> None:
+def spd_service_attn_merge(shape, q, pub, partial_in, out, ws, stream=None, plan=None) -> None:
     kv = paged_kv(pub)
     part = Partial(partial_in[0].data_ptr(), partial_in[1].data_ptr(), partial_in[2].data_ptr())
-    _check(lib().spd_service_attn_merge(C.byref(shape), q.data_ptr(), C.byref(kv), part, out.data_ptr(),
-                                        _dtype_code(out.dtype), ws.data_ptr(), ws.numel(), _stream_ptr(stream)),
-           "spd_service_attn_merge")
+    if plan is None:
+        _check(lib().spd_service_attn_merge(C.byref(shape), q.data_ptr(), C.byref(kv), part, out.data_ptr(),
+                                            _dtype_code(out.dtype), ws.data_ptr(), ws.numel(), _stream_ptr(stream)),
+               "spd_service_attn_merge")
+    else:
+        _check(lib().spd_service_attn_merge_planned(C.byref(shape), q.data_ptr(), C.byref(kv), part, out.data_ptr(),
+                                                    _dtype_code(out.dtype), int(plan), ws.data_ptr(), ws.numel(),
+                                                    _stream_ptr(stream)), "spd_service_attn_merge_planned")
 
 
-def spd_decode_step(shape, q, priv, pub, out, ws, fused=True, stream=None) -> None:
+def spd_decode_step(shape, q, priv, pub, out, ws, fused=True, stream=None, plan=None) -> None:
     a, b = paged_kv(priv), paged_kv(pub)
-    _check(lib().spd_decode_step(C.byref(shape), q.data_ptr(), C.byref(a), C.byref(b), out.data_ptr(),
-                                 _dtype_code(out.dtype), 1 if fused else 0, ws.data_ptr(), ws.numel(),
-                                 _stream_ptr(stream)), "spd_decode_step")
+    if plan is None:
+        _check(lib().spd_decode_step(C.byref(shape), q.data_ptr(), C.byref(a), C.byref(b), out.data_ptr(),
+                                     _dtype_code(out.dtype), 1 if fused else 0, ws.data_ptr(), ws.numel(),
+                                     _stream_ptr(stream)), "spd_decode_step")
+    else:
+        _check(lib().spd_decode_step_planned(C.byref(shape), q.data_ptr(), C.byref(a), C.byref(b), out.data_ptr(),
+                                             _dtype_code(out.dtype), 1 if fused else 0, int(plan), ws.data_ptr(),
+                                             ws.numel(), _stream_ptr(stream)), "spd_decode_step_planned")
 
 
 def spd_step_blob_layout(shape, priv_pages_listed: int, pub_pages_listed: int, out_dtype) -> StepBlob:
@@ -204,7 +233,7 @@ def spd_decode_step_host(shape, layout, host_blob, device_blob, priv_pools, pub_
     code = lib().spd_decode_step_host(C.byref(shape), C.byref(layout), host_blob.data_ptr(), device_blob.data_ptr(),
                                       C.byref(a), C.byref(b), _dtype_code(out_dtype), C.byref(bad), ws.data_ptr(),
                                       ws.numel(), _stream_ptr(stream))
-    if code not in (SPD_OK, 4, 6):
+    if code not in _DEVICE_CODES:
         raise SpdError(code, "spd_decode_step_host")
     return int(code), int(bad.value)
 
@@ -225,7 +254,7 @@ class HostStep:
 
     def __call__(self) -> Tuple[int, int]:
         code = self._fn(*self._args)
-        if code not in (SPD_OK, 4, 6):
+        if code not in _DEVICE_CODES:
             raise SpdError(code, "spd_decode_step_host")
         return int(code), int(self._bad.value)
 
@@ -279,7 +308,7 @@ def spd_decode_step_static(shape, q, priv, pub, out, wait_and_check=True, stream
     code = lib().spd_decode_step_static(C.byref(shape), q.data_ptr(), C.byref(a), C.byref(b), out.data_ptr(),
                                         _dtype_code(out.dtype), 1 if wait_and_check else 0, C.byref(bad),
                                         _stream_ptr(stream))
-    if code not in (SPD_OK, 4, 6):
+    if code not in _DEVICE_CODES:
         raise SpdError(code, "spd_decode_step_static")
     return int(code), int(bad.value)
 
@@ -293,14 +322,15 @@ def spd_append_kv(shape, k_new, v_new, part, ws, stream=None) -> None:
                                _stream_ptr(stream)), "spd_append_kv")
 
 
-def spd_token_step(shape, layers, ws, stream=None) -> None:
-    """layers: a sequence of (q, k_new, v_new, priv, pub, out) per layer; appends to each pub and runs each decode step."""
+def spd_token_step(shape, layers, ws, stream=None, same_lengths=False) -> None:
+    """layers: a sequence of (q, k_new, v_new, priv, pub, out) per layer; appends to each pub and runs each decode step.
+    same_lengths: every layer's lengths equal layer 0's, so its plan is derived once and reused."""
     arr = (Layer * len(layers))()
     for i, (q, k_new, v_new, priv, pub, out) in enumerate(layers):
         assert q.is_contiguous() and k_new.is_contiguous() and v_new.is_contiguous() and out.is_contiguous()
         arr[i] = Layer(q.data_ptr(), k_new.data_ptr(), v_new.data_ptr(), paged_kv(priv), paged_kv(pub), out.data_ptr())
-    _check(lib().spd_token_step(C.byref(shape), len(layers), arr, _dtype_code(layers[0][5].dtype), ws.data_ptr(),
-                                ws.numel(), _stream_ptr(stream)), "spd_token_step")
+    _check(lib().spd_token_step(C.byref(shape), len(layers), arr, _dtype_code(layers[0][5].dtype),
+                                1 if same_lengths else 0, ws.data_ptr(), ws.numel(), _stream_ptr(stream)), "spd_token_step")
 
 
 def _watch(tok_lo, tok_hi, out) -> Watch:
@@ -325,6 +355,33 @@ def spd_decode_step_watch(shape, q, priv, pub, out, tok_lo, tok_hi, watch_out, w
 def spd_set_bf16_math(path: int) -> None:
     """0 = tensor cores (default), 1 = FMA pipes (comparison arm); process-wide."""
     _check(lib().spd_set_bf16_math(int(path)), "spd_set_bf16_math")
+
+
+def spd_set_split(min_tiles_per_share: int = 0, uniform_shares: bool = False) -> None:
+    """How the tile stream is cut from now on, process-wide: fewest tiles per share (0 = default) and whether
+    every CTA weighs the same (the measured rates are ignored; results become repeatable bit for bit)."""
+    _check(lib().spd_set_split(int(min_tiles_per_share), 1 if uniform_shares else 0), "spd_set_split")
+
+
+def spd_set_programmatic_launch(on: bool) -> None:
+    _check(lib().spd_set_programmatic_launch(1 if on else 0), "spd_set_programmatic_launch")
+
+
+def spd_debug_read_plan(ws, which: int = 2, stream=None, capacity: int = 256 * 16 + 1):
+    """(tiles, shares, bnd) of the last derived plan of kind `which` (0 private only, 1 public only, 2 both)."""
+    T, A = C.c_int32(0), C.c_int32(0)
+    bnd = (C.c_int32 * capacity)()
+    _check(lib().spd_debug_read_plan(ws.data_ptr(), int(which), _stream_ptr(stream), C.byref(T), C.byref(A), bnd, capacity),
+           "spd_debug_read_plan")
+    n = min(capacity, A.value + 1)
+    return int(T.value), int(A.value), [int(bnd[i]) for i in range(n)]
+
+
+def spd_debug_sm_moves(ws, stream=None) -> Tuple[int, int]:
+    """(launches that could compare, CTAs that ran on another SM than the same CTA index one launch earlier)."""
+    a, b = C.c_int64(0), C.c_int64(0)
+    _check(lib().spd_debug_sm_moves(ws.data_ptr(), _stream_ptr(stream), C.byref(a), C.byref(b)), "spd_debug_sm_moves")
+    return int(a.value), int(b.value)
 
 
 def spd_set_prefill_rows(rows: int) -> None:

@@ -7,6 +7,7 @@
 #include <cstdlib>
 #include <cstring>
 #include <mutex>
+#include <unordered_map>
 #include <vector>
 
 #include "spd_kernels.cuh"
@@ -34,6 +35,28 @@ void prof_mark(int job, int k, cudaStream_t st) {
 std::atomic<uint32_t> g_epoch{0};
 std::atomic<int> g_bf16_math{0};   // 0 = tensor cores (default), 1 = FMA pipes (comparison arm)
 std::atomic<int> g_prefill_rows{0};   // query rows per prefill CTA: 0 = by mean prompt length, 128, 256
+std::atomic<int> g_min_tiles{kMinTilesPerWarp};   // fewest page tiles a share of the tile stream may hold
+std::atomic<int> g_uniform_shares{0};             // 1 = equal shares, the measured rates are ignored
+std::atomic<int> g_pdl{-1};                       // programmatic launch: -1 = not decided yet (environment), 0 off, 1 on
+
+// Attention launches made so far on each workspace (keyed by its address).  The kernel rotates through the three
+// thirds of the workspace's rate table by this count, so it must advance by exactly one per attention launch on
+// that workspace whatever else the process launches in between.
+uint32_t next_rate_sel(const void *ws) {
+    static std::mutex mu;
+    static std::unordered_map<const void *, uint32_t> count;
+    std::lock_guard<std::mutex> lock(mu);
+    return count[ws]++ % 3u;
+}
+
+bool programmatic_launch() {
+    int v = g_pdl.load();
+    if (v < 0) {
+        v = getenv("SPD_NO_PDL") == nullptr ? 1 : 0;
+        g_pdl.store(v);
+    }
+    return v != 0;
+}
 constexpr int64_t kPrefillPairFrom = 768;    // mean prompt length from which the 256-row kernel is used
 
 // Ids of calls: non-zero, so that a zeroed workspace matches none.
@@ -93,19 +116,38 @@ constexpr size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
 // Workspace layout.  The header, the per-user flags and the tickets come first so that the status
 // query can find them without knowing the shape.
 struct WsLayout {
-    size_t hdr, rates, bad, tickets, scratch, partial_o, partial_m, partial_l, total;
+    size_t hdr, rates, plan, bad, tickets, scratch, partial_o, partial_m, partial_l, total;
 };
+
+// The part of the layout that the status query must find from the header alone: it depends only on the batch
+// size and the number of sequences, which the kernels leave in the header.
+struct WsHead {
+    size_t hdr, rates, plan, bad, tickets, end;
+};
+
+constexpr size_t kPlanBytes = static_cast<size_t>(PLAN_WORDS) * 4;   // one stored plan
+constexpr int kPlanSlots = 3;                                        // private only, public only, both partitions
+
+WsHead ws_head(size_t batch, size_t seqs) {
+    WsHead H;
+    size_t off = 0;
+    H.hdr = off;       off = align_up(off + HDR_WORDS * 4, 256);
+    H.rates = off;     off = align_up(off + 3 * kMaxGrid * sizeof(float2), 256);
+    H.plan = off;      off = align_up(off + kPlanSlots * kPlanBytes, 256);
+    H.bad = off;       off = align_up(off + batch * 4, 256);
+    H.tickets = off;   off = align_up(off + seqs * 4, 256);
+    H.end = off;
+    return H;
+}
 
 WsLayout ws_layout(const spd_shape &s, int sms) {
     WsLayout L;
-    size_t off = 0;
     const size_t B = s.batch;
-    L.hdr = off;       off = align_up(off + HDR_WORDS * 4, 256);
-    L.rates = off;     off = align_up(off + 3 * kMaxGrid * sizeof(float2), 256);
-    L.bad = off;       off = align_up(off + B * 4, 256);
     const int g = s.num_q_heads / s.num_kv_heads;
     const size_t seqs = B * s.num_kv_heads * (g > kHeadsPerItem ? g / kHeadsPerItem : 1);
-    L.tickets = off;   off = align_up(off + seqs * 4, 256);
+    const WsHead H = ws_head(B, seqs);
+    L.hdr = H.hdr; L.rates = H.rates; L.plan = H.plan; L.bad = H.bad; L.tickets = H.tickets;
+    size_t off = H.end;
     constexpr int wmax = MathBF16<128>::kWarps > MathF32<128, 1>::kWarps ? MathBF16<128>::kWarps : MathF32<128, 1>::kWarps;
     const size_t max_warps = static_cast<size_t>(sms) * wmax;
     L.scratch = off;   off = align_up(off + 2 * max_warps * slot_floats(s.head_dim) * 4, 256);
@@ -162,7 +204,7 @@ spd_status make_map(CUtensorMap *map, const spd_shape &s, const void *pool, int6
 }
 
 template <class Math>
-spd_status launch_attn(const Params &p_in, const CUtensorMap *maps, int sms, cudaStream_t st) {
+spd_status launch_attn(const Params &p_in, const CUtensorMap *maps, int sms, cudaStream_t st, bool pdl) {
     if (sms > kMaxGrid) return SPD_ERR_UNSUPPORTED;
     Params p = p_in;
     p.num_warps = sms * Math::kWarps;   // the plan cuts the tile stream into one share per warp of THIS grid
@@ -176,10 +218,8 @@ spd_status launch_attn(const Params &p_in, const CUtensorMap *maps, int sms, cud
                                         static_cast<int>(smem));
     });
     if (attr_err != cudaSuccess) return SPD_ERR_CUDA;
-    // Programmatic stream serialisation: this kernel's read-only preamble may overlap the tail of the
-    // previous kernel on the stream if that kernel allows it (this library's kernels do).  Setting
-    // SPD_NO_PDL in the environment launches with plain stream order.
-    static const bool pdl = getenv("SPD_NO_PDL") == nullptr;
+    // Programmatic stream serialisation (pdl): this kernel's read-only preamble may overlap the tail of the
+    // previous kernel on the stream if that kernel allows it (the attention kernel does).
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3(sms);
     cfg.blockDim = dim3(Math::kWarps * 32);
@@ -208,7 +248,19 @@ struct Job {
     int32_t epoch;                 // id of the call (both halves of a chained step share one)
     int32_t *status_words;         // where the kernel raises its status; null = the workspace header
     const spd_watch *watch;        // optional monitor of a private token range
+    int plan_mode;                 // PlanMode: derive per call (default), derive and store, or load the stored plan
+    bool plain_order;              // launch in plain stream order (an input was written by the kernel just before)
 };
+
+// The stored plan of a call is tagged with what it was cut for besides the lengths, so that a launch told to load a
+// plan which was never stored (or stored for another shape) reports SPD_ERR_PLAN instead of using it.
+int32_t plan_tag_of(const spd_shape &s, int min_tiles, int uniform) {
+    uint32_t h = 0x9e3779b9u;
+    const int32_t v[] = {s.batch, s.num_q_heads, s.num_kv_heads, s.head_dim, static_cast<int32_t>(s.dtype), min_tiles, uniform};
+    for (int32_t x : v) h = (h ^ static_cast<uint32_t>(x)) * 0x01000193u + 0x7f4a7c15u;
+    h &= 0x7fffffffu;
+    return static_cast<int32_t>(h ? h : 1u);
+}
 
 spd_status run_job(const Job &job, void *ws, size_t ws_bytes, void *stream) {
     const spd_shape &s = *job.shape;
@@ -235,7 +287,14 @@ spd_status run_job(const Job &job, void *ws, size_t ws_bytes, void *stream) {
     p.bad = reinterpret_cast<int32_t *>(w + L.bad);
     p.tickets = reinterpret_cast<int32_t *>(w + L.tickets);
     p.rates = reinterpret_cast<float2 *>(w + L.rates);
-    p.rate_sel = static_cast<int32_t>(g_launches.load() % 3);   // launches rotate through the three thirds
+    p.rate_sel = static_cast<int32_t>(next_rate_sel(ws));       // this workspace's launches rotate through the three thirds
+    p.min_tiles = g_min_tiles.load();
+    p.uniform = g_uniform_shares.load();
+    const int slot = (job.part[0] ? 1 : 0) + (job.part[1] ? 2 : 0) - 1;   // one stored plan per kind of call
+    if (slot < 0) return SPD_ERR_INVALID_ARG;
+    p.plan = reinterpret_cast<int32_t *>(w + L.plan + slot * kPlanBytes);
+    p.plan_mode = job.plan_mode;
+    p.plan_tag = plan_tag_of(s, p.min_tiles, p.uniform);
     p.epoch = job.epoch;
     p.scratch = reinterpret_cast<float *>(w + L.scratch);
     p.mode = job.mode;
@@ -279,15 +338,16 @@ spd_status run_job(const Job &job, void *ws, size_t ws_bytes, void *stream) {
     }
     prof_mark(pj, 0, st);
     const int D = s.head_dim;
+    const bool pdl = programmatic_launch() && !job.plain_order;
     if (bf && g_bf16_math.load() == 1) {
-#define SPD_SIMT_CASE(DD, GG) if (D == DD && p.geff == GG) rc = launch_attn<MathBF16Simt<DD, GG>>(p, maps, di.sms, st);
+#define SPD_SIMT_CASE(DD, GG) if (D == DD && p.geff == GG) rc = launch_attn<MathBF16Simt<DD, GG>>(p, maps, di.sms, st, pdl);
         SPD_SIMT_CASE(64, 1) SPD_SIMT_CASE(64, 2) SPD_SIMT_CASE(64, 4) SPD_SIMT_CASE(64, 8)
         SPD_SIMT_CASE(128, 1) SPD_SIMT_CASE(128, 2) SPD_SIMT_CASE(128, 4) SPD_SIMT_CASE(128, 8)
 #undef SPD_SIMT_CASE
     } else if (bf) {
-        rc = D == 128 ? launch_attn<MathBF16<128>>(p, maps, di.sms, st) : launch_attn<MathBF16<64>>(p, maps, di.sms, st);
+        rc = D == 128 ? launch_attn<MathBF16<128>>(p, maps, di.sms, st, pdl) : launch_attn<MathBF16<64>>(p, maps, di.sms, st, pdl);
     } else {
-#define SPD_F32_CASE(DD, GG) if (D == DD && p.geff == GG) rc = launch_attn<MathF32<DD, GG>>(p, maps, di.sms, st);
+#define SPD_F32_CASE(DD, GG) if (D == DD && p.geff == GG) rc = launch_attn<MathF32<DD, GG>>(p, maps, di.sms, st, pdl);
         SPD_F32_CASE(64, 1) SPD_F32_CASE(64, 2) SPD_F32_CASE(64, 4) SPD_F32_CASE(64, 8)
         SPD_F32_CASE(128, 1) SPD_F32_CASE(128, 2) SPD_F32_CASE(128, 4) SPD_F32_CASE(128, 8)
 #undef SPD_F32_CASE
@@ -320,8 +380,12 @@ spd_status spd_workspace_size(const spd_shape *shape, size_t *bytes) {
     return SPD_OK;
 }
 
-spd_status spd_partial_attn(const spd_shape *shape, const void *q, const spd_paged_kv *priv, spd_partial out,
-                            void *ws, size_t ws_bytes, void *cuda_stream) {
+static spd_status check_plan(int32_t plan) {
+    return (plan == SPD_PLAN_PER_CALL || plan == SPD_PLAN_STORE || plan == SPD_PLAN_REUSE) ? SPD_OK : SPD_ERR_INVALID_ARG;
+}
+
+static spd_status partial_attn_impl(const spd_shape *shape, const void *q, const spd_paged_kv *priv, spd_partial out,
+                                    int plan, void *ws, size_t ws_bytes, void *cuda_stream) {
     spd_status rc = check_shape(shape);
     if (rc != SPD_OK) return rc;
     if ((rc = check_kv(shape, priv)) != SPD_OK) return rc;
@@ -330,11 +394,13 @@ spd_status spd_partial_attn(const spd_shape *shape, const void *q, const spd_pag
     job.shape = shape; job.q = q; job.part[0] = priv; job.part[1] = nullptr;
     job.mode = OUT_PARTIAL; job.pout = out; job.pin = nullptr; job.out = nullptr; job.out_dtype = SPD_F32;
     job.epoch = next_epoch();
+    job.plan_mode = plan;
     return run_job(job, ws, ws_bytes, cuda_stream);
 }
 
-spd_status spd_service_attn_merge(const spd_shape *shape, const void *q, const spd_paged_kv *pub, spd_partial in,
-                                  void *out, spd_dtype out_dtype, void *ws, size_t ws_bytes, void *cuda_stream) {
+static spd_status service_attn_merge_impl(const spd_shape *shape, const void *q, const spd_paged_kv *pub, spd_partial in,
+                                          void *out, spd_dtype out_dtype, int plan, void *ws, size_t ws_bytes,
+                                          void *cuda_stream) {
     spd_status rc = check_shape(shape);
     if (rc != SPD_OK) return rc;
     if ((rc = check_kv(shape, pub)) != SPD_OK) return rc;
@@ -345,12 +411,13 @@ spd_status spd_service_attn_merge(const spd_shape *shape, const void *q, const s
     job.shape = shape; job.q = q; job.part[0] = nullptr; job.part[1] = pub;
     job.mode = OUT_FINAL; job.pin = &in; job.out = out; job.out_dtype = out_dtype;
     job.epoch = next_epoch();
+    job.plan_mode = plan;
     return run_job(job, ws, ws_bytes, cuda_stream);
 }
 
-spd_status spd_decode_step(const spd_shape *shape, const void *q, const spd_paged_kv *priv, const spd_paged_kv *pub,
-                           void *out, spd_dtype out_dtype, int32_t fused, void *ws, size_t ws_bytes,
-                           void *cuda_stream) {
+static spd_status decode_step_impl(const spd_shape *shape, const void *q, const spd_paged_kv *priv,
+                                   const spd_paged_kv *pub, void *out, spd_dtype out_dtype, int32_t fused, int plan,
+                                   bool plain_order, void *ws, size_t ws_bytes, void *cuda_stream) {
     spd_status rc = check_shape(shape);
     if (rc != SPD_OK) return rc;
     if ((rc = check_kv(shape, priv)) != SPD_OK) return rc;
@@ -362,6 +429,8 @@ spd_status spd_decode_step(const spd_shape *shape, const void *q, const spd_page
         job.shape = shape; job.q = q; job.part[0] = priv; job.part[1] = pub;
         job.mode = OUT_FINAL; job.pin = nullptr; job.out = out; job.out_dtype = out_dtype;
         job.epoch = next_epoch();
+        job.plan_mode = plan;
+        job.plain_order = plain_order;
         return run_job(job, ws, ws_bytes, cuda_stream);
     }
     DeviceInfo di;
@@ -375,8 +444,46 @@ spd_status spd_decode_step(const spd_shape *shape, const void *q, const spd_page
     a.part[0] = priv; a.mode = OUT_PARTIAL; a.pout = mid; a.out_dtype = SPD_F32;
     b.part[1] = pub; b.mode = OUT_FINAL; b.pin = &mid; b.out = out; b.out_dtype = out_dtype;
     a.epoch = b.epoch = next_epoch();
+    a.plan_mode = b.plan_mode = plan;     // each half has a stored plan of its own
+    a.plain_order = plain_order;
     if ((rc = run_job(a, ws, ws_bytes, cuda_stream)) != SPD_OK) return rc;
     return run_job(b, ws, ws_bytes, cuda_stream);
+}
+
+spd_status spd_partial_attn(const spd_shape *shape, const void *q, const spd_paged_kv *priv, spd_partial out,
+                            void *ws, size_t ws_bytes, void *cuda_stream) {
+    return partial_attn_impl(shape, q, priv, out, PLAN_DERIVE, ws, ws_bytes, cuda_stream);
+}
+
+spd_status spd_service_attn_merge(const spd_shape *shape, const void *q, const spd_paged_kv *pub, spd_partial in,
+                                  void *out, spd_dtype out_dtype, void *ws, size_t ws_bytes, void *cuda_stream) {
+    return service_attn_merge_impl(shape, q, pub, in, out, out_dtype, PLAN_DERIVE, ws, ws_bytes, cuda_stream);
+}
+
+spd_status spd_decode_step(const spd_shape *shape, const void *q, const spd_paged_kv *priv, const spd_paged_kv *pub,
+                           void *out, spd_dtype out_dtype, int32_t fused, void *ws, size_t ws_bytes,
+                           void *cuda_stream) {
+    return decode_step_impl(shape, q, priv, pub, out, out_dtype, fused, PLAN_DERIVE, false, ws, ws_bytes, cuda_stream);
+}
+
+spd_status spd_partial_attn_planned(const spd_shape *shape, const void *q, const spd_paged_kv *priv, spd_partial out,
+                                    spd_plan_mode plan, void *ws, size_t ws_bytes, void *cuda_stream) {
+    if (check_plan(plan) != SPD_OK) return SPD_ERR_INVALID_ARG;
+    return partial_attn_impl(shape, q, priv, out, plan, ws, ws_bytes, cuda_stream);
+}
+
+spd_status spd_service_attn_merge_planned(const spd_shape *shape, const void *q, const spd_paged_kv *pub,
+                                          spd_partial in, void *out, spd_dtype out_dtype, spd_plan_mode plan, void *ws,
+                                          size_t ws_bytes, void *cuda_stream) {
+    if (check_plan(plan) != SPD_OK) return SPD_ERR_INVALID_ARG;
+    return service_attn_merge_impl(shape, q, pub, in, out, out_dtype, plan, ws, ws_bytes, cuda_stream);
+}
+
+spd_status spd_decode_step_planned(const spd_shape *shape, const void *q, const spd_paged_kv *priv,
+                                   const spd_paged_kv *pub, void *out, spd_dtype out_dtype, int32_t fused,
+                                   spd_plan_mode plan, void *ws, size_t ws_bytes, void *cuda_stream) {
+    if (check_plan(plan) != SPD_OK) return SPD_ERR_INVALID_ARG;
+    return decode_step_impl(shape, q, priv, pub, out, out_dtype, fused, plan, false, ws, ws_bytes, cuda_stream);
 }
 
 static spd_status check_watch(const spd_watch *w) {
@@ -544,7 +651,7 @@ spd_status spd_append_kv(const spd_shape *shape, const void *k_new, const void *
 }
 
 spd_status spd_token_step(const spd_shape *shape, int32_t num_layers, const spd_layer *layers, spd_dtype out_dtype,
-                          void *ws, size_t ws_bytes, void *cuda_stream) {
+                          int32_t same_lengths, void *ws, size_t ws_bytes, void *cuda_stream) {
     if (!layers || num_layers <= 0) return SPD_ERR_INVALID_ARG;
     for (int32_t i = 0; i < num_layers; ++i) {
         const spd_layer &ly = layers[i];
@@ -554,7 +661,10 @@ spd_status spd_token_step(const spd_shape *shape, int32_t num_layers, const spd_
                                       ly.pub.page_indices, const_cast<int32_t *>(ly.pub.seq_lens), ws, ws_bytes,
                                       cuda_stream);
         if (rc != SPD_OK) return rc;
-        rc = spd_decode_step(shape, ly.q, &ly.priv, &ly.pub, ly.out, out_dtype, 1, ws, ws_bytes, cuda_stream);
+        // With equal lengths in every layer the first layer's plan serves them all.  The attention kernel follows
+        // the append that has just written its lengths and cache: it starts in plain stream order.
+        const int plan = !same_lengths ? PLAN_DERIVE : (i == 0 ? PLAN_DERIVE_STORE : PLAN_LOAD);
+        rc = decode_step_impl(shape, ly.q, &ly.priv, &ly.pub, ly.out, out_dtype, 1, plan, true, ws, ws_bytes, cuda_stream);
         if (rc != SPD_OK) return rc;
     }
     return SPD_OK;
@@ -652,11 +762,10 @@ spd_status spd_query_device_status(void *ws, void *cuda_stream, int32_t *first_b
     if (first_bad_user) *first_bad_user = hdr[HDR_BAD_ENC] ? 0x7fffffff - hdr[HDR_BAD_ENC] : -1;
     if (hdr[HDR_STATUS] == 0) return SPD_OK;
     // clear the sticky words, the per-user flags and the tickets (a kernel that gave up on a wait may
-    // have left tickets drawn); they sit right behind the header
-    const size_t nbad = hdr[HDR_BATCH] > 0 ? align_up(static_cast<size_t>(hdr[HDR_BATCH]) * 4, 256) : 0;
-    const size_t ntic = hdr[HDR_NSEQ] > 0 ? align_up(static_cast<size_t>(hdr[HDR_NSEQ]) * 4, 256) : 0;
+    // have left tickets drawn)
+    const WsHead H = ws_head(hdr[HDR_BATCH] > 0 ? hdr[HDR_BATCH] : 0, hdr[HDR_NSEQ] > 0 ? hdr[HDR_NSEQ] : 0);
     if (cudaMemsetAsync(ws, 0, 8, st) != cudaSuccess) return SPD_ERR_CUDA;
-    if (nbad + ntic && cudaMemsetAsync(static_cast<uint8_t *>(ws) + align_up(HDR_WORDS * 4, 256) + align_up(3 * kMaxGrid * sizeof(float2), 256), 0, nbad + ntic, st) != cudaSuccess)
+    if (H.end > H.bad && cudaMemsetAsync(static_cast<uint8_t *>(ws) + H.bad, 0, H.end - H.bad, st) != cudaSuccess)
         return SPD_ERR_CUDA;
     if (cudaStreamSynchronize(st) != cudaSuccess) return SPD_ERR_CUDA;
     return static_cast<spd_status>(hdr[HDR_STATUS]);
@@ -673,6 +782,52 @@ spd_status spd_set_bf16_math(int32_t path) {
 spd_status spd_set_prefill_rows(int32_t rows) {
     if (rows != 0 && rows != 128 && rows != 256) return SPD_ERR_INVALID_ARG;
     g_prefill_rows.store(rows);
+    return SPD_OK;
+}
+
+spd_status spd_set_split(int32_t min_tiles_per_share, int32_t uniform_shares) {
+    if (min_tiles_per_share < 0 || min_tiles_per_share > (1 << 30)) return SPD_ERR_INVALID_ARG;
+    if (uniform_shares != 0 && uniform_shares != 1) return SPD_ERR_INVALID_ARG;
+    g_min_tiles.store(min_tiles_per_share == 0 ? kMinTilesPerWarp : min_tiles_per_share);
+    g_uniform_shares.store(uniform_shares);
+    return SPD_OK;
+}
+
+spd_status spd_set_programmatic_launch(int32_t on) {
+    if (on != 0 && on != 1) return SPD_ERR_INVALID_ARG;
+    g_pdl.store(on);
+    return SPD_OK;
+}
+
+spd_status spd_debug_read_plan(void *ws, int32_t which, void *cuda_stream, int32_t *tiles, int32_t *shares,
+                               int32_t *bnd, int32_t bnd_capacity) {
+    if (!ws || which < 0 || which >= kPlanSlots || bnd_capacity < 0 || (bnd_capacity > 0 && !bnd)) return SPD_ERR_INVALID_ARG;
+    cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+    const uint8_t *pl = static_cast<const uint8_t *>(ws) + ws_head(0, 0).plan + which * kPlanBytes;
+    int32_t head[PLAN_HDR_WORDS];
+    if (cudaMemcpyAsync(head, pl, sizeof head, cudaMemcpyDeviceToHost, st) != cudaSuccess) return SPD_ERR_CUDA;
+    if (cudaStreamSynchronize(st) != cudaSuccess) return SPD_ERR_CUDA;
+    const int32_t A = head[PLAN_A];
+    if (A < 0 || A > kMaxGrid * kMaxWarpsPerCta) return SPD_ERR_PLAN;
+    if (tiles) *tiles = head[PLAN_T];
+    if (shares) *shares = A;
+    const int32_t nb = bnd_capacity < A + 1 ? bnd_capacity : A + 1;
+    if (nb > 0) {
+        if (cudaMemcpyAsync(bnd, pl + PLAN_BND * 4, static_cast<size_t>(nb) * 4, cudaMemcpyDeviceToHost, st) != cudaSuccess ||
+            cudaStreamSynchronize(st) != cudaSuccess)
+            return SPD_ERR_CUDA;
+    }
+    return SPD_OK;
+}
+
+spd_status spd_debug_sm_moves(void *ws, void *cuda_stream, int64_t *launches, int64_t *moves) {
+    if (!ws) return SPD_ERR_INVALID_ARG;
+    cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+    int32_t hdr[8];
+    if (cudaMemcpyAsync(hdr, ws, sizeof hdr, cudaMemcpyDeviceToHost, st) != cudaSuccess) return SPD_ERR_CUDA;
+    if (cudaStreamSynchronize(st) != cudaSuccess) return SPD_ERR_CUDA;
+    if (launches) *launches = hdr[HDR_SM_LAUNCHES];
+    if (moves) *moves = hdr[HDR_SM_MOVES];
     return SPD_OK;
 }
 
@@ -715,6 +870,7 @@ const char *spd_status_string(spd_status status) {
         case SPD_ERR_BAD_PAGE: return "page index or sequence length out of range (seen on the device)";
         case SPD_ERR_CUDA: return "CUDA call failed";
         case SPD_ERR_TIMEOUT: return "a bounded wait inside a kernel ran out";
+        case SPD_ERR_PLAN: return "no stored plan fits this call (never stored, or stored for another shape or grid)";
     }
     return "unknown status";
 }
@@ -763,11 +919,13 @@ extern "C" spd_status spd_decode_step_static(const spd_shape *shape, const void 
     void *ws = nullptr;
     if ((rc = static_ws_address(&ws)) != SPD_OK) return rc;
     cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
-    // The array still holds the previous call's contents.  Everything in it is rewritten before it is
-    // read, except the sticky status words and the per-user flags: those must start at zero.
+    // The array still holds the previous call's contents, laid out for the previous call's shape.  Three things
+    // must start at zero: the sticky status words, the per-user flags and the merge tickets (this shape's ticket
+    // region may lie where an earlier, smaller shape kept scratch floats, and a call that gave up on a wait leaves
+    // tickets drawn).  The rest -- rate table, stored plans, scratch, the chained step's partial -- is either
+    // rewritten before it is read or harmless when stale.
     if (cudaMemsetAsync(ws, 0, 8, st) != cudaSuccess) return SPD_ERR_CUDA;
-    if (cudaMemsetAsync(static_cast<uint8_t *>(ws) + L.bad, 0, static_cast<size_t>(shape->batch) * 4, st) != cudaSuccess)
-        return SPD_ERR_CUDA;
+    if (cudaMemsetAsync(static_cast<uint8_t *>(ws) + L.bad, 0, L.scratch - L.bad, st) != cudaSuccess) return SPD_ERR_CUDA;
     rc = spd_decode_step(shape, q, priv, pub, out, out_dtype, 1, ws, SPD_STATIC_WS_BYTES, cuda_stream);
     if (rc != SPD_OK || !wait_and_check) return rc;
     return spd_query_device_status(ws, cuda_stream, first_bad_user);

@@ -12,7 +12,9 @@ namespace spd {
 
 constexpr int kPage = 16;             // tokens per KV page
 constexpr int kHeadsPerItem = 8;      // query heads one warp carries for one KV head
-constexpr int kMinTilesPerWarp = 4;   // do not spread tiny batches thinner than this
+constexpr int kMinTilesPerWarp = 4;   // default: do not spread tiny batches thinner than this (tiles per share)
+constexpr int kMaxGrid = 256;         // CTAs (one per SM) the share tables are sized for
+constexpr int kMaxWarpsPerCta = 16;
 constexpr uint32_t kWaitLimit = 1u << 22;  // bounded mbarrier polling (each poll may block ~us)
 
 // Words of the workspace header (int32 each).
@@ -21,7 +23,28 @@ enum HdrWord {
     HDR_BAD_ENC = 1,       // 0 = none, else 0x7fffffff - lowest flagged user (atomicMax)
     HDR_BATCH = 2,         // batch size of the last call (size of the per-user flag array)
     HDR_NSEQ = 3,          // sequences of the last call (size of the ticket array)
+    HDR_SM_LAUNCHES = 4,   // attention launches that compared their CTAs' SMs with the previous launch's
+    HDR_SM_MOVES = 5,      // CTAs of those launches that found themselves on another SM than last time
     HDR_WORDS = 64
+};
+
+// The plan of the last planning launch, kept in the workspace (int32 words): what a later launch with the same
+// lengths loads instead of deriving it again, and what the debugging export reads.
+enum PlanWord {
+    PLAN_TAG = 0,          // id (epoch) of the launch that wrote the plan; 0 = none
+    PLAN_T = 1,            // tiles in the stream
+    PLAN_A = 2,            // warps that own a share
+    PLAN_GRID = 3,         // CTAs of the grid the plan was cut for
+    PLAN_WARPS = 4,        // warps per CTA
+    PLAN_B = 5,            // users
+    PLAN_S = 6,            // sequences per user
+    PLAN_PARTS = 7,        // which partitions the call read (bit 0 private, bit 1 public)
+    PLAN_HDR_WORDS = 16,
+    PLAN_WQ = PLAN_HDR_WORDS,                 // [kMaxGrid] share weight of each CTA
+    PLAN_SMID = PLAN_WQ + kMaxGrid,           // [kMaxGrid] 1 + SM the CTA ran on at the last launch (0 = unknown)
+    PLAN_BND = PLAN_SMID + kMaxGrid,          // [kMaxGrid * kMaxWarpsPerCta + 1] share boundaries
+    PLAN_REC = PLAN_BND + kMaxGrid * kMaxWarpsPerCta + 16,   // [kMaxGrid * kMaxWarpsPerCta][8] where each warp starts
+    PLAN_WORDS = PLAN_REC + kMaxGrid * kMaxWarpsPerCta * 8
 };
 
 // One KV partition as the kernels see it.
@@ -34,6 +57,9 @@ struct PartDev {
 };
 
 enum OutMode { OUT_PARTIAL = 0, OUT_FINAL = 1 };
+// How a launch gets its plan: derives it and keeps only the boundaries for inspection; derives it and stores all of
+// it for later launches; or loads what an earlier launch on this workspace stored (same lengths, same grid).
+enum PlanMode { PLAN_DERIVE = 0, PLAN_DERIVE_STORE = 1, PLAN_LOAD = 2 };
 
 struct Params {
     int32_t B, Hq, Hkv, g;
@@ -50,7 +76,13 @@ struct Params {
     int32_t *tickets;       // [B * S] pieces delivered so far per sequence; zero between calls
     int32_t epoch;          // non-zero id of this call
     float2 *rates;          // [3][kMaxGrid] per-CTA (share weight, cycles) of earlier launches
-    int32_t rate_sel;       // launch counter: this launch writes third rate_sel % 3, reads (rate_sel + 1) % 3
+    int32_t rate_sel;       // attention launches on this workspace so far: this launch writes third rate_sel % 3,
+                            // reads (rate_sel + 1) % 3
+    int32_t *plan;          // [PLAN_WORDS] the stored plan
+    int32_t plan_mode;      // PlanMode
+    int32_t plan_tag;       // what PLAN_TAG must hold for a plan to be loaded / holds once this launch has stored one
+    int32_t min_tiles;      // fewest tiles a share may hold (>= 1)
+    int32_t uniform;        // non-zero: equal shares, the rate table is ignored
     float *scratch;         // [2 * num_warps][8 * D + 16]
     // outputs
     int32_t mode;           // OutMode

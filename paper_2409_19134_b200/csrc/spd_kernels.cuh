@@ -722,9 +722,10 @@ struct Cursor {
 
 constexpr int kUserCache = 1024;   // users whose validated tile counts a CTA keeps in shared memory
 
-// Tile counts of user u: from the CTA's cache when it holds them, else recomputed from the inputs.
+// Tile counts of user u: from the CTA's cache when it holds them (a launch that loaded its plan has no cache:
+// cache == nullptr), else recomputed from the inputs.
 __device__ __forceinline__ void cached_tiles(const Params &p, const int2 *cache, int u, int &n0, int &n1) {
-    if (u < kUserCache) {
+    if (cache != nullptr && u < kUserCache) {
         const int2 v = cache[u];
         n0 = v.x;
         n1 = v.y;
@@ -762,7 +763,6 @@ template <class Math>
 __host__ __device__ constexpr size_t attn_extra_offset() {
     return attn_desc_offset<Math>() + static_cast<size_t>(Math::kWarps) * Math::kStages * 32;
 }
-constexpr int kMaxGrid = 256;   // CTAs (one per SM) the share tables are sized for
 template <class Math>
 __host__ __device__ constexpr size_t attn_bnd_offset() {
     return attn_extra_offset<Math>() + static_cast<size_t>(Math::kWarps) * Math::kExtraBytes;
@@ -795,6 +795,8 @@ attn_kernel(const __grid_constant__ Params p, const __grid_constant__ CUtensorMa
     __shared__ int2 sh_np[kUserCache];
     __shared__ long long cta_clock0;
     __shared__ int32_t cta_exits;
+    __shared__ int32_t sh_jump[Math::kWarps][4];   // (user, sequence, tile) at which each warp resumes after its trailing piece
+    __shared__ int32_t sh_prev_smid;
     uint8_t *base = reinterpret_cast<uint8_t *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
     const int wid = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int gwarp = blockIdx.x * Math::kWarps + wid;
@@ -805,20 +807,31 @@ attn_kernel(const __grid_constant__ Params p, const __grid_constant__ CUtensorMa
     uint8_t *extra = tail + attn_extra_offset<Math>() + static_cast<size_t>(wid) * Math::kExtraBytes;
 
     griddep_launch_dependents();   // the next kernel on the stream may begin its own read-only preamble
-    // the four tensor maps are needed ~7 us from now: fetch them meanwhile (when no partition owns a page they
-    // are never used and hold nothing)
+    // the four tensor maps are needed a few microseconds from now: fetch them meanwhile (when no partition owns a
+    // page they are never used and hold nothing)
     if (wid == 0 && lane < 4 && (p.part[0].num_pages > 0 || p.part[1].num_pages > 0))
         prefetch_tensormap(lane == 0 ? &mk0 : lane == 1 ? &mv0 : lane == 2 ? &mk1 : &mv1);
+    uint32_t smid;
+    asm("mov.u32 %0, %%smid;" : "=r"(smid));
 
-    // ---- plan: every CTA computes the same thing from the inputs alone -------------------------
-    // Thread t sums the tiles of users [t*C, (t+1)*C); a block scan gives chunk prefixes.
     const int C = (p.B + NT - 1) / NT;
     const int G = gridDim.x;
-    // launch N writes third N % 3 and reads the one launch N-2 wrote: launch N-1 may still be running
+    // launch N on a workspace writes third N % 3 and reads the one launch N-2 wrote: launch N-1 may still be running
     const float2 *rate_rd = p.rates + ((p.rate_sel + 1) % 3) * kMaxGrid;
     float2 *rate_wr = p.rates + (p.rate_sel % 3) * kMaxGrid;
+    int32_t *bnd = reinterpret_cast<int32_t *>(tail + attn_bnd_offset<Math>());
+    const bool loaded = p.plan_mode == PLAN_LOAD;
+    const int2 *np_cache = loaded ? nullptr : sh_np;
+    int64_t T64 = 0;
+    int T = 0, A = 0;
+    bool plan_ok = true;
+    int rec = 0;               // PLAN_LOAD: lane k < 8 holds word k of this warp's start record
+    if (threadIdx.x == 0) cta_exits = 0;
+
+    if (!loaded) {
+    // ---- plan: every CTA computes the same thing from the inputs alone -------------------------
+    // Thread t sums the tiles of users [t*C, (t+1)*C); a block scan gives chunk prefixes.
     {
-        if (threadIdx.x == 0) cta_exits = 0;
         // the rate table travels together with the lengths: its loads are issued first and used last, so that
         // the two round trips to memory overlap (G <= 2 NT)
         const int i0 = threadIdx.x, i1 = threadIdx.x + NT;
@@ -862,9 +875,10 @@ attn_kernel(const __grid_constant__ Params p, const __grid_constant__ CUtensorMa
         // CTA left its (weight, cycles) in the rate table.  New weight = old weight moved towards the measured
         // rate (both relative to the mean): most of the way when they disagree by more than 4 % (a real
         // difference between SMs), a quarter of the way otherwise (so that run-to-run noise is averaged out
-        // instead of chased); quantised to integers so that all CTAs cut alike.
+        // instead of chased); quantised to integers so that all CTAs cut alike.  With p.uniform every CTA
+        // weighs the same and the table is not consulted.
         float tw = 0.f, tr = 0.f;
-        bool ok = true;
+        bool ok = p.uniform == 0;
         for (int w = 0; w < Math::kWarps; ++w) { tw += red_w[w]; tr += red_r[w]; ok = ok && red_ok[w] != 0; }
         const float nw = ok ? G / tw : 0.f, nr = ok ? G / tr : 0.f;
         auto quantise = [&](float w_old, float r) {
@@ -878,8 +892,8 @@ attn_kernel(const __grid_constant__ Params p, const __grid_constant__ CUtensorMa
         if (i1 < G) sh_wq[i1] = quantise(v1.x, r1);
         __syncthreads();
     }
-    const int64_t T64 = static_cast<int64_t>(chunk_pfx[NT]) * p.S;
-    const int T = T64 >= (1ll << 31) ? 0 : static_cast<int>(T64);
+    T64 = static_cast<int64_t>(chunk_pfx[NT]) * p.S;
+    T = T64 >= (1ll << 31) ? 0 : static_cast<int>(T64);
 
     // ---- shares, second half: warp w of the grid owns tiles [bnd[w], bnd[w+1]); prefix sums of the CTA weights
     if (wid == 0) {
@@ -897,9 +911,10 @@ attn_kernel(const __grid_constant__ Params p, const __grid_constant__ CUtensorMa
         if (lane == 31) sh_pc[G] = inc;
     }
     __syncthreads();
-    int32_t *bnd = reinterpret_cast<int32_t *>(tail + attn_bnd_offset<Math>());
-    int A = (T + kMinTilesPerWarp - 1) / kMinTilesPerWarp;     // warps that get a share
-    if (A > p.num_warps) A = p.num_warps;
+    {
+        const int64_t want = (static_cast<int64_t>(T) + p.min_tiles - 1) / p.min_tiles;   // warps that get a share
+        A = want > p.num_warps ? p.num_warps : static_cast<int>(want);
+    }
     {
         auto wsum = [&](int w) {     // weights of warps < w; a CTA's warps all carry the CTA's weight
             const int c = w / Math::kWarps;
@@ -913,9 +928,81 @@ attn_kernel(const __grid_constant__ Params p, const __grid_constant__ CUtensorMa
             bnd[w] = static_cast<int32_t>(static_cast<double>(T) * static_cast<double>(wsum(w)) / total);
     }
     __syncthreads();
+    } else {
+    // ---- plan loaded: an earlier launch on this stream and workspace, over the same lengths, left its share
+    // boundaries, the CTA weights and every warp's starting point in the workspace.  It has completed, and its
+    // writes are visible, once the wait below returns.
+        griddep_wait();
+        const int32_t *pl = p.plan;
+        T = __ldcg(pl + PLAN_T);
+        A = __ldcg(pl + PLAN_A);
+        plan_ok = __ldcg(pl + PLAN_TAG) == p.plan_tag && __ldcg(pl + PLAN_GRID) == G &&
+                  __ldcg(pl + PLAN_WARPS) == Math::kWarps && __ldcg(pl + PLAN_B) == p.B && __ldcg(pl + PLAN_S) == p.S &&
+                  __ldcg(pl + PLAN_PARTS) == (p.part[0].present | (p.part[1].present << 1)) && T >= 0 && A >= 0 &&
+                  A <= p.num_warps;
+        if (!plan_ok) T = A = 0;     // nothing is streamed; the status says why
+        T64 = T;
+        for (int w = threadIdx.x; w <= A; w += NT) bnd[w] = __ldcg(pl + PLAN_BND + w);
+        if (threadIdx.x == 0) sh_wq[blockIdx.x] = __ldcg(pl + PLAN_WQ + blockIdx.x);
+        if (lane < 8 && gwarp < A) rec = __ldcg(pl + PLAN_REC + gwarp * 8 + lane);
+        __syncthreads();
+    }
 
     const int t0 = gwarp < A ? bnd[gwarp] : 0;
     const int n = gwarp < A ? bnd[gwarp + 1] - t0 : 0;
+    const int t1 = t0 + n;
+    int tb = t0;               // the warp streams [tb, t1) first, then [t0, tb)
+    Cursor c;
+    c.u = c.sq = c.j = 0;
+
+    // Where tile t sits: its user (the u with S * pfx[u] <= t < S * pfx[u + 1]), the tiles per
+    // sequence of that user, the sequence and the tile within it.  (Needs the derived plan.)
+    auto seq_of_tile = [&](int t, int &u, int &np, int &sq, int &jt) {
+        const int x = t / p.S;    // in units of tiles per sequence
+        int lo = 0, hi = NT;      // invariant: chunk_pfx[lo] <= x < chunk_pfx[hi]
+        while (hi - lo > 1) {
+            const int mid = (lo + hi) >> 1;
+            if (chunk_pfx[mid] <= x) lo = mid; else hi = mid;
+        }
+        int acc = chunk_pfx[lo], n0 = 0, n1 = 0;
+        for (u = lo * C;; ++u) {  // ends inside the chunk, because the chunk holds tile x
+            cached_tiles(p, sh_np, u, n0, n1);
+            if (acc + n0 + n1 > x) break;
+            acc += n0 + n1;
+        }
+        np = n0 + n1;
+        const int r = t - acc * p.S;
+        sq = r / np;
+        jt = r - sq * np;
+    };
+
+    // Order of work.  A share usually ends inside a sequence; that trailing piece needs a ticket
+    // (a fence and an atomic, perhaps a merge: round trips to memory).  Done last they would be
+    // exposed at the end of the kernel, done first the other warps cover them.  So the warp
+    // streams [tb, t1) -- its trailing piece -- first and [t0, tb) afterwards.  Where the warp starts
+    // (tile tb) and where it resumes (tile t0, kept in shared memory until then) make up its start record.
+    if (n > 0) {
+        int ju = 0, jsq = 0, jj = 0;
+        if (!loaded) {
+            int u, np, sq, jt;
+            seq_of_tile(t1 - 1, u, np, sq, jt);
+            if (jt != np - 1 && t1 - 1 - jt > t0) tb = t1 - 1 - jt;
+            seq_of_tile(tb, c.u, np, c.sq, c.j);
+            if (tb != t0) seq_of_tile(t0, ju, np, jsq, jj);
+        } else {
+            tb = __shfl_sync(0xffffffffu, rec, 0);
+            c.u = __shfl_sync(0xffffffffu, rec, 1);
+            c.sq = __shfl_sync(0xffffffffu, rec, 2);
+            c.j = __shfl_sync(0xffffffffu, rec, 3);
+            ju = __shfl_sync(0xffffffffu, rec, 4);
+            jsq = __shfl_sync(0xffffffffu, rec, 5);
+            jj = __shfl_sync(0xffffffffu, rec, 6);
+            if (tb < t0 || tb >= t1) tb = t0;      // cannot happen with a plan this kernel stored
+        }
+        if (lane == 0) { sh_jump[wid][0] = ju; sh_jump[wid][1] = jsq; sh_jump[wid][2] = jj; }
+        rec = lane == 0 ? tb : lane == 1 ? c.u : lane == 2 ? c.sq : lane == 3 ? c.j : lane == 4 ? ju : lane == 5 ? jsq : jj;
+        __syncwarp();
+    }
 
     // Everything up to the first tile loads only READS the call's inputs (lengths, page tables, the
     // KV pools, a rate table nobody writes any more), so it may run while the previous kernel on the
@@ -923,16 +1010,37 @@ attn_kernel(const __grid_constant__ Params p, const __grid_constant__ CUtensorMa
     // partial and the outputs, and waits for that kernel (griddep_wait below).
     auto after_previous_kernel = [&]() {
         griddep_wait();
-        if (threadIdx.x == 0) cta_clock0 = clock64();
+        if (threadIdx.x == 0) {
+            cta_clock0 = clock64();
+            sh_prev_smid = __ldcg(p.plan + PLAN_SMID + blockIdx.x);
+        }
         if (blockIdx.x == 0 && threadIdx.x == 0) {
             p.hdr[HDR_BATCH] = p.B;
             p.hdr[HDR_NSEQ] = p.B * p.S;
             if (T64 >= (1ll << 31)) flag_error(p.hdr, 2 /* SPD_ERR_UNSUPPORTED */, -1);   // 32-bit tile counter
+            if (!plan_ok) flag_error(p.hdr, 7 /* SPD_ERR_PLAN */, -1);
+        }
+        // the plan stays in the workspace: boundaries and weights always (for inspection), the start records and
+        // a valid tag when a later launch is to load it
+        if (!loaded) {
+            int32_t *pl = p.plan;
+            if (blockIdx.x == 0) {
+                for (int w = threadIdx.x; w <= A; w += NT) pl[PLAN_BND + w] = bnd[w];
+                for (int i = threadIdx.x; i < G; i += NT) pl[PLAN_WQ + i] = sh_wq[i];
+                if (threadIdx.x == 0) {
+                    pl[PLAN_TAG] = p.plan_mode == PLAN_DERIVE_STORE ? p.plan_tag : 0;
+                    pl[PLAN_T] = T; pl[PLAN_A] = A; pl[PLAN_GRID] = G; pl[PLAN_WARPS] = Math::kWarps;
+                    pl[PLAN_B] = p.B; pl[PLAN_S] = p.S;
+                    pl[PLAN_PARTS] = p.part[0].present | (p.part[1].present << 1);
+                }
+            }
+            if (p.plan_mode == PLAN_DERIVE_STORE && n > 0 && lane < 8) pl[PLAN_REC + gwarp * 8 + lane] = rec;
         }
         // users that own no tile (nothing cached, or tables inconsistent): written and flagged here
+        if (plan_ok)
         for (int u = gwarp; u < p.B; u += p.num_warps) {
             int n0, n1;
-            cached_tiles(p, sh_np, u, n0, n1);
+            cached_tiles(p, np_cache, u, n0, n1);
             if (n0 + n1 != 0) continue;
             const bool bad = user_tiles<true>(p, u, n0, n1);
             for (int sq = 0; sq < p.S; ++sq) {
@@ -955,46 +1063,8 @@ attn_kernel(const __grid_constant__ Params p, const __grid_constant__ CUtensorMa
     }
     __syncwarp();
 
-    // Where tile t sits: its user (the u with S * pfx[u] <= t < S * pfx[u + 1]), the tiles per
-    // sequence of that user, the sequence and the tile within it.
-    auto seq_of_tile = [&](int t, int &u, int &np, int &sq, int &jt) {
-        const int x = t / p.S;    // in units of tiles per sequence
-        int lo = 0, hi = NT;      // invariant: chunk_pfx[lo] <= x < chunk_pfx[hi]
-        while (hi - lo > 1) {
-            const int mid = (lo + hi) >> 1;
-            if (chunk_pfx[mid] <= x) lo = mid; else hi = mid;
-        }
-        int acc = chunk_pfx[lo], n0 = 0, n1 = 0;
-        for (u = lo * C;; ++u) {  // ends inside the chunk, because the chunk holds tile x
-            cached_tiles(p, sh_np, u, n0, n1);
-            if (acc + n0 + n1 > x) break;
-            acc += n0 + n1;
-        }
-        np = n0 + n1;
-        const int r = t - acc * p.S;
-        sq = r / np;
-        jt = r - sq * np;
-    };
-    Cursor c;
-    auto seek = [&](int t) {
-        int np;
-        seq_of_tile(t, c.u, np, c.sq, c.j);
-        cursor_load_user(c, p, sh_np);
-    };
-
-    // Order of work.  A share usually ends inside a sequence; that trailing piece needs a ticket
-    // (a fence and an atomic, perhaps a merge: round trips to memory).  Done last they would be
-    // exposed at the end of the kernel, done first the other warps cover them.  So the warp
-    // streams [tb, t1) -- its trailing piece -- first and [t0, tb) afterwards.
-    const int t1 = t0 + n;
-    int tb = t0;
-    {
-        int u, np, sq, jt;
-        seq_of_tile(t1 - 1, u, np, sq, jt);
-        if (jt != np - 1 && t1 - 1 - jt > t0) tb = t1 - 1 - jt;
-    }
     const int n2 = tb == t0 ? n : t1 - tb;   // tiles streamed before the jump back to t0
-    seek(tb);
+    cursor_load_user(c, p, np_cache);
     int cur_t = tb;            // index in the tile stream of the next tile to issue
 
     const uint64_t stream_policy = l2_evict_first_policy();
@@ -1003,7 +1073,11 @@ attn_kernel(const __grid_constant__ Params p, const __grid_constant__ CUtensorMa
     bool seg_has_t0 = false;   // ... and holds the share's first tile
 
     auto issue = [&](int stage) {
-        if (issued == n2 && n2 < n) { seek(t0); cur_t = t0; }
+        if (issued == n2 && n2 < n) {      // the trailing piece is out: back to the share's first tile
+            c.u = sh_jump[wid][0]; c.sq = sh_jump[wid][1]; c.j = sh_jump[wid][2];
+            cursor_load_user(c, p, np_cache);
+            cur_t = t0;
+        }
         // page of tile (c.u, c.sq, c.j)
         const int part = c.j >= c.npp ? 1 : 0;
         const int jj = part ? c.j - c.npp : c.j;
@@ -1049,7 +1123,15 @@ attn_kernel(const __grid_constant__ Params p, const __grid_constant__ CUtensorMa
             c.j = 0;
             if (++c.sq == p.S) {
                 c.sq = 0;
-                do { ++c.u; cursor_load_user(c, p, sh_np); } while (c.np == 0 && c.u < p.B - 1);
+                do {
+                    if (c.u + 1 >= p.B) {     // only a loaded plan that no longer fits the lengths runs off the end
+                        c.np = c.npp = 0;
+                        if (lane == 0) flag_error(p.hdr, 7 /* SPD_ERR_PLAN */, -1);
+                        break;
+                    }
+                    ++c.u;
+                    cursor_load_user(c, p, np_cache);
+                } while (c.np == 0);
             } else {
                 c.key = -1;   // same user, page table starts over
             }
@@ -1084,7 +1166,9 @@ attn_kernel(const __grid_constant__ Params p, const __grid_constant__ CUtensorMa
             __syncwarp();
             const int kind = d.y >> 8;
             if (kind == 0) {
-                finalize_segment<D>(p, So, Sm, Sl, d.z, d.w, lane, seg_bad);
+                // a chained step's second half: a user flagged by the first half (same call id) stays zeroed
+                const bool flagged = p.in_o != nullptr && __ldcg(p.bad + d.z) == p.epoch;
+                finalize_segment<D>(p, So, Sm, Sl, d.z, d.w, lane, seg_bad || flagged);
             } else {
                 piece_store<D>(p, So, Sm, Sl, kind, gwarp, lane);
                 const PieceInfo pp{d.z, d.w, e.x, e.z - e.y, seg_bad};
@@ -1105,6 +1189,7 @@ attn_kernel(const __grid_constant__ Params p, const __grid_constant__ CUtensorMa
 
     // ---- the CTA's last warp out leaves (weight, cycles) for the next call's shares -------------
     __syncwarp();
+    __threadfence_block();
     if (lane == 0 && atomicAdd(&cta_exits, 1) == Math::kWarps - 1) {
         const int wa = blockIdx.x * Math::kWarps, wb = wa + Math::kWarps;
         const int tiles = (wb <= A ? bnd[wb] : T) - (wa <= A ? bnd[wa] : T);
@@ -1112,6 +1197,14 @@ attn_kernel(const __grid_constant__ Params p, const __grid_constant__ CUtensorMa
         if (tiles >= 32 * Math::kWarps)
             v = make_float2(static_cast<float>(sh_wq[blockIdx.x]), static_cast<float>(clock64() - cta_clock0));
         __stcg(rate_wr + blockIdx.x, v);
+        // The rates belong to SMs, the table is indexed by CTA: count how often a CTA index comes back on another SM
+        // than at the previous launch on this workspace (read by spd_debug_sm_moves).
+        const int sm = static_cast<int>(smid) + 1, prev = sh_prev_smid;
+        if (prev != 0) {
+            if (prev != sm) atomicAdd(&p.hdr[HDR_SM_MOVES], 1);
+            if (blockIdx.x == 0) atomicAdd(&p.hdr[HDR_SM_LAUNCHES], 1);
+        }
+        p.plan[PLAN_SMID + blockIdx.x] = sm;
     }
 }
 

@@ -34,8 +34,8 @@ def test_every_declared_symbol_is_exported(lib):
 
 
 def test_status_strings(lib):
-    seen = {spd.status_string(c) for c in range(7)}
-    assert len(seen) == 7 and "unknown status" not in seen
+    seen = {spd.status_string(c) for c in range(8)}
+    assert len(seen) == 8 and "unknown status" not in seen
     assert spd.status_string(99) == "unknown status"
 
 
@@ -75,8 +75,16 @@ def test_bad_arguments_are_rejected_on_the_host(lib):
     assert lib.spd_prefill_attn(C.byref(ok), *pf_args) == 2
     assert lib.spd_prefill_attn(C.byref(spd.make_shape(2, 8, 8, 128, torch.bfloat16, -1.0)), *pf_args) == 2
     assert lib.spd_prefill_attn(C.byref(spd.make_shape(2, 8, 8, 128, torch.bfloat16, 0.1)), *pf_args) == 1   # null offsets
-    assert lib.spd_token_step(C.byref(ok), 0, None, 0, None, 0, None) == 1
-    assert lib.spd_token_step(C.byref(ok), 2, None, 0, None, 0, None) == 1
+    assert lib.spd_token_step(C.byref(ok), 0, None, 0, 0, None, 0, None) == 1
+    assert lib.spd_token_step(C.byref(ok), 2, None, 0, 1, None, 0, None) == 1
+    # the planned calls check the plan mode first; the knobs and the debugging aids check their arguments
+    assert lib.spd_decode_step_planned(C.byref(ok), None, None, None, None, 0, 1, 3, None, 0, None) == 1
+    assert lib.spd_partial_attn_planned(C.byref(ok), None, None, part, -1, None, 0, None) == 1
+    assert lib.spd_service_attn_merge_planned(C.byref(ok), None, None, part, None, 0, 5, None, 0, None) == 1
+    assert lib.spd_set_split(-1, 0) == 1 and lib.spd_set_split(4, 2) == 1 and lib.spd_set_split(0, 0) == 0
+    assert lib.spd_set_programmatic_launch(2) == 1
+    assert lib.spd_debug_read_plan(None, 0, None, None, None, None, 0) == 1
+    assert lib.spd_debug_sm_moves(None, None, None, None) == 1
     assert lib.spd_set_prefill_rows(64) == 1 and lib.spd_set_prefill_rows(256) == 0 and lib.spd_set_prefill_rows(0) == 0
     assert lib.spd_set_bf16_math(2) == 1
 

@@ -39,7 +39,7 @@ def _close(a, b):
 
 def test_static_workspace_matches_regular_entry_point_twice_in_a_row():
     cfgs = [dict(batch=9, hq=32, hkv=8, d=128, dtype="bf16", lin=("uniform", 1, 2500), lout=("uniform", 0, 300), seed=31),
-            # second call: fewer users and other lengths, so the array holds a stale, larger plan
+            # second call: fewer users and long prompts, cut into many pieces that leave their floats in the scratch
             dict(batch=4, hq=32, hkv=8, d=128, dtype="bf16", lin=("uniform", 20000, 30000), lout=("uniform", 1, 60), seed=32)]
     for cfg in cfgs:
         w = wl.make_workload(cfg, device="cuda", slack=True)
@@ -52,6 +52,31 @@ def test_static_workspace_matches_regular_entry_point_twice_in_a_row():
         assert (code, bad) == (spd.SPD_OK, -1)
         assert (torch.cuda.memory_allocated(), torch.cuda.memory_reserved()) == before
         _close(out, ref)
+
+
+def test_static_workspace_survives_a_change_of_shape_between_calls():
+    """The array is laid out per call.  When the batch grows, the new call's merge tickets lie where the previous
+    call kept scratch floats; when the dtype or the number of KV heads changes, pitch and offsets move.  Whatever
+    the previous call left there, every row of the output must be written and right."""
+    seq = [dict(batch=4, hq=32, hkv=8, d=128, dtype="bf16", lin=("uniform", 20000, 30000), lout=("uniform", 1, 60), seed=34),
+           dict(batch=128, hq=32, hkv=8, d=128, dtype="bf16", lin=("uniform", 600, 5000), lout=("uniform", 0, 100), seed=35),   # batch grows
+           dict(batch=3, hq=8, hkv=2, d=128, dtype="f32", lin=("uniform", 9000, 12000), lout=("uniform", 1, 50), seed=36),      # fp32: 4 warps per CTA
+           dict(batch=70, hq=32, hkv=32, d=128, dtype="bf16", lin=("uniform", 900, 4000), lout=("uniform", 1, 100), seed=37),   # bf16 again, four times the KV heads
+           dict(batch=9, hq=16, hkv=1, d=64, dtype="bf16", lin=("uniform", 3000, 9000), lout=("uniform", 0, 40), seed=38)]      # one KV head, groups of 8, head_dim 64
+    for k, cfg in enumerate(seq):
+        w = wl.make_workload(cfg, device="cuda")
+        shape, ref = _regular(w)
+        assert spd.spd_workspace_size(shape) <= spd.STATIC_WS_BYTES
+        for wait in (False, True):
+            out = torch.full_like(ref, float("nan"))
+            code, bad = spd.spd_decode_step_static(shape, w.q, w.priv, w.pub, out, wait_and_check=wait)
+            torch.cuda.synchronize()
+            assert (code, bad) == (spd.SPD_OK, -1), f"call {k}"
+            assert bool(torch.isfinite(out).all()), f"call {k}: rows left unwritten"
+            if w.dtype == torch.float32:
+                assert float((out - ref).abs().max()) <= 1e-5
+            else:
+                _close(out, ref)
 
 
 def test_static_workspace_clears_stale_flags_and_rejects_big_shapes():
