@@ -458,8 +458,8 @@ def time_append(spd, w, shape, ws, calls=8):
 
 
 def time_token_step(spd, w, shape, ws, n_layers=8, replays=4):
-    """spd_token_step: the append plus the fused decode step for each of `n_layers` layers (every layer with its
-    own copy of the caches), run eagerly and replayed from one CUDA graph; microseconds per token step.  Every
+    """spd_token_step: the append and the fused decode step, one launch per layer, for each of `n_layers` layers
+    (every layer with its own copy of the caches), run eagerly and replayed from one CUDA graph; microseconds per token step.  Every
     run appends a token per user and layer, so the lengths are first moved back by the number of runs."""
     if int(w.pub.seq_lens.min()) < 1:
         return None
@@ -502,7 +502,7 @@ def time_token_step(spd, w, shape, ws, n_layers=8, replays=4):
     if code != spd.SPD_OK:
         raise RuntimeError(f"token step failed: status {code}, user {bad}")
     kv = sum(int(p[3].seq_lens.sum()) + int(p[4].seq_lens.sum()) for p in layers) * 2 * w.num_kv_heads * w.head_dim * w.elem_size
-    return {"layers": n_layers, "eager_us": eager, "graph_us": replay, "kernels_per_step": 2 * n_layers,
+    return {"layers": n_layers, "eager_us": eager, "graph_us": replay, "kernels_per_step": n_layers,
             "kv_gbs_graph": kv / replay / 1e3, "plan": "derived by layer 0, loaded by the other layers"}
 
 
@@ -679,13 +679,11 @@ def run_cuda(args):
             if name in (cfg, co):
                 continue
             others[name], w = measure_config(spd, name, dev, steps, warmup, local_rank, seconds=0.4)
-            if name != "c2_llama2_7b":
-                del w
-                torch.cuda.empty_cache()
+            del w
+            torch.cuda.empty_cache()
         line["other_configs"] = others
         # the studies around the path run on the Llama-2-7B-shaped layer (the smallest bf16 configuration)
-        if "c2_llama2_7b" not in others:
-            w = wl.make_workload("c2_llama2_7b", device=dev)
+        w = wl.make_workload("c2_llama2_7b", device=dev)
         shape2 = spd.make_shape(w.batch, w.num_q_heads, w.num_kv_heads, w.head_dim, w.dtype, w.sm_scale)
         ws2 = spd.alloc_workspace(shape2)
         line["prefill"] = time_prefill(spd, dev)

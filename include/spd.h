@@ -31,7 +31,7 @@
  *     stream is still finishing; q, an incoming partial, the workspace and the outputs are touched only after
  *     that kernel has completed.  If a kernel of yours on the same stream writes lengths, page tables or KV rows
  *     immediately before a call, launch in plain stream order: spd_set_programmatic_launch(0), or SPD_NO_PDL=1
- *     in the environment.  The library's own append is followed by a plain-order launch inside spd_token_step.
+ *     in the environment.  Where the library's own calls write such inputs (the appends), they order themselves.
  *   - Threads.  Calls may come from several host threads; calls that share a workspace must be ordered by the
  *     caller (one stream at a time per workspace).  Each workspace keeps a small table of streaming rates that
  *     sizes the next call's shares; it is rotated by a per-workspace launch count held on the host, so calls on
@@ -152,7 +152,8 @@ spd_status spd_decode_step(const spd_shape *shape, const void *q, const spd_page
  *                       partitions) on this workspace and stream left, instead of deriving it.  The caller
  *                       states thereby that shape and every length are what they were at that call (page tables,
  *                       pools, q may differ).  A plan that was never stored, or was stored for another shape,
- *                       raises SPD_ERR_PLAN and the call writes nothing; lengths that changed silently give
+ *                       raises SPD_ERR_PLAN and the call writes nothing (a plain or PER_CALL call of the same
+ *                       kind in between discards the stored plan); lengths that changed silently give
  *                       wrong results for the users concerned (never a fault: every index is still checked).
  * Reuse pays for small calls, where deriving the plan is most of the time; large calls hide it anyway.
  */
@@ -232,20 +233,37 @@ spd_status spd_append_kv(const spd_shape *shape, const void *k_new, const void *
                          void *cuda_stream);
 
 /*
+ * The append and the decode step in ONE launch (protocol steps 3a, 3b and 3c; Fig. 3 steps 2 to 5): the fused
+ * spd_decode_step over a public partition that already counts the new token, whose K and V rows are taken from
+ * k_new / v_new ([batch][num_kv_heads][head_dim], shape dtype) instead of the cache, and written to the cache on
+ * the way.  On return of the kernel the row of user u sits at token position seq_lens[u] of `pub` (the value
+ * before the call) and seq_lens[u] has grown by one, in place, as with spd_append_kv; `pub`'s pools and seq_lens
+ * are written although the struct declares them const.  A user whose listed pages are full, or who is flagged
+ * for any other reason during the call (inconsistent table, page index outside a pool), gets zeros as output, no
+ * append and an unchanged length, and raises SPD_ERR_BAD_PAGE.  `plan` as in the *_planned calls; a plan is
+ * cut for the lengths INCLUDING the new token, so SPD_PLAN_REUSE fits a cache with the same lengths as the one
+ * the storing call saw before ITS append.  A call that derives its plan starts in plain stream order.
+ */
+spd_status spd_decode_step_append(const spd_shape *shape, const void *q, const void *k_new, const void *v_new,
+                                  const spd_paged_kv *priv, const spd_paged_kv *pub, void *out,
+                                  spd_dtype out_dtype, spd_plan_mode plan, void *ws, size_t ws_bytes,
+                                  void *cuda_stream);
+
+/*
  * One token step over `num_layers` layers (protocol step 3 for every layer of the model; Fig. 3 steps 2 to
- * 5): for each layer in order, the new token's K and V rows are appended to that layer's public cache
- * (spd_append_kv) and the layer's decode step runs fused (spd_decode_step).  `layers` is a HOST array;
+ * 5): for each layer in order, the new token's K and V rows are appended to that layer's public cache and the
+ * layer's decode step runs, both inside one launch (spd_decode_step_append).  `layers` is a HOST array;
  * every pointer inside it is a device pointer that the caller owns.  Each layer brings its own caches,
- * page tables and lengths (layers[i].pub's pools and seq_lens are written by the append), its own q and
- * its own output.  In a model q of layer i+1 depends on layer i's output through the weights; those are
- * not this library's, so all inputs are taken as given and the driver only fixes the order and the launch
- * structure: 2 * num_layers kernels on `cuda_stream`, nothing else, so that a caller can capture the whole
- * token step in one CUDA graph and replay it (what is frozen into a graph is listed under "CUDA graphs" at the
- * top of this file).  The workspace is shared by the layers.  same_lengths != 0 states that every layer's
- * private and public seq_lens hold the same values as layer 0's (as in a model, whose layers all cache the same
- * tokens): the plan is then derived once, by layer 0, and loaded by the other layers (SPD_PLAN_STORE /
- * SPD_PLAN_REUSE above).  Stops at the first host-side error; device-side mistakes are reported through
- * spd_query_device_status as for the single calls.
+ * page tables and lengths (layers[i].pub's pools and seq_lens are written by the append; two layers must not
+ * share a seq_lens array), its own q and its own output.  In a model q of layer i+1 depends on layer i's output
+ * through the weights; those are not this library's, so all inputs are taken as given and the driver only fixes
+ * the order and the launch structure: num_layers kernels on `cuda_stream`, nothing else, so that a caller can
+ * capture the whole token step in one CUDA graph and replay it (what is frozen into a graph is listed under
+ * "CUDA graphs" at the top of this file).  The workspace is shared by the layers.  same_lengths != 0 states
+ * that every layer's private and public seq_lens hold the same values as layer 0's (as in a model, whose layers
+ * all cache the same tokens): the plan is then derived once, by layer 0, and loaded by the other layers
+ * (SPD_PLAN_STORE / SPD_PLAN_REUSE above).  Stops at the first host-side error; device-side mistakes are
+ * reported through spd_query_device_status as for the single calls.
  */
 typedef struct {
     const void *q;             /* [batch][num_q_heads][head_dim]                                  */

@@ -27,7 +27,7 @@ EXPORTS = ["spd_workspace_size", "spd_partial_attn", "spd_service_attn_merge", "
            "spd_partial_attn_watch", "spd_decode_step_watch", "spd_set_bf16_math", "spd_merge_partials", "spd_prefill_attn",
            "spd_set_prefill_rows", "spd_token_step", "spd_partial_attn_planned", "spd_service_attn_merge_planned",
            "spd_decode_step_planned", "spd_set_split", "spd_set_programmatic_launch", "spd_debug_read_plan",
-           "spd_debug_sm_moves"]
+           "spd_debug_sm_moves", "spd_decode_step_append"]
 
 
 class SpdError(RuntimeError):
@@ -104,6 +104,8 @@ def lib() -> C.CDLL:
                                                      vp, sz, vp]
         L.spd_decode_step_planned.argtypes = [C.POINTER(Shape), vp, C.POINTER(PagedKV), C.POINTER(PagedKV), vp, C.c_int,
                                               C.c_int32, C.c_int, vp, sz, vp]
+        L.spd_decode_step_append.argtypes = [C.POINTER(Shape), vp, vp, vp, C.POINTER(PagedKV), C.POINTER(PagedKV), vp, C.c_int,
+                                             C.c_int, vp, sz, vp]
         L.spd_set_split.argtypes = [C.c_int32, C.c_int32]
         L.spd_set_programmatic_launch.argtypes = [C.c_int32]
         L.spd_debug_read_plan.argtypes = [vp, C.c_int32, vp, C.POINTER(C.c_int32), C.POINTER(C.c_int32),
@@ -320,6 +322,16 @@ def spd_append_kv(shape, k_new, v_new, part, ws, stream=None) -> None:
                                part.v_pool.data_ptr(), int(part.k_pool.shape[0]), part.page_indptr.data_ptr(),
                                _ptr(part.page_indices), part.seq_lens.data_ptr(), ws.data_ptr(), ws.numel(),
                                _stream_ptr(stream)), "spd_append_kv")
+
+
+def spd_decode_step_append(shape, q, k_new, v_new, priv, pub, out, ws, plan=SPD_PLAN_PER_CALL, stream=None) -> None:
+    """The append of the new token's rows to `pub` (pools and seq_lens updated in place) and the fused decode step
+    over the grown cache, in one launch."""
+    assert k_new.is_contiguous() and v_new.is_contiguous()
+    a, b = paged_kv(priv), paged_kv(pub)
+    _check(lib().spd_decode_step_append(C.byref(shape), q.data_ptr(), k_new.data_ptr(), v_new.data_ptr(), C.byref(a),
+                                        C.byref(b), out.data_ptr(), _dtype_code(out.dtype), int(plan), ws.data_ptr(),
+                                        ws.numel(), _stream_ptr(stream)), "spd_decode_step_append")
 
 
 def spd_token_step(shape, layers, ws, stream=None, same_lengths=False) -> None:

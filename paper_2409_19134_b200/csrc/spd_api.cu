@@ -250,6 +250,7 @@ struct Job {
     const spd_watch *watch;        // optional monitor of a private token range
     int plan_mode;                 // PlanMode: derive per call (default), derive and store, or load the stored plan
     bool plain_order;              // launch in plain stream order (an input was written by the kernel just before)
+    const void *k_new, *v_new;     // optional append of the new token's rows to part[1] inside the launch
 };
 
 // The stored plan of a call is tagged with what it was cut for besides the lengths, so that a launch told to load a
@@ -303,6 +304,16 @@ spd_status run_job(const Job &job, void *ws, size_t ws_bytes, void *stream) {
     p.out = job.out;
     p.out_bf16 = job.out_dtype == SPD_BF16;
     if (job.watch) { p.watch_lo = job.watch->tok_lo; p.watch_hi = job.watch->tok_hi; p.watch_out = job.watch->out; }
+    if (job.k_new) {
+        if (!job.part[1] || !job.v_new || job.part[1]->num_pages <= 0 || misaligned(job.k_new, 16) || misaligned(job.v_new, 16))
+            return SPD_ERR_INVALID_ARG;
+        p.k_new = static_cast<const uint8_t *>(job.k_new);
+        p.v_new = static_cast<const uint8_t *>(job.v_new);
+        // the append writes through pointers that spd_paged_kv declares const for the readers
+        p.k_pool_w = static_cast<uint8_t *>(const_cast<void *>(job.part[1]->k_pool));
+        p.v_pool_w = static_cast<uint8_t *>(const_cast<void *>(job.part[1]->v_pool));
+        p.lens_w = const_cast<int32_t *>(job.part[1]->seq_lens);
+    }
 
     CUtensorMap maps[4];
     int have = -1;
@@ -417,7 +428,8 @@ static spd_status service_attn_merge_impl(const spd_shape *shape, const void *q,
 
 static spd_status decode_step_impl(const spd_shape *shape, const void *q, const spd_paged_kv *priv,
                                    const spd_paged_kv *pub, void *out, spd_dtype out_dtype, int32_t fused, int plan,
-                                   bool plain_order, void *ws, size_t ws_bytes, void *cuda_stream) {
+                                   bool plain_order, void *ws, size_t ws_bytes, void *cuda_stream,
+                                   const void *k_new = nullptr, const void *v_new = nullptr) {
     spd_status rc = check_shape(shape);
     if (rc != SPD_OK) return rc;
     if ((rc = check_kv(shape, priv)) != SPD_OK) return rc;
@@ -431,8 +443,10 @@ static spd_status decode_step_impl(const spd_shape *shape, const void *q, const 
         job.epoch = next_epoch();
         job.plan_mode = plan;
         job.plain_order = plain_order;
+        job.k_new = k_new; job.v_new = v_new;
         return run_job(job, ws, ws_bytes, cuda_stream);
     }
+    if (k_new) return SPD_ERR_UNSUPPORTED;      // the append rides on the fused step only
     DeviceInfo di;
     if ((rc = device_info(&di)) != SPD_OK) return rc;
     if (!ws || misaligned(ws, 256)) return SPD_ERR_INVALID_ARG;
@@ -477,6 +491,17 @@ spd_status spd_service_attn_merge_planned(const spd_shape *shape, const void *q,
                                           size_t ws_bytes, void *cuda_stream) {
     if (check_plan(plan) != SPD_OK) return SPD_ERR_INVALID_ARG;
     return service_attn_merge_impl(shape, q, pub, in, out, out_dtype, plan, ws, ws_bytes, cuda_stream);
+}
+
+spd_status spd_decode_step_append(const spd_shape *shape, const void *q, const void *k_new, const void *v_new,
+                                  const spd_paged_kv *priv, const spd_paged_kv *pub, void *out, spd_dtype out_dtype,
+                                  spd_plan_mode plan, void *ws, size_t ws_bytes, void *cuda_stream) {
+    if (check_plan(plan) != SPD_OK || !k_new || !v_new) return SPD_ERR_INVALID_ARG;
+    // A launch that derives its plan reads the lengths before the previous kernel on the stream has finished, and
+    // that kernel may be the previous call of this very function, which adds one to them as its last act: plain
+    // stream order.  A launch that loads its plan waits first anyway.
+    return decode_step_impl(shape, q, priv, pub, out, out_dtype, 1, plan, plan != SPD_PLAN_REUSE, ws, ws_bytes,
+                            cuda_stream, k_new, v_new);
 }
 
 spd_status spd_decode_step_planned(const spd_shape *shape, const void *q, const spd_paged_kv *priv,
@@ -655,16 +680,14 @@ spd_status spd_token_step(const spd_shape *shape, int32_t num_layers, const spd_
     if (!layers || num_layers <= 0) return SPD_ERR_INVALID_ARG;
     for (int32_t i = 0; i < num_layers; ++i) {
         const spd_layer &ly = layers[i];
-        // the append writes through pointers that spd_paged_kv declares const for the readers
-        spd_status rc = spd_append_kv(shape, ly.k_new, ly.v_new, const_cast<void *>(ly.pub.k_pool),
-                                      const_cast<void *>(ly.pub.v_pool), ly.pub.num_pages, ly.pub.page_indptr,
-                                      ly.pub.page_indices, const_cast<int32_t *>(ly.pub.seq_lens), ws, ws_bytes,
-                                      cuda_stream);
-        if (rc != SPD_OK) return rc;
-        // With equal lengths in every layer the first layer's plan serves them all.  The attention kernel follows
-        // the append that has just written its lengths and cache: it starts in plain stream order.
+        if (!ly.k_new || !ly.v_new) return SPD_ERR_INVALID_ARG;
+        // With equal lengths in every layer the first layer's plan serves them all.  The first launch of the token
+        // step starts in plain stream order (the kernel before it may be the previous token step's launch on the
+        // same layer, which bumps the lengths this one reads); the others read their own layer's arrays, which
+        // were last written a whole token step ago.
         const int plan = !same_lengths ? PLAN_DERIVE : (i == 0 ? PLAN_DERIVE_STORE : PLAN_LOAD);
-        rc = decode_step_impl(shape, ly.q, &ly.priv, &ly.pub, ly.out, out_dtype, 1, plan, true, ws, ws_bytes, cuda_stream);
+        spd_status rc = decode_step_impl(shape, ly.q, &ly.priv, &ly.pub, ly.out, out_dtype, 1, plan, i == 0, ws, ws_bytes,
+                                         cuda_stream, ly.k_new, ly.v_new);
         if (rc != SPD_OK) return rc;
     }
     return SPD_OK;

@@ -25,6 +25,7 @@ enum HdrWord {
     HDR_NSEQ = 3,          // sequences of the last call (size of the ticket array)
     HDR_SM_LAUNCHES = 4,   // attention launches that compared their CTAs' SMs with the previous launch's
     HDR_SM_MOVES = 5,      // CTAs of those launches that found themselves on another SM than last time
+    HDR_GRID_EXITS = 6,    // CTAs of the running launch that have finished (only counted by launches that append); zero between calls
     HDR_WORDS = 64
 };
 
@@ -90,6 +91,12 @@ struct Params {
     const float *in_o, *in_m, *in_l;  // OUT_FINAL: optional partial to merge in (may be null)
     void *out;              // OUT_FINAL destination
     int32_t out_bf16;
+    // optional append inside the launch (protocol step 3a): the new token's K and V rows, [B][Hkv][D] in the pools'
+    // dtype, go to position lens[u] of the public partition, which the launch reads as one token longer; the last
+    // CTA to finish adds one to the length of every user that was not flagged.  k_new == nullptr: no append.
+    const uint8_t *k_new, *v_new;
+    uint8_t *k_pool_w, *v_pool_w;   // the public pools, writable
+    int32_t *lens_w;                // the public seq_lens, writable
     // optional monitor: softmax mass on tokens [watch_lo[u], watch_hi[u]) of the private partition
     const int32_t *watch_lo, *watch_hi;   // [B]
     float *watch_out;                      // [B][Hq]; null = not watching

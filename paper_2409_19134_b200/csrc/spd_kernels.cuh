@@ -46,8 +46,9 @@ __device__ __forceinline__ bool user_tiles(const Params &p, int u, int &n0, int 
         const PartDev &pt = p.part[s];
         if (!pt.present) continue;
         const int64_t lo = pt.indptr[u], hi = pt.indptr[u + 1], end = pt.indptr[p.B];
-        const int64_t len = pt.lens[u];
-        if (lo < 0 || hi < lo || hi > end || len < 0 || len > (hi - lo) * kPage ||
+        const int64_t raw = pt.lens[u];
+        const int64_t len = raw + ((s == 1 && p.k_new != nullptr) ? 1 : 0);   // an appending launch counts the new token
+        if (lo < 0 || hi < lo || hi > end || raw < 0 || len > (hi - lo) * kPage ||
             (len > 0 && pt.indices == nullptr)) {
             bad = true;
         } else {
@@ -318,6 +319,8 @@ struct MathBF16 {
     static constexpr int kStages = SPD_BF16_STAGES;
     static constexpr int kExtraBytes = 0;
     static constexpr int KS = D / 16;
+    // byte offset, inside a K or V tile in shared memory, of 16-byte chunk c of token row r
+    __device__ static __forceinline__ int chunk_offset(int r, int c) { return (c >> 3) * kBoxBytes + r * 128 + (((c & 7) ^ (r & 7)) << 4); }
 
     struct State {
         uint32_t qf[KS][2];
@@ -463,6 +466,7 @@ struct MathBF16Simt {
     static constexpr int kStages = SPD_BF16_STAGES;
     static constexpr int kExtraBytes = (kHeadsPerItem * D + kHeadsPerItem * kPage) * 4;  // q (fp32), P
     static constexpr int V = D / 32;
+    __device__ static __forceinline__ int chunk_offset(int r, int c) { return (c >> 3) * kBoxBytes + r * 128 + (((c & 7) ^ (r & 7)) << 4); }
 
     struct State {
         float o[GE][V];
@@ -602,6 +606,7 @@ struct MathF32 {
     static constexpr int kStages = D == 128 ? 2 : 3;   // 16 KB per stage at head_dim 128
     static constexpr int kExtraBytes = (kHeadsPerItem * D + kHeadsPerItem * kPage) * 4;  // q, P
     static constexpr int V = D / 32;
+    __device__ static __forceinline__ int chunk_offset(int r, int c) { return r * D * 4 + c * 16; }
 
     struct State {
         float o[GE][V];
@@ -709,6 +714,30 @@ struct MathF32 {
 };
 
 // ------------------------------------------------------------------------------------------------
+// Append inside the attention launch (protocol step 3a; Fig. 3 step 2).  The tile that holds the new token has
+// just landed in shared memory with whatever the cache held at the token's slot; the warp overwrites that row of
+// K and of V with the new rows, so that the query attends to its own token, and -- one head group per KV head --
+// writes the same bytes through to the cache.  Other head groups of the KV head fetch the tile on their own
+// and patch their own copy, so nobody depends on when the write lands.
+template <class Math>
+__device__ __forceinline__ void append_row(const Params &p, uint8_t *Ks, uint8_t *Vs, int u, int sq, int slot, int page, int lane) {
+    constexpr int RB = Math::kTileBytes / kPage;     // bytes of one token row
+    constexpr int NCH = RB / 16;
+    const int kvh = sq / p.hgroups;
+    const bool writer = sq - kvh * p.hgroups == 0;
+    const int64_t src_row = (static_cast<int64_t>(u) * p.Hkv + kvh) * RB;
+    const int64_t dst_row = ((static_cast<int64_t>(page) * p.Hkv + kvh) * kPage + slot) * RB;
+    for (int i = lane; i < 2 * NCH; i += 32) {
+        const int which = i / NCH, c = i - which * NCH;
+        const uint4 val = *reinterpret_cast<const uint4 *>((which ? p.v_new : p.k_new) + src_row + c * 16);
+        *reinterpret_cast<uint4 *>((which ? Vs : Ks) + Math::chunk_offset(slot, c)) = val;
+        if (writer) *reinterpret_cast<uint4 *>((which ? p.v_pool_w : p.k_pool_w) + dst_row + c * 16) = val;
+    }
+    fence_proxy_async();
+    __syncwarp();
+}
+
+// ------------------------------------------------------------------------------------------------
 // Where a warp stands in the flattened tile stream.  Tiles are ordered by user, then sequence
 // (kv head x head group), then page; tile index = S * (tiles of earlier users) + sq * np + j.
 struct Cursor {
@@ -742,7 +771,7 @@ __device__ __forceinline__ void cursor_load_user(Cursor &c, const Params &p, con
     c.base0 = p.part[0].present ? p.part[0].indptr[c.u] : 0;
     c.base1 = p.part[1].present ? p.part[1].indptr[c.u] : 0;
     c.len0 = p.part[0].present ? p.part[0].lens[c.u] : 0;
-    c.len1 = p.part[1].present ? p.part[1].lens[c.u] : 0;
+    c.len1 = p.part[1].present ? p.part[1].lens[c.u] + (p.k_new != nullptr ? 1 : 0) : 0;
     c.key = -1;
 }
 
@@ -754,14 +783,14 @@ __device__ __forceinline__ int cursor_fetch_batch(const Cursor &c, const Params 
 }
 
 // Shared-memory carve-up behind the rings: mbarriers (8 B each), then the per-stage descriptors
-// (two int4 each, so 16-byte aligned), then each warp's private extra area (16-byte aligned).
+// (three int4 each, so 16-byte aligned), then each warp's private extra area (16-byte aligned).
 template <class Math>
 __host__ __device__ constexpr size_t attn_desc_offset() {
     return (static_cast<size_t>(Math::kWarps) * Math::kStages * 8 + 15) / 16 * 16;
 }
 template <class Math>
 __host__ __device__ constexpr size_t attn_extra_offset() {
-    return attn_desc_offset<Math>() + static_cast<size_t>(Math::kWarps) * Math::kStages * 32;
+    return attn_desc_offset<Math>() + static_cast<size_t>(Math::kWarps) * Math::kStages * 48;
 }
 template <class Math>
 __host__ __device__ constexpr size_t attn_bnd_offset() {
@@ -803,7 +832,7 @@ attn_kernel(const __grid_constant__ Params p, const __grid_constant__ CUtensorMa
     uint8_t *ring = base + static_cast<size_t>(wid) * NS * 2 * TB;
     uint8_t *tail = base + static_cast<size_t>(Math::kWarps) * NS * 2 * TB;
     uint64_t *bars = reinterpret_cast<uint64_t *>(tail) + wid * NS;
-    int4 *descs = reinterpret_cast<int4 *>(tail + attn_desc_offset<Math>()) + wid * NS * 2;
+    int4 *descs = reinterpret_cast<int4 *>(tail + attn_desc_offset<Math>()) + wid * NS * 3;
     uint8_t *extra = tail + attn_extra_offset<Math>() + static_cast<size_t>(wid) * Math::kExtraBytes;
 
     griddep_launch_dependents();   // the next kernel on the stream may begin its own read-only preamble
@@ -1097,9 +1126,11 @@ attn_kernel(const __grid_constant__ Params p, const __grid_constant__ CUtensorMa
         int kind = 0;
         if (last && !(seg_from0 && c.j == c.np - 1)) kind = seg_has_t0 ? 1 : 2;
         if (page < 0 || page >= p.part[part].num_pages) valid = 0;   // never fetched; flagged when consumed
+        const bool newtok = p.k_new != nullptr && part == 1 && jj == npart - 1;   // the tile that takes the appended row
         if (lane == 0) {
-            descs[2 * stage] = make_int4(valid, (first ? 1 : 0) | (last ? 2 : 0) | (kind << 8), c.u, c.sq);
-            descs[2 * stage + 1] = make_int4(c.np, c.j, cur_t, c.npp);
+            descs[3 * stage] = make_int4(valid, (first ? 1 : 0) | (last ? 2 : 0) | (newtok ? 4 : 0) | (kind << 8), c.u, c.sq);
+            descs[3 * stage + 1] = make_int4(c.np, c.j, cur_t, c.npp);
+            descs[3 * stage + 2] = make_int4(page, 0, 0, 0);
             const uint32_t bar = smem_u32(&bars[stage]);
             if (valid == 0) {
                 mbar_arrive(bar);
@@ -1147,10 +1178,11 @@ attn_kernel(const __grid_constant__ Params p, const __grid_constant__ CUtensorMa
     for (; i < n; ++i) {
         const int stage = i % NS;
         if (!mbar_wait(smem_u32(&bars[stage]), (i / NS) & 1)) { dead = true; break; }
-        const int4 d = descs[2 * stage];
+        const int4 d = descs[3 * stage];
         uint8_t *Ks = ring + static_cast<size_t>(stage) * 2 * TB, *Vs = Ks + TB;
         if (d.y & 1) { Math::begin(st, p, d.z, d.w, lane, extra); seg_bad = false; }
-        const int4 e = descs[2 * stage + 1];
+        const int4 e = descs[3 * stage + 1];
+        if ((d.y & 4) && d.x > 0) append_row<Math>(p, Ks, Vs, d.z, d.w, d.x - 1, descs[3 * stage + 2].x, lane);
         if (d.x > 0) {
             Math::tile(st, p, Ks, Vs, d.x, lane, extra, e.y < e.w ? e.y * kPage : -(1 << 30));
         } else {                                   // a page index outside the pool: flag the user, skip the tile
@@ -1189,7 +1221,8 @@ attn_kernel(const __grid_constant__ Params p, const __grid_constant__ CUtensorMa
 
     // ---- the CTA's last warp out leaves (weight, cycles) for the next call's shares -------------
     __syncwarp();
-    __threadfence_block();
+    __threadfence();      // this warp's flags and rows are visible before anybody can see it counted out
+    int last_cta = 0;
     if (lane == 0 && atomicAdd(&cta_exits, 1) == Math::kWarps - 1) {
         const int wa = blockIdx.x * Math::kWarps, wb = wa + Math::kWarps;
         const int tiles = (wb <= A ? bnd[wb] : T) - (wa <= A ? bnd[wa] : T);
@@ -1205,6 +1238,31 @@ attn_kernel(const __grid_constant__ Params p, const __grid_constant__ CUtensorMa
             if (blockIdx.x == 0) atomicAdd(&p.hdr[HDR_SM_LAUNCHES], 1);
         }
         p.plan[PLAN_SMID + blockIdx.x] = sm;
+        if (p.k_new != nullptr) {
+            __threadfence();
+            last_cta = atomicAdd(&p.hdr[HDR_GRID_EXITS], 1) == G - 1;
+        }
+    }
+    if (p.k_new == nullptr) return;
+    // ---- an appending launch: once every CTA has finished (nobody reads the lengths any more), the last warp out
+    // of the last CTA makes the new token count: length + 1 for every user that this call did not flag
+    last_cta = __shfl_sync(0xffffffffu, last_cta, 0);
+    if (!last_cta) return;
+    if (lane == 0) p.hdr[HDR_GRID_EXITS] = 0;
+    __threadfence();
+    for (int base = 0; base < p.B; base += 256) {
+        int32_t fl[8], ln[8];
+#pragma unroll
+        for (int k = 0; k < 8; ++k) {
+            const int u = base + k * 32 + lane;
+            fl[k] = u < p.B ? __ldcg(p.bad + u) : p.epoch;
+            ln[k] = u < p.B ? __ldcg(p.lens_w + u) : 0;
+        }
+#pragma unroll
+        for (int k = 0; k < 8; ++k) {
+            const int u = base + k * 32 + lane;
+            if (u < p.B && fl[k] != p.epoch) p.lens_w[u] = ln[k] + 1;
+        }
     }
 }
 

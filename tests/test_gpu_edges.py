@@ -215,6 +215,76 @@ def test_append_kv_is_bit_exact_and_feeds_the_next_step(dtype):
     assert_close(out.cpu().numpy(), orc.full(q, kin, kout, w.sm_scale), w.dtype, "decode after append")
 
 
+@pytest.mark.parametrize("dtype,hq,hkv,d", [("bf16", 8, 4, 128), ("f32", 8, 4, 128), ("bf16", 32, 2, 128), ("bf16", 4, 4, 64), ("f32", 16, 2, 64)])
+def test_append_inside_the_decode_launch(dtype, hq, hkv, d):
+    """Steps 3a to 3c in one launch: the new rows reach the cache bit for bit, the lengths grow by one, and the
+    output is the attention over the grown cache -- on page boundaries, for an empty public partition, with group
+    sizes that split a KV head over several warps (16 query heads per KV head), twice in a row on a stored plan.
+    A user whose listed pages are full gets zeros, no append and an unchanged length."""
+    rng = np.random.default_rng(151)
+    B = 7
+    lout = np.array([0, 15, 16, 31, 5, 47, 32])        # the append lands at slot 0, 15, 0 (new page), 15, 5, 15, 0 (no room)
+    lin = rng.integers(1, 260, size=B)
+    lin[2] = 2900                                       # one long prompt: its sequence is cut into pieces
+    cfg = dict(name="append_fused", batch=B, hq=hq, hkv=hkv, d=d, dtype=dtype, lin=("const", 0), lout=("const", 0), seed=152)
+    w = wl.make_workload(cfg, lengths=(lin, lout), slack=False, over_alloc=2.0)
+    need = (lout + 15) // 16
+    cap = need + 1
+    cap[-1] = need[-1]                                  # the last user's pages are exactly full
+    used = set(w.pub.page_indices.tolist())
+    free = iter(sorted(set(range(w.pub.num_pages)) - used))
+    indices, indptr = [], [0]
+    for u in range(B):
+        own = w.pub.page_indices[int(w.pub.page_indptr[u]):int(w.pub.page_indptr[u + 1])].tolist()
+        while len(own) < cap[u]:
+            own.append(next(free))
+        indices += own
+        indptr.append(len(indices))
+    w.pub.page_indptr = torch.tensor(indptr, dtype=torch.int32)
+    w.pub.page_indices = torch.tensor(indices, dtype=torch.int32)
+    q, kin, kout = oracle_inputs(w)
+    wg = w.to("cuda")
+    shape = spd.make_shape(B, hq, hkv, d, w.dtype, w.sm_scale)
+    ws = spd.alloc_workspace(shape)
+    gen = torch.Generator().manual_seed(153)
+
+    def bits(t):
+        return t.cpu().view(torch.int16 if t.dtype == torch.bfloat16 else torch.int32).numpy()
+
+    for step, plan in enumerate((spd.SPD_PLAN_PER_CALL, spd.SPD_PLAN_STORE)):
+        k_new = torch.randn((B, hkv, d), generator=gen).to(w.dtype)
+        v_new = torch.randn((B, hkv, d), generator=gen).to(w.dtype)
+        done = orc.append(kout, orc.q_from_torch(k_new), orc.q_from_torch(v_new))
+        ref = orc.full(q, kin, kout, w.sm_scale)
+        out = torch.full((B, hq, d), float("nan"), dtype=torch.float32, device="cuda")
+        spd.spd_decode_step_append(shape, wg.q, k_new.cuda(), v_new.cuda(), wg.priv, wg.pub, out, ws, plan=plan)
+        full = [u for u in range(B) if not done[u]]
+        status = spd.spd_query_device_status(ws)
+        assert status == ((4, full[0]) if full else (spd.SPD_OK, -1)), (step, status)
+        assert np.array_equal(wg.pub.seq_lens.cpu().numpy(), kout.seq_lens), f"lengths after append {step}"
+        assert np.array_equal(bits(wg.pub.k_pool), kout.k_pool.view(bits(wg.pub.k_pool).dtype)), f"K cache after append {step}"
+        assert np.array_equal(bits(wg.pub.v_pool), kout.v_pool.view(bits(wg.pub.v_pool).dtype)), f"V cache after append {step}"
+        ok = [u for u in range(B) if done[u]]
+        assert bool((out[full] == 0).all())
+        assert_close(out[ok].cpu().numpy(), ref[ok], w.dtype, f"attention over the grown cache, step {step}")
+    # the stored plan serves another cache with the lengths this one had before the storing call's append
+    # (same arrays moved back by one), values of the rows that are appended again differ
+    wg.pub.seq_lens.copy_(torch.clamp(wg.pub.seq_lens - 1, min=0))
+    kout.seq_lens[:] = np.maximum(kout.seq_lens - 1, 0)
+    wg.pub.seq_lens[-1] = int(lout[-1]); kout.seq_lens[-1] = int(lout[-1])     # the full user never moved
+    k_new = torch.randn((B, hkv, d), generator=gen).to(w.dtype)
+    v_new = torch.randn((B, hkv, d), generator=gen).to(w.dtype)
+    done = orc.append(kout, orc.q_from_torch(k_new), orc.q_from_torch(v_new))
+    ref = orc.full(q, kin, kout, w.sm_scale)
+    out = torch.full((B, hq, d), float("nan"), dtype=torch.float32, device="cuda")
+    spd.spd_decode_step_append(shape, wg.q, k_new.cuda(), v_new.cuda(), wg.priv, wg.pub, out, ws, plan=spd.SPD_PLAN_REUSE)
+    assert spd.spd_query_device_status(ws)[0] == 4
+    ok = [u for u in range(B) if done[u]]
+    assert np.array_equal(wg.pub.seq_lens.cpu().numpy(), kout.seq_lens)
+    assert np.array_equal(bits(wg.pub.k_pool), kout.k_pool.view(bits(wg.pub.k_pool).dtype))
+    assert_close(out[ok].cpu().numpy(), ref[ok], w.dtype, "append on a reused plan")
+
+
 @pytest.mark.parametrize("name", ["bf16_gqa4_d128", "bf16_gqa8_d128", "bf16_long_split", "f32_mha_d64", "f32_long_split"])
 def test_watched_attention_mass(name):
     """The input-attention monitor: softmax mass on a watched range of the private partition."""

@@ -93,7 +93,7 @@ def test_cuda_graph_replay(name):
 
 @pytest.mark.parametrize("dtype", ["bf16", "f32"])
 def test_token_step_over_layers_eager_and_as_one_graph(dtype):
-    """Step 3 for every layer of a model in one call: per layer the append, then the fused decode step.  Run once
+    """Step 3 for every layer of a model in one call: per layer the append and the fused decode step.  Run once
     eagerly, then captured in a CUDA graph and replayed twice; after every run each layer's output, cache and
     lengths must be what the oracle gets from the same number of appends."""
     n_layers, B, hq, hkv, d = 3, 5, 8, 2, 128
@@ -133,7 +133,7 @@ def test_token_step_over_layers_eager_and_as_one_graph(dtype):
 
     launches = spd.spd_kernel_launch_count()
     spd.spd_token_step(shape, layers_gpu, ws)
-    assert spd.spd_kernel_launch_count() - launches == 2 * n_layers
+    assert spd.spd_kernel_launch_count() - launches == n_layers      # append and attention share a launch
     check("eager")
     graph = torch.cuda.CUDAGraph()
     with torch.cuda.graph(graph):
