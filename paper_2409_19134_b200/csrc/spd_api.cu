@@ -39,14 +39,28 @@ std::atomic<int> g_min_tiles{kMinTilesPerWarp};   // fewest page tiles a share o
 std::atomic<int> g_uniform_shares{0};             // 1 = equal shares, the measured rates are ignored
 std::atomic<int> g_pdl{-1};                       // programmatic launch: -1 = not decided yet (environment), 0 off, 1 on
 
-// Attention launches made so far on each workspace (keyed by its address).  The kernel rotates through the three
-// thirds of the workspace's rate table by this count, so it must advance by exactly one per attention launch on
-// that workspace whatever else the process launches in between.
-uint32_t next_rate_sel(const void *ws) {
+// What the host remembers about a workspace (keyed by its address): the attention launches made on it so far, and
+// at which of them each kind of call last stored its plan.  The kernel rotates through the three thirds of the
+// workspace's rate table by the launch count, so it must advance by exactly one per attention launch on that
+// workspace whatever else the process launches in between.
+struct WsHostState {
+    uint64_t launches = 0;
+    uint64_t stored_at[3] = {~0ull, ~0ull, ~0ull};
+};
+
+// Registers one attention launch.  *early_plan: a launch that loads a stored plan may read it before the
+// previous kernel on the stream has finished when that kernel is not the one that stored it (the launch before
+// the previous one has left every SM by the time this one starts, since each CTA takes a whole SM).
+uint32_t register_launch(const void *ws, int slot, int plan_mode, bool *early_plan) {
     static std::mutex mu;
-    static std::unordered_map<const void *, uint32_t> count;
+    static std::unordered_map<const void *, WsHostState> table;
     std::lock_guard<std::mutex> lock(mu);
-    return count[ws]++ % 3u;
+    WsHostState &st = table[ws];
+    const uint64_t n = st.launches++;
+    *early_plan = plan_mode == PLAN_LOAD && st.stored_at[slot] != ~0ull && n >= st.stored_at[slot] + 2;
+    if (plan_mode == PLAN_DERIVE_STORE) st.stored_at[slot] = n;
+    if (plan_mode == PLAN_DERIVE) st.stored_at[slot] = ~0ull;
+    return static_cast<uint32_t>(n % 3u);
 }
 
 bool programmatic_launch() {
@@ -208,7 +222,9 @@ spd_status launch_attn(const Params &p_in, const CUtensorMap *maps, int sms, cud
     if (sms > kMaxGrid) return SPD_ERR_UNSUPPORTED;
     Params p = p_in;
     p.num_warps = sms * Math::kWarps;   // the plan cuts the tile stream into one share per warp of THIS grid
-    const size_t smem = attn_smem_bytes<Math>(sms);
+    // At least 117 KB, so that an SM never holds two of these CTAs whatever the variant needs: the kernel's
+    // reasoning about which launch can still be running when the next but one starts rests on one CTA per SM.
+    const size_t smem = attn_smem_bytes<Math>(sms) > 117 * 1024 ? attn_smem_bytes<Math>(sms) : 117 * 1024;
     static std::once_flag once[64];
     int dev = 0;
     cudaGetDevice(&dev);
@@ -251,6 +267,7 @@ struct Job {
     int plan_mode;                 // PlanMode: derive per call (default), derive and store, or load the stored plan
     bool plain_order;              // launch in plain stream order (an input was written by the kernel just before)
     const void *k_new, *v_new;     // optional append of the new token's rows to part[1] inside the launch
+    bool wait_first;               // read nothing before the previous kernel on the stream has finished, not even a stored plan
 };
 
 // The stored plan of a call is tagged with what it was cut for besides the lengths, so that a launch told to load a
@@ -288,11 +305,13 @@ spd_status run_job(const Job &job, void *ws, size_t ws_bytes, void *stream) {
     p.bad = reinterpret_cast<int32_t *>(w + L.bad);
     p.tickets = reinterpret_cast<int32_t *>(w + L.tickets);
     p.rates = reinterpret_cast<float2 *>(w + L.rates);
-    p.rate_sel = static_cast<int32_t>(next_rate_sel(ws));       // this workspace's launches rotate through the three thirds
-    p.min_tiles = g_min_tiles.load();
-    p.uniform = g_uniform_shares.load();
     const int slot = (job.part[0] ? 1 : 0) + (job.part[1] ? 2 : 0) - 1;   // one stored plan per kind of call
     if (slot < 0) return SPD_ERR_INVALID_ARG;
+    bool early_plan = false;
+    p.rate_sel = static_cast<int32_t>(register_launch(ws, slot, job.plan_mode, &early_plan));   // rotates through the thirds
+    p.plan_early = early_plan && !job.wait_first ? 1 : 0;
+    p.min_tiles = g_min_tiles.load();
+    p.uniform = g_uniform_shares.load();
     p.plan = reinterpret_cast<int32_t *>(w + L.plan + slot * kPlanBytes);
     p.plan_mode = job.plan_mode;
     p.plan_tag = plan_tag_of(s, p.min_tiles, p.uniform);
@@ -429,7 +448,7 @@ static spd_status service_attn_merge_impl(const spd_shape *shape, const void *q,
 static spd_status decode_step_impl(const spd_shape *shape, const void *q, const spd_paged_kv *priv,
                                    const spd_paged_kv *pub, void *out, spd_dtype out_dtype, int32_t fused, int plan,
                                    bool plain_order, void *ws, size_t ws_bytes, void *cuda_stream,
-                                   const void *k_new = nullptr, const void *v_new = nullptr) {
+                                   const void *k_new = nullptr, const void *v_new = nullptr, bool wait_first = false) {
     spd_status rc = check_shape(shape);
     if (rc != SPD_OK) return rc;
     if ((rc = check_kv(shape, priv)) != SPD_OK) return rc;
@@ -444,6 +463,7 @@ static spd_status decode_step_impl(const spd_shape *shape, const void *q, const 
         job.plan_mode = plan;
         job.plain_order = plain_order;
         job.k_new = k_new; job.v_new = v_new;
+        job.wait_first = wait_first;
         return run_job(job, ws, ws_bytes, cuda_stream);
     }
     if (k_new) return SPD_ERR_UNSUPPORTED;      // the append rides on the fused step only
@@ -497,11 +517,10 @@ spd_status spd_decode_step_append(const spd_shape *shape, const void *q, const v
                                   const spd_paged_kv *priv, const spd_paged_kv *pub, void *out, spd_dtype out_dtype,
                                   spd_plan_mode plan, void *ws, size_t ws_bytes, void *cuda_stream) {
     if (check_plan(plan) != SPD_OK || !k_new || !v_new) return SPD_ERR_INVALID_ARG;
-    // A launch that derives its plan reads the lengths before the previous kernel on the stream has finished, and
-    // that kernel may be the previous call of this very function, which adds one to them as its last act: plain
-    // stream order.  A launch that loads its plan waits first anyway.
-    return decode_step_impl(shape, q, priv, pub, out, out_dtype, 1, plan, plan != SPD_PLAN_REUSE, ws, ws_bytes,
-                            cuda_stream, k_new, v_new);
+    // The kernel before this one on the stream may be the previous call of this very function on the same cache,
+    // which adds one to the lengths as its last act: nothing is read before that kernel has finished.
+    return decode_step_impl(shape, q, priv, pub, out, out_dtype, 1, plan, true, ws, ws_bytes, cuda_stream, k_new, v_new,
+                            true);
 }
 
 spd_status spd_decode_step_planned(const spd_shape *shape, const void *q, const spd_paged_kv *priv,

@@ -81,6 +81,7 @@ struct Params {
                             // reads (rate_sel + 1) % 3
     int32_t *plan;          // [PLAN_WORDS] the stored plan
     int32_t plan_mode;      // PlanMode
+    int32_t plan_early;     // PLAN_LOAD: the plan may be read before the previous kernel on the stream has finished
     int32_t plan_tag;       // what PLAN_TAG must hold for a plan to be loaded / holds once this launch has stored one
     int32_t min_tiles;      // fewest tiles a share may hold (>= 1)
     int32_t uniform;        // non-zero: equal shares, the rate table is ignored

@@ -150,12 +150,15 @@ __device__ __forceinline__ int warp_of_tile(const int32_t *bnd, int A, int t) {
 
 // Recombine the pieces that warps w_first..w_last left for one sequence (Theorem 1 applied n-ways,
 // every piece brought to the common maximum) and finalise it.  Run by the warp that delivered the
-// last piece.  Pieces are read past L1 (other SMs wrote them).  Lane c of a batch looks after the
-// (m, l) of piece c; the O rows are fetched 16 at a time so that the loads overlap.
+// last piece.  Pieces are read past L1 (other SMs wrote them).  Lane c of a block of 32 pieces looks after the
+// (m, l) of piece c; the O rows are fetched 16 at a time.  Every load here is a round trip to L2 on the critical
+// path of a small call, so the first 16 O rows, the (m, l) values and the user's flag are requested together,
+// before anything waits for any of them.
 template <int D, int GE>
 __device__ __noinline__ void merge_pieces(const Params &p, int u, int sq, int w_first, int w_last, const int32_t *bnd,
                                           int s0, int lane, bool bad) {
     constexpr int V = D / 32, H = kHeadsPerItem, PB = 16 / GE;   // PB pieces per batch of loads
+    const int32_t flag = __ldcg(p.bad + u);      // used at the very end: was the user flagged by anybody during this call?
     float M[GE], L[GE], LW[GE], o[GE][V];
 #pragma unroll
     for (int hh = 0; hh < GE; ++hh) {
@@ -165,8 +168,28 @@ __device__ __noinline__ void merge_pieces(const Params &p, int u, int sq, int w_
 #pragma unroll
         for (int i = 0; i < V; ++i) o[hh][i] = 0.f;
     }
+    float x[PB][GE][V];
+    auto load_rows = [&](int b0, int nb, int c0) {     // O rows of pieces [c0, c0 + PB) of the block that starts at warp b0
+#pragma unroll
+        for (int k = 0; k < PB; ++k) {
+            const int c = c0 + k;
+            const bool live = c < nb && bnd[b0 + c + 1] > bnd[b0 + c];
+            const float *src = piece_slot(p, D, live ? b0 + c : b0, bnd, s0) + lane * V;
+#pragma unroll
+            for (int hh = 0; hh < GE; ++hh) {
+                if constexpr (V == 4) {
+                    const float4 t = live ? __ldcg(reinterpret_cast<const float4 *>(src + hh * D)) : make_float4(0.f, 0.f, 0.f, 0.f);
+                    x[k][hh][0] = t.x; x[k][hh][1] = t.y; x[k][hh][2] = t.z; x[k][hh][3] = t.w;
+                } else {
+                    const float2 t = live ? __ldcg(reinterpret_cast<const float2 *>(src + hh * D)) : make_float2(0.f, 0.f);
+                    x[k][hh][0] = t.x; x[k][hh][1] = t.y;
+                }
+            }
+        }
+    };
     for (int b0 = w_first; b0 <= w_last; b0 += 32) {
         const int nb = min(32, w_last - b0 + 1);
+        load_rows(b0, nb, 0);
         const bool mine = lane < nb && bnd[b0 + lane + 1] > bnd[b0 + lane];   // warps with an empty share left nothing
         const float *ms = piece_slot(p, D, mine ? b0 + lane : b0, bnd, s0) + H * D;
         float wgt[GE];
@@ -194,23 +217,7 @@ __device__ __noinline__ void merge_pieces(const Params &p, int u, int sq, int w_
             for (int i = 0; i < V; ++i) o[hh][i] *= resc;
         }
         for (int c0 = 0; c0 < nb; c0 += PB) {
-            float x[PB][GE][V];
-#pragma unroll
-            for (int k = 0; k < PB; ++k) {
-                const int c = c0 + k;
-                const bool live = c < nb && bnd[b0 + c + 1] > bnd[b0 + c];
-                const float *src = piece_slot(p, D, live ? b0 + c : b0, bnd, s0) + lane * V;
-#pragma unroll
-                for (int hh = 0; hh < GE; ++hh) {
-                    if constexpr (V == 4) {
-                        const float4 t = live ? __ldcg(reinterpret_cast<const float4 *>(src + hh * D)) : make_float4(0.f, 0.f, 0.f, 0.f);
-                        x[k][hh][0] = t.x; x[k][hh][1] = t.y; x[k][hh][2] = t.z; x[k][hh][3] = t.w;
-                    } else {
-                        const float2 t = live ? __ldcg(reinterpret_cast<const float2 *>(src + hh * D)) : make_float2(0.f, 0.f);
-                        x[k][hh][0] = t.x; x[k][hh][1] = t.y;
-                    }
-                }
-            }
+            if (c0 > 0) load_rows(b0, nb, c0);
 #pragma unroll
             for (int k = 0; k < PB; ++k) {
                 const int c = (c0 + k) & 31;
@@ -224,6 +231,7 @@ __device__ __noinline__ void merge_pieces(const Params &p, int u, int sq, int w_
         }
     }
     const int hbase = first_head(p, sq);
+    bad = bad || flag == p.epoch;
 #pragma unroll
     for (int hh = 0; hh < GE; ++hh) finalize_store<D>(p, u, hbase + hh, o[hh], M[hh], L[hh], lane, bad, LW[hh]);
 }
@@ -291,12 +299,11 @@ __device__ __forceinline__ void piece_ticket(const Params &p, const PieceInfo &p
     if (ticket != pieces - 1) return;         // other pieces are still to come
     __threadfence();
     if (lane == 0) *counter = 0;              // everybody has drawn: ready for the next call
-    const bool bad = pp.bad || (__ldcg(p.bad + pp.u) == p.epoch);
-    switch (p.geff) {
-        case 1: merge_pieces<D, 1>(p, pp.u, pp.sq, w_first, w_last, bnd, pp.s0, lane, bad); break;
-        case 2: merge_pieces<D, 2>(p, pp.u, pp.sq, w_first, w_last, bnd, pp.s0, lane, bad); break;
-        case 4: merge_pieces<D, 4>(p, pp.u, pp.sq, w_first, w_last, bnd, pp.s0, lane, bad); break;
-        default: merge_pieces<D, 8>(p, pp.u, pp.sq, w_first, w_last, bnd, pp.s0, lane, bad); break;
+    switch (p.geff) {      // the user's flag (raised by anybody during this call) is looked up inside, with the pieces
+        case 1: merge_pieces<D, 1>(p, pp.u, pp.sq, w_first, w_last, bnd, pp.s0, lane, pp.bad); break;
+        case 2: merge_pieces<D, 2>(p, pp.u, pp.sq, w_first, w_last, bnd, pp.s0, lane, pp.bad); break;
+        case 4: merge_pieces<D, 4>(p, pp.u, pp.sq, w_first, w_last, bnd, pp.s0, lane, pp.bad); break;
+        default: merge_pieces<D, 8>(p, pp.u, pp.sq, w_first, w_last, bnd, pp.s0, lane, pp.bad); break;
     }
 }
 
@@ -959,9 +966,10 @@ attn_kernel(const __grid_constant__ Params p, const __grid_constant__ CUtensorMa
     __syncthreads();
     } else {
     // ---- plan loaded: an earlier launch on this stream and workspace, over the same lengths, left its share
-    // boundaries, the CTA weights and every warp's starting point in the workspace.  It has completed, and its
-    // writes are visible, once the wait below returns.
-        griddep_wait();
+    // boundaries, the CTA weights and every warp's starting point in the workspace.  If that launch is the previous
+    // kernel on the stream it has completed, and its writes are visible, once the wait below returns; an older one
+    // had left every SM before this launch could start.
+        if (!p.plan_early) griddep_wait();
         const int32_t *pl = p.plan;
         T = __ldcg(pl + PLAN_T);
         A = __ldcg(pl + PLAN_A);
@@ -1064,6 +1072,7 @@ attn_kernel(const __grid_constant__ Params p, const __grid_constant__ CUtensorMa
                 }
             }
             if (p.plan_mode == PLAN_DERIVE_STORE && n > 0 && lane < 8) pl[PLAN_REC + gwarp * 8 + lane] = rec;
+            __threadfence();
         }
         // users that own no tile (nothing cached, or tables inconsistent): written and flagged here
         if (plan_ok)
