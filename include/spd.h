@@ -194,6 +194,18 @@ spd_status spd_decode_step_watch(const spd_shape *shape, const void *q, const sp
                                  const spd_watch *watch, void *ws, size_t ws_bytes, void *cuda_stream);
 
 /*
+ * The decision on top of the monitor (Sec. 2.4.4: an attack is detected whenever the monitored attention score
+ * falls below an empirical threshold; the distraction effect shows in some specific heads).  HOST arrays only, no
+ * device work: mass [batch][num_q_heads] is what a *_watch call produced, copied to the host by the caller;
+ * head_mask [num_q_heads] (may be NULL = all heads) selects the heads that are watched; score[u] (may be NULL)
+ * receives the mean of mass[u][h] over the selected heads and alarm[u] is set to 1 where that mean is below
+ * `threshold`, else 0.  A user with no selected head, or a non-finite mean, raises the alarm.  Returns
+ * SPD_ERR_INVALID_ARG for null mass or alarm, non-positive sizes or a threshold that is not a number.
+ */
+spd_status spd_watch_alarm(const float *mass, int32_t batch, int32_t num_q_heads, const uint8_t *head_mask,
+                           float threshold, int32_t *alarm, float *score);
+
+/*
  * Prefill (protocol step 2; Fig. 3 step 0): causal self-attention over every user's prompt, and the
  * hand-over of the prompt's K and V rows to the private paged cache that the decode calls read.
  *   q [total_tokens][num_q_heads][head_dim], k, v [total_tokens][num_kv_heads][head_dim]: the prompts of

@@ -27,7 +27,7 @@ EXPORTS = ["spd_workspace_size", "spd_partial_attn", "spd_service_attn_merge", "
            "spd_partial_attn_watch", "spd_decode_step_watch", "spd_set_bf16_math", "spd_merge_partials", "spd_prefill_attn",
            "spd_set_prefill_rows", "spd_token_step", "spd_partial_attn_planned", "spd_service_attn_merge_planned",
            "spd_decode_step_planned", "spd_set_split", "spd_set_programmatic_launch", "spd_debug_read_plan",
-           "spd_debug_sm_moves", "spd_decode_step_append"]
+           "spd_debug_sm_moves", "spd_decode_step_append", "spd_watch_alarm"]
 
 
 class SpdError(RuntimeError):
@@ -106,6 +106,7 @@ def lib() -> C.CDLL:
                                               C.c_int32, C.c_int, vp, sz, vp]
         L.spd_decode_step_append.argtypes = [C.POINTER(Shape), vp, vp, vp, C.POINTER(PagedKV), C.POINTER(PagedKV), vp, C.c_int,
                                              C.c_int, vp, sz, vp]
+        L.spd_watch_alarm.argtypes = [vp, C.c_int32, C.c_int32, vp, C.c_float, vp, vp]
         L.spd_set_split.argtypes = [C.c_int32, C.c_int32]
         L.spd_set_programmatic_launch.argtypes = [C.c_int32]
         L.spd_debug_read_plan.argtypes = [vp, C.c_int32, vp, C.POINTER(C.c_int32), C.POINTER(C.c_int32),
@@ -362,6 +363,20 @@ def spd_decode_step_watch(shape, q, priv, pub, out, tok_lo, tok_hi, watch_out, w
     _check(lib().spd_decode_step_watch(C.byref(shape), q.data_ptr(), C.byref(a), C.byref(b), out.data_ptr(),
                                        _dtype_code(out.dtype), C.byref(w), ws.data_ptr(), ws.numel(),
                                        _stream_ptr(stream)), "spd_decode_step_watch")
+
+
+def spd_watch_alarm(mass, threshold: float, head_mask=None):
+    """mass: float32 HOST tensor [batch, heads] from a *_watch call; head_mask: optional bool/uint8 [heads].
+    Returns (alarm int32 [batch], score float32 [batch]): score = mean watched mass over the selected heads,
+    alarm = 1 where it is below the threshold."""
+    assert mass.device.type == "cpu" and mass.dtype == torch.float32 and mass.is_contiguous() and mass.dim() == 2
+    B, H = mass.shape
+    alarm = torch.zeros(B, dtype=torch.int32)
+    score = torch.zeros(B, dtype=torch.float32)
+    hm = None if head_mask is None else head_mask.to(torch.uint8).contiguous()
+    _check(lib().spd_watch_alarm(mass.data_ptr(), B, H, None if hm is None else hm.data_ptr(), float(threshold),
+                                 alarm.data_ptr(), score.data_ptr()), "spd_watch_alarm")
+    return alarm, score
 
 
 def spd_set_bf16_math(path: int) -> None:

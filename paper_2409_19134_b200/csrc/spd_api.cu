@@ -568,6 +568,21 @@ spd_status spd_decode_step_watch(const spd_shape *shape, const void *q, const sp
     return run_job(job, ws, ws_bytes, cuda_stream);
 }
 
+spd_status spd_watch_alarm(const float *mass, int32_t batch, int32_t num_q_heads, const uint8_t *head_mask, float threshold,
+                           int32_t *alarm, float *score) {
+    if (!mass || !alarm || batch <= 0 || num_q_heads <= 0 || !(threshold == threshold)) return SPD_ERR_INVALID_ARG;
+    for (int32_t u = 0; u < batch; ++u) {
+        double sum = 0.0;
+        int32_t n = 0;
+        for (int32_t h = 0; h < num_q_heads; ++h)
+            if (!head_mask || head_mask[h]) { sum += mass[static_cast<size_t>(u) * num_q_heads + h]; ++n; }
+        const double mean = n ? sum / n : 0.0;
+        if (score) score[u] = static_cast<float>(mean);
+        alarm[u] = (n == 0 || !(mean >= static_cast<double>(threshold))) ? 1 : 0;     // NaN compares false: alarm
+    }
+    return SPD_OK;
+}
+
 // [T][H][128] bf16 as a 3-D tensor map; one box = `rows` tokens x 64 channels of one head, 128-byte swizzle.
 static spd_status make_prompt_map(CUtensorMap *map, const void *ptr, int64_t T, int heads, int rows) {
     EncodeTiledFn fn = encode_fn();

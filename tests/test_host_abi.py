@@ -89,6 +89,26 @@ def test_bad_arguments_are_rejected_on_the_host(lib):
     assert lib.spd_set_bf16_math(2) == 1
 
 
+def test_watch_alarm_thresholds_the_mean_over_the_watched_heads(lib):
+    """Sec. 2.4.4: an attack is detected whenever the monitored attention score falls below a threshold."""
+    mass = torch.tensor([[0.50, 0.10, 0.30, 0.10],      # mean 0.25 over all heads, 0.40 over heads 0 and 2
+                         [0.05, 0.90, 0.01, 0.90],      # mean 0.465 over all, 0.03 over heads 0 and 2
+                         [0.20, 0.20, 0.20, 0.20],
+                         [float("nan"), 0.9, 0.9, 0.9]], dtype=torch.float32)
+    alarm, score = spd.spd_watch_alarm(mass, 0.25)
+    assert alarm.tolist() == [0, 0, 1, 1]                # 0.25 is not below 0.25; NaN raises the alarm
+    assert torch.allclose(score[:3], torch.tensor([0.25, 0.465, 0.20]), atol=1e-7)
+    alarm, score = spd.spd_watch_alarm(mass, 0.25, head_mask=torch.tensor([1, 0, 1, 0]))
+    assert alarm.tolist() == [0, 1, 1, 1]
+    assert torch.allclose(score[:3], torch.tensor([0.40, 0.03, 0.20]), atol=1e-7)
+    alarm, _ = spd.spd_watch_alarm(mass, 0.0, head_mask=torch.zeros(4))
+    assert alarm.tolist() == [1, 1, 1, 1]                # nothing watched: nothing vouches for the user
+    a = (C.c_int32 * 4)()
+    assert lib.spd_watch_alarm(None, 4, 4, None, 0.1, a, None) == 1
+    assert lib.spd_watch_alarm(mass.data_ptr(), 0, 4, None, 0.1, a, None) == 1
+    assert lib.spd_watch_alarm(mass.data_ptr(), 4, 4, None, float("nan"), a, None) == 1
+
+
 def test_binding_fails_loudly_without_the_library(monkeypatch):
     monkeypatch.setattr(spd, "_lib", None)
     monkeypatch.setattr(spd, "LIB_PATH", "/nonexistent/libspd.so")
