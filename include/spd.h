@@ -219,8 +219,10 @@ spd_status spd_watch_alarm(const float *mass, int32_t batch, int32_t num_q_heads
  *   tok_indptr must be non-decreasing and end at total_tokens; where it is not, the users before the first
  *   inconsistent one are served, the rows of that user and of all later ones are left unwritten, and the
  *   same status is raised.  Nothing is read or written out of bounds either way.
- * Supported: BF16, head_dim 128, sm_scale > 0 (else SPD_ERR_UNSUPPORTED).  Two kernels on `cuda_stream`:
- * the copy into the cache and the attention (tcgen05 tensor-core MMAs with accumulators in tensor memory).
+ * Supported: every shape the decode calls take, with sm_scale > 0 (else SPD_ERR_UNSUPPORTED).  Two kernels on
+ * `cuda_stream`: the copy into the cache and the attention -- for BF16 with head_dim 128 on the tensor cores
+ * (tcgen05 MMAs with accumulators in tensor memory), for FP32 prompts and for head_dim 64 on the FMA pipes (fp32
+ * arithmetic throughout; a correctness path, not a fast one).
  */
 spd_status spd_prefill_attn(const spd_shape *shape, int64_t total_tokens, const void *q, const void *k,
                             const void *v, const int32_t *tok_indptr, void *k_pool, void *v_pool,
@@ -386,8 +388,9 @@ spd_status spd_set_bf16_math(int32_t path);
 /*
  * Tuning and test aid (no counterpart in the paper): query rows per CTA of spd_prefill_attn from now on,
  * process-wide.  0 (default) = chosen per call from the mean prompt length (256 rows, two tiles sharing
- * their K/V loads, from 768 tokens on, else 128); 128 or 256 force one kernel.  Both compute the same
- * thing within tolerance.
+ * their K/V loads, from 768 tokens on, else 128); 128 or 256 force one tensor-core kernel; 8 forces the FMA-pipe
+ * kernel (the one FP32 and head_dim 64 always take) for BF16 with head_dim 128 too.  All compute the same thing
+ * within tolerance.
  */
 spd_status spd_set_prefill_rows(int32_t rows);
 

@@ -13,6 +13,7 @@
 #include "spd_kernels.cuh"
 #include "spd_prefill.cuh"
 #include "spd_prefill_pair.cuh"
+#include "spd_prefill_fma.cuh"
 
 namespace {
 
@@ -603,8 +604,7 @@ spd_status spd_prefill_attn(const spd_shape *shape, int64_t total_tokens, const 
                             spd_dtype out_dtype, void *ws, size_t ws_bytes, void *cuda_stream) {
     spd_status rc = check_shape(shape);
     if (rc != SPD_OK) return rc;
-    if (shape->dtype != SPD_BF16 || shape->head_dim != 128) return SPD_ERR_UNSUPPORTED;
-    if (!(shape->sm_scale > 0.f)) return SPD_ERR_UNSUPPORTED;   // the kernels take row maxima before scaling
+    if (!(shape->sm_scale > 0.f)) return SPD_ERR_UNSUPPORTED;   // the tensor-core kernels take row maxima before scaling
     if (out_dtype != SPD_F32 && out_dtype != SPD_BF16) return SPD_ERR_UNSUPPORTED;
     if (total_tokens < 0 || total_tokens >= (1ll << 31) - kPfBlock) return SPD_ERR_INVALID_ARG;
     if (!tok_indptr || !page_indptr || !seq_lens || !ws || misaligned(ws, 256)) return SPD_ERR_INVALID_ARG;
@@ -619,7 +619,8 @@ spd_status spd_prefill_attn(const spd_shape *shape, int64_t total_tokens, const 
     const int64_t T = total_tokens;
 
     PromptKvParams kp;
-    kp.B = shape->batch; kp.Hkv = shape->num_kv_heads; kp.row_bytes = 128 * 2; kp.T = T;
+    kp.B = shape->batch; kp.Hkv = shape->num_kv_heads; kp.T = T;
+    kp.row_bytes = shape->head_dim * (shape->dtype == SPD_BF16 ? 2 : 4);
     kp.k = static_cast<const uint8_t *>(k); kp.v = static_cast<const uint8_t *>(v); kp.tok_indptr = tok_indptr;
     kp.k_pool = static_cast<uint8_t *>(k_pool); kp.v_pool = static_cast<uint8_t *>(v_pool); kp.num_pages = num_pages;
     kp.page_indptr = page_indptr; kp.page_indices = page_indices; kp.lens = seq_lens; kp.hdr = static_cast<int32_t *>(ws);
@@ -627,6 +628,26 @@ spd_status spd_prefill_attn(const spd_shape *shape, int64_t total_tokens, const 
     ++g_launches;
     if (cudaGetLastError() != cudaSuccess) return SPD_ERR_CUDA;
     if (T == 0) return SPD_OK;
+
+    PrefillParams pp;
+    pp.B = shape->batch; pp.Hq = shape->num_q_heads; pp.Hkv = shape->num_kv_heads; pp.T = T;
+    pp.sm_scale = shape->sm_scale; pp.tok_indptr = tok_indptr; pp.out = out; pp.out_bf16 = out_dtype == SPD_BF16;
+    pp.hdr = static_cast<int32_t *>(ws);
+    // fp32 prompts and head_dim 64 run on the FMA pipes (so does any shape when spd_set_prefill_rows(8) asks for it);
+    // bf16 with head_dim 128, the shape that matters for throughput, runs on the tensor cores
+    if (shape->dtype != SPD_BF16 || shape->head_dim != 128 || g_prefill_rows.load() == kFmaRows) {
+        const int64_t max_blocks = (T + kFmaRows - 1) / kFmaRows + shape->batch;
+        if (max_blocks >= (1ll << 31)) return SPD_ERR_UNSUPPORTED;
+        dim3 grid(static_cast<unsigned>(max_blocks), static_cast<unsigned>(shape->num_q_heads));
+        const bool bf = shape->dtype == SPD_BF16;
+        const int D = shape->head_dim;
+        if (bf && D == 128) prefill_fma_kernel<__nv_bfloat16, 128><<<grid, kFmaRows * 32, 0, st>>>(pp, static_cast<const __nv_bfloat16 *>(q), static_cast<const __nv_bfloat16 *>(k), static_cast<const __nv_bfloat16 *>(v));
+        else if (bf) prefill_fma_kernel<__nv_bfloat16, 64><<<grid, kFmaRows * 32, 0, st>>>(pp, static_cast<const __nv_bfloat16 *>(q), static_cast<const __nv_bfloat16 *>(k), static_cast<const __nv_bfloat16 *>(v));
+        else if (D == 128) prefill_fma_kernel<float, 128><<<grid, kFmaRows * 32, 0, st>>>(pp, static_cast<const float *>(q), static_cast<const float *>(k), static_cast<const float *>(v));
+        else prefill_fma_kernel<float, 64><<<grid, kFmaRows * 32, 0, st>>>(pp, static_cast<const float *>(q), static_cast<const float *>(k), static_cast<const float *>(v));
+        ++g_launches;
+        return cudaGetLastError() == cudaSuccess ? SPD_OK : SPD_ERR_CUDA;
+    }
 
     // Long prompts go to the kernel with two 128-row tiles per CTA (each K/V block crosses from L2 once for
     // 256 rows); short ones to the one-tile kernel, whose CTAs are finer grained.  Only the mean length is
@@ -637,10 +658,6 @@ spd_status spd_prefill_attn(const spd_shape *shape, int64_t total_tokens, const 
     if ((rc = make_prompt_map(&mq, q, T, shape->num_q_heads, kPfBlock)) != SPD_OK) return rc;
     if ((rc = make_prompt_map(&mk, k, T, shape->num_kv_heads, kPfKeys)) != SPD_OK) return rc;
     if ((rc = make_prompt_map(&mv, v, T, shape->num_kv_heads, kPfKeys)) != SPD_OK) return rc;
-    PrefillParams pp;
-    pp.B = shape->batch; pp.Hq = shape->num_q_heads; pp.Hkv = shape->num_kv_heads; pp.T = T;
-    pp.sm_scale = shape->sm_scale; pp.tok_indptr = tok_indptr; pp.out = out; pp.out_bf16 = out_dtype == SPD_BF16;
-    pp.hdr = static_cast<int32_t *>(ws);
     static std::once_flag once[64];
     int dev = 0;
     cudaGetDevice(&dev);
@@ -837,7 +854,7 @@ spd_status spd_set_bf16_math(int32_t path) {
 }
 
 spd_status spd_set_prefill_rows(int32_t rows) {
-    if (rows != 0 && rows != 128 && rows != 256) return SPD_ERR_INVALID_ARG;
+    if (rows != 0 && rows != 128 && rows != 256 && rows != kFmaRows) return SPD_ERR_INVALID_ARG;
     g_prefill_rows.store(rows);
     return SPD_OK;
 }

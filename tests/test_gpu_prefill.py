@@ -190,3 +190,92 @@ def test_prefill_with_inconsistent_offsets_serves_the_users_before_them(tile):
     assert np.abs(got[:good] - ref).max() <= TOL_ABS
     assert np.all(np.isnan(got[good:]))
     assert pg.seq_lens.cpu().tolist()[:2] == lens[:2]
+
+
+# ------------------------------------------------------------------------------------------------ FMA-pipe kernel
+def _case_any(lens, hq, hkv, D, dtype, seed):
+    """Like _case, for any head_dim and dtype."""
+    B = len(lens)
+    rng = np.random.default_rng(seed)
+    gen = torch.Generator().manual_seed(seed)
+    ip = np.concatenate([[0], np.cumsum(lens)]).astype(np.int32)
+    T = int(ip[-1])
+    q, k, v = (torch.randn((T, h, D), generator=gen).to(dtype) for h in (hq, hkv, hkv))
+    need = (np.asarray(lens) + 15) // 16 + 1
+    pidx = np.concatenate([[0], np.cumsum(need)]).astype(np.int32)
+    total = int(pidx[-1])
+    perm = rng.permutation(total + 5)[:total].astype(np.int32)
+    pool = torch.full((total + 5, hkv, 16, D), float("nan"), dtype=dtype)
+    part = wl.PagedKV(pool.clone(), pool.clone(), torch.from_numpy(pidx), torch.from_numpy(perm),
+                      torch.full((B,), -7, dtype=torch.int32))
+    return q, k, v, ip, part
+
+
+def _bits(t):
+    return t.cpu().view(torch.int16 if t.dtype == torch.bfloat16 else torch.int32).numpy()
+
+
+@pytest.mark.parametrize("dtype,D,force", [(torch.float32, 64, False), (torch.float32, 128, False), (torch.bfloat16, 64, False),
+                                           (torch.bfloat16, 128, True)])
+@pytest.mark.parametrize("lens,hq,hkv", [([256, 256, 256, 256], 8, 8), ([33, 0, 1, 500, 8, 9], 4, 2), ([700], 16, 2),
+                                         (MANY_USERS, 2, 1)])
+def test_prefill_on_the_fma_pipes(dtype, D, force, lens, hq, hkv):
+    """fp32 prompts and head_dim 64 (the tiny configuration's shape among them: 4 users x 256 tokens, 8 heads, D 64,
+    fp32) are prefilled on the FMA pipes in fp32 arithmetic: causal attention against the oracle at the decode
+    tolerances, the hand-over bit for bit, the first decode step on top.  bf16 / D 128 can be forced onto the same
+    kernel, which checks it against the tensor-core kernels' oracle too."""
+    q, k, v, ip, part = _case_any(lens, hq, hkv, D, dtype, seed=sum(lens) + D)
+    B, T = len(lens), int(ip[-1])
+    scale = 1.0 / np.sqrt(D)
+    ref = orc.prefill(orc.q_from_torch(q), orc.q_from_torch(k), orc.q_from_torch(v), ip, scale)
+    shape = spd.make_shape(B, hq, hkv, D, dtype, scale)
+    ws = spd.alloc_workspace(shape)
+    pg = part.to("cuda")
+    out = torch.full((T, hq, D), float("nan"), dtype=torch.float32, device="cuda")
+    if force:
+        spd.spd_set_prefill_rows(8)
+    try:
+        n0 = spd.spd_kernel_launch_count()
+        spd.spd_prefill_attn(shape, q.cuda(), k.cuda(), v.cuda(), torch.from_numpy(ip).cuda(), pg, out, ws)
+        assert spd.spd_kernel_launch_count() - n0 == 2
+    finally:
+        spd.spd_set_prefill_rows(0)
+    assert spd.spd_query_device_status(ws) == (spd.SPD_OK, -1)
+    got = out.cpu().numpy().astype(np.float64)
+    assert np.all(np.isfinite(got))
+    tol_abs, tol_rel = (1e-5, 1e-5) if dtype == torch.float32 else (2e-3, 1e-3)
+    assert np.max(np.abs(got - ref)) <= tol_abs and np.linalg.norm(got - ref) / np.linalg.norm(ref) <= tol_rel
+    okv = orc.kv_from_torch(part)
+    orc.write_prompt_kv(okv, orc.q_from_torch(k), orc.q_from_torch(v), ip)
+    assert np.array_equal(pg.seq_lens.cpu().numpy(), okv.seq_lens)
+    assert np.array_equal(_bits(pg.k_pool), okv.k_pool.view(_bits(pg.k_pool).dtype))
+    assert np.array_equal(_bits(pg.v_pool), okv.v_pool.view(_bits(pg.v_pool).dtype))
+    qd = torch.randn((B, hq, D), generator=torch.Generator().manual_seed(3)).to(dtype)
+    empty = wl.PagedKV(torch.zeros((1, hkv, 16, D), dtype=dtype), torch.zeros((1, hkv, 16, D), dtype=dtype),
+                       torch.zeros(B + 1, dtype=torch.int32), torch.zeros(0, dtype=torch.int32), torch.zeros(B, dtype=torch.int32))
+    yd = torch.full((B, hq, D), float("nan"), dtype=torch.float32, device="cuda")
+    spd.spd_decode_step(shape, qd.cuda(), pg, empty.to("cuda"), yd, ws, fused=True)
+    assert spd.spd_query_device_status(ws) == (spd.SPD_OK, -1)
+    assert np.max(np.abs(yd.cpu().numpy() - orc.full(orc.q_from_torch(qd), okv, None, scale))) <= tol_abs * (1 if dtype == torch.float32 else 1)
+
+
+def test_prefill_fma_bf16_output_and_inconsistent_offsets():
+    """bf16 output rounding, and token offsets that go backwards: users before the first inconsistent one are served,
+    later rows stay unwritten, the status says so (as in the tensor-core kernels)."""
+    q, k, v, ip, part = _case_any([40, 60, 30], 4, 4, 64, torch.float32, seed=5)
+    scale = 0.125
+    shape = spd.make_shape(3, 4, 4, 64, torch.float32, scale)
+    ws = spd.alloc_workspace(shape)
+    ref = orc.prefill(orc.q_from_torch(q), orc.q_from_torch(k), orc.q_from_torch(v), ip, scale)
+    out = torch.full((130, 4, 64), float("nan"), dtype=torch.bfloat16, device="cuda")
+    spd.spd_prefill_attn(shape, q.cuda(), k.cuda(), v.cuda(), torch.from_numpy(ip).cuda(), part.to("cuda"), out, ws)
+    assert spd.spd_query_device_status(ws) == (spd.SPD_OK, -1)
+    assert np.max(np.abs(out.float().cpu().numpy() - ref)) <= 1e-5 + 2.0 ** -8 * np.max(np.abs(ref))
+    bad = ip.copy()
+    bad[2] = 20                                              # user 1 would end before it starts
+    out32 = torch.full((130, 4, 64), float("nan"), dtype=torch.float32, device="cuda")
+    spd.spd_prefill_attn(shape, q.cuda(), k.cuda(), v.cuda(), torch.from_numpy(bad).cuda(), part.to("cuda"), out32, ws)
+    code, _ = spd.spd_query_device_status(ws)
+    got = out32.cpu().numpy()
+    assert np.max(np.abs(got[:40] - ref[:40])) <= 1e-5       # user 0 is served
+    assert np.all(np.isnan(got[40:]))                        # nothing from the inconsistent user on

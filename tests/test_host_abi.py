@@ -70,9 +70,9 @@ def test_bad_arguments_are_rejected_on_the_host(lib):
     assert lay.in_bytes >= 4 * 8 * 64 * 4 + 2 * (5 + 4 + 10) * 4 and lay.total_bytes >= lay.out + 4 * 8 * 64 * 4
     assert lay.q == 0 and lay.out == lay.in_bytes and lay.status + 256 == lay.in_bytes and lay.priv_indices % 256 == 0
     assert lib.spd_decode_step_host(C.byref(ok), C.byref(lay), None, None, None, None, 0, None, None, 0, None) == 1
-    # prefill: bf16 and head_dim 128 only, positive scale only; the token step and the knobs check their arguments
+    # prefill: positive scale only, null offsets refused; the token step and the knobs check their arguments
     pf_args = (C.c_int64(0), None, None, None, None, None, None, 0, None, None, None, None, 1, None, 0, None)
-    assert lib.spd_prefill_attn(C.byref(ok), *pf_args) == 2
+    assert lib.spd_prefill_attn(C.byref(ok), *pf_args) == 1
     assert lib.spd_prefill_attn(C.byref(spd.make_shape(2, 8, 8, 128, torch.bfloat16, -1.0)), *pf_args) == 2
     assert lib.spd_prefill_attn(C.byref(spd.make_shape(2, 8, 8, 128, torch.bfloat16, 0.1)), *pf_args) == 1   # null offsets
     assert lib.spd_token_step(C.byref(ok), 0, None, 0, 0, None, 0, None) == 1
@@ -85,7 +85,8 @@ def test_bad_arguments_are_rejected_on_the_host(lib):
     assert lib.spd_set_programmatic_launch(2) == 1
     assert lib.spd_debug_read_plan(None, 0, None, None, None, None, 0) == 1
     assert lib.spd_debug_sm_moves(None, None, None, None) == 1
-    assert lib.spd_set_prefill_rows(64) == 1 and lib.spd_set_prefill_rows(256) == 0 and lib.spd_set_prefill_rows(0) == 0
+    assert lib.spd_set_prefill_rows(64) == 1 and lib.spd_set_prefill_rows(256) == 0 and lib.spd_set_prefill_rows(8) == 0
+    assert lib.spd_set_prefill_rows(0) == 0
     assert lib.spd_set_bf16_math(2) == 1
 
 
