@@ -273,16 +273,16 @@ def kernel_split(spd, w, shape, ws, out, steps):
     return {"attn_ms": r["kernel_ms"] / max(r["calls"], 1)}
 
 
-def time_e2e(spd, w, shape, ws, steps, warmup):
+def time_e2e(spd, w, shape, ws, steps, warmup, out_dtype=torch.float32):
     """Per step: q, page tables and lengths go in from one pinned host blob, the output comes back."""
     dev = w.q.device
-    lay = spd.spd_step_blob_layout(shape, int(w.priv.page_indices.numel()), int(w.pub.page_indices.numel()), torch.float32)
+    lay = spd.spd_step_blob_layout(shape, int(w.priv.page_indices.numel()), int(w.pub.page_indices.numel()), out_dtype)
     host = torch.zeros(lay.total_bytes, dtype=torch.uint8).pin_memory()
     spd.fill_step_blob(lay, host, w.q, w.priv, w.pub)
     devb = torch.empty(lay.total_bytes, dtype=torch.uint8, device=dev)
     pools = [(w.priv.k_pool, w.priv.v_pool), (w.pub.k_pool, w.pub.v_pool)]
 
-    step = spd.HostStep(shape, lay, host, devb, pools[0], pools[1], torch.float32, ws)
+    step = spd.HostStep(shape, lay, host, devb, pools[0], pools[1], out_dtype, ws)
 
     def call():
         code, bad = step()
@@ -299,7 +299,8 @@ def time_e2e(spd, w, shape, ws, steps, warmup):
     torch.cuda.synchronize()
     d2h = lay.total_bytes - lay.status
     n_out = w.batch * w.num_q_heads * w.head_dim
-    outh = host[lay.out:lay.out + 4 * n_out].view(torch.float32).reshape(w.batch, w.num_q_heads, w.head_dim).clone()
+    es = 4 if out_dtype == torch.float32 else 2
+    outh = host[lay.out:lay.out + es * n_out].view(out_dtype).reshape(w.batch, w.num_q_heads, w.head_dim).float().clone()
     return e0.elapsed_time(e1) / steps, lay.in_bytes, d2h, outh
 
 
@@ -592,7 +593,13 @@ def measure_config(spd, cfg, dev, steps, warmup, local_rank, users=None, seconds
         if not torch.allclose(outh, out.cpu(), atol=2e-3, rtol=0):   # share sizes adapt, so rounding order may differ
             raise RuntimeError("host-buffer path and device path disagree")
         res["e2e"] = {"value": kvb / e2e_ms / 1e6, "unit": "GB/s", "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
-                      "ms_per_step": e2e_ms, "call": "spd_decode_step_host"}
+                      "ms_per_step": e2e_ms, "call": "spd_decode_step_host", "out_dtype": "f32"}
+        # the same with the output read back in bf16 (what a bf16 model consumes): half the device-to-host bytes
+        b_ms, b_h2d, b_d2h, outb = time_e2e(spd, w, shape, ws, min(300, max(steps, int(0.2 * seconds * 1e3 / ms))), warmup, torch.bfloat16)
+        if not torch.allclose(outb, out.cpu(), atol=2e-3 + 2.0 ** -8 * float(out.abs().max()), rtol=0):
+            raise RuntimeError("host-buffer path with bf16 output and device path disagree")
+        res["e2e_bf16_out"] = {"value": kvb / b_ms / 1e6, "unit": "GB/s", "h2d_bytes_per_step": b_h2d, "d2h_bytes_per_step": b_d2h,
+                               "ms_per_step": b_ms}
         brief = 0.25 * seconds
         m, *_ = time_config(spd, w, steps, warmup, fused=False, min_seconds=brief)
         res["chained"] = {"ms_per_step": m, "gbs": kvb / m / 1e6}
@@ -663,7 +670,7 @@ def run_cuda(args):
         "e2e": e2e, "gpu_launches": head["gpu_launches"], "roofline": head["roofline"], "clocks": head["clocks"],
         "sm_moves": head["sm_moves"],
     }
-    for k in ("chained", "plan_cached", "uniform_shares"):
+    for k in ("e2e_bf16_out", "chained", "plan_cached", "uniform_shares"):
         if k in head:
             line[k] = head[k]
     if world == 1 and not args.no_extras and not args.kernel_only and args.users is None:
