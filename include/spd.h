@@ -32,8 +32,9 @@
  *     that kernel has completed.  If a kernel of yours on the same stream writes lengths, page tables or KV rows
  *     immediately before a call, launch in plain stream order: spd_set_programmatic_launch(0), or SPD_NO_PDL=1
  *     in the environment.  Where the library's own calls write such inputs (the appends), they order themselves.
- *   - Threads.  Calls may come from several host threads; calls that share a workspace must be ordered by the
- *     caller (one stream at a time per workspace).  Each workspace keeps a small table of streaming rates that
+ *   - Threads.  Calls may come from several host threads, also from threads that have made no CUDA call of their
+ *     own yet (the library makes the current device's context current on such a thread at its first call); calls
+ *     that share a workspace must be ordered by the caller (one stream at a time per workspace).  Each workspace keeps a small table of streaming rates that
  *     sizes the next call's shares; it is rotated by a per-workspace launch count held on the host, so calls on
  *     other workspaces or streams never disturb it.
  *   - CUDA graphs.  Every call may be captured.  What is decided on the host at call time is then frozen into
@@ -262,6 +263,19 @@ spd_status spd_decode_step_append(const spd_shape *shape, const void *q, const v
                                   const spd_paged_kv *priv, const spd_paged_kv *pub, void *out,
                                   spd_dtype out_dtype, spd_plan_mode plan, void *ws, size_t ws_bytes,
                                   void *cuda_stream);
+
+/*
+ * The service's whole share of a decode step in one launch (protocol steps 3a and 3c; Fig. 3 steps 2, 3 and 5):
+ * spd_service_attn_merge with the append of the new token's K and V rows at its head -- the public partition counts
+ * the new token, whose rows come from k_new / v_new and are written to the cache on the way, the public partial is
+ * merged with `in` (the private partial that a per-user process computed meanwhile, which never sees the public
+ * cache) and the attention output is written.  Lengths, flags, `plan` and stream order as for
+ * spd_decode_step_append.
+ */
+spd_status spd_service_attn_merge_append(const spd_shape *shape, const void *q, const void *k_new,
+                                         const void *v_new, const spd_paged_kv *pub, spd_partial in, void *out,
+                                         spd_dtype out_dtype, spd_plan_mode plan, void *ws, size_t ws_bytes,
+                                         void *cuda_stream);
 
 /*
  * One token step over `num_layers` layers (protocol step 3 for every layer of the model; Fig. 3 steps 2 to

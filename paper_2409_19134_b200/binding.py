@@ -27,7 +27,7 @@ EXPORTS = ["spd_workspace_size", "spd_partial_attn", "spd_service_attn_merge", "
            "spd_partial_attn_watch", "spd_decode_step_watch", "spd_set_bf16_math", "spd_merge_partials", "spd_prefill_attn",
            "spd_set_prefill_rows", "spd_token_step", "spd_partial_attn_planned", "spd_service_attn_merge_planned",
            "spd_decode_step_planned", "spd_set_split", "spd_set_programmatic_launch", "spd_debug_read_plan",
-           "spd_debug_sm_moves", "spd_decode_step_append", "spd_watch_alarm"]
+           "spd_debug_sm_moves", "spd_decode_step_append", "spd_watch_alarm", "spd_service_attn_merge_append"]
 
 
 class SpdError(RuntimeError):
@@ -106,6 +106,8 @@ def lib() -> C.CDLL:
                                               C.c_int32, C.c_int, vp, sz, vp]
         L.spd_decode_step_append.argtypes = [C.POINTER(Shape), vp, vp, vp, C.POINTER(PagedKV), C.POINTER(PagedKV), vp, C.c_int,
                                              C.c_int, vp, sz, vp]
+        L.spd_service_attn_merge_append.argtypes = [C.POINTER(Shape), vp, vp, vp, C.POINTER(PagedKV), Partial, vp, C.c_int, C.c_int,
+                                                    vp, sz, vp]
         L.spd_watch_alarm.argtypes = [vp, C.c_int32, C.c_int32, vp, C.c_float, vp, vp]
         L.spd_set_split.argtypes = [C.c_int32, C.c_int32]
         L.spd_set_programmatic_launch.argtypes = [C.c_int32]
@@ -333,6 +335,17 @@ def spd_decode_step_append(shape, q, k_new, v_new, priv, pub, out, ws, plan=SPD_
     _check(lib().spd_decode_step_append(C.byref(shape), q.data_ptr(), k_new.data_ptr(), v_new.data_ptr(), C.byref(a),
                                         C.byref(b), out.data_ptr(), _dtype_code(out.dtype), int(plan), ws.data_ptr(),
                                         ws.numel(), _stream_ptr(stream)), "spd_decode_step_append")
+
+
+def spd_service_attn_merge_append(shape, q, k_new, v_new, pub, partial_in, out, ws, plan=SPD_PLAN_PER_CALL, stream=None) -> None:
+    """The service call with the append at its head: `pub` grows by the new token (pools and seq_lens updated in
+    place), its partial is merged with `partial_in` and the attention output written, in one launch."""
+    assert k_new.is_contiguous() and v_new.is_contiguous()
+    kv = paged_kv(pub)
+    part = Partial(partial_in[0].data_ptr(), partial_in[1].data_ptr(), partial_in[2].data_ptr())
+    _check(lib().spd_service_attn_merge_append(C.byref(shape), q.data_ptr(), k_new.data_ptr(), v_new.data_ptr(), C.byref(kv),
+                                               part, out.data_ptr(), _dtype_code(out.dtype), int(plan), ws.data_ptr(),
+                                               ws.numel(), _stream_ptr(stream)), "spd_service_attn_merge_append")
 
 
 def spd_token_step(shape, layers, ws, stream=None, same_lengths=False) -> None:

@@ -92,6 +92,16 @@ spd_status device_info(DeviceInfo *out) {
     static DeviceInfo cache[64];
     int dev = 0;
     if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return SPD_ERR_CUDA;
+    // The tensor maps are encoded through the driver API, which wants the device's context current on the CALLING
+    // thread; the runtime only makes it so at a thread's first call that needs a context.  A host thread that has
+    // made no such call yet (a worker that only ever calls this library) gets it here, once: a stream query does it
+    // and neither allocates nor waits.
+    static thread_local int bound_dev = -1;
+    if (bound_dev != dev) {
+        const cudaError_t e = cudaStreamQuery(cudaStreamLegacy);
+        if (e != cudaSuccess && e != cudaErrorNotReady) return SPD_ERR_CUDA;
+        bound_dev = dev;
+    }
     std::lock_guard<std::mutex> lock(mu);
     if (!cache[dev].ok) {
         int sms = 0, major = 0;
@@ -215,6 +225,7 @@ spd_status make_map(CUtensorMap *map, const spd_shape &s, const void *pool, int6
                     const_cast<void *>(pool), dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
                     bf ? CU_TENSOR_MAP_SWIZZLE_128B : CU_TENSOR_MAP_SWIZZLE_NONE, SPD_TMA_L2_PROMOTION,
                     CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    if (r != CUDA_SUCCESS) fprintf(stderr, "libspd: cuTensorMapEncodeTiled failed with CUresult %d\n", static_cast<int>(r));
     return r == CUDA_SUCCESS ? SPD_OK : SPD_ERR_CUDA;
 }
 
@@ -234,7 +245,10 @@ spd_status launch_attn(const Params &p_in, const CUtensorMap *maps, int sms, cud
         attr_err = cudaFuncSetAttribute(attn_kernel<Math>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                         static_cast<int>(smem));
     });
-    if (attr_err != cudaSuccess) return SPD_ERR_CUDA;
+    if (attr_err != cudaSuccess) {
+        fprintf(stderr, "libspd: cudaFuncSetAttribute(dynamic shared memory %zu): %s\n", smem, cudaGetErrorString(attr_err));
+        return SPD_ERR_CUDA;
+    }
     // Programmatic stream serialisation (pdl): this kernel's read-only preamble may overlap the tail of the
     // previous kernel on the stream if that kernel allows it (the attention kernel does).
     cudaLaunchConfig_t cfg = {};
@@ -249,6 +263,7 @@ spd_status launch_attn(const Params &p_in, const CUtensorMap *maps, int sms, cud
     cfg.numAttrs = pdl ? 1 : 0;
     const cudaError_t err = cudaLaunchKernelEx(&cfg, attn_kernel<Math>, p, maps[0], maps[1], maps[2], maps[3]);
     ++g_launches;
+    if (err != cudaSuccess) fprintf(stderr, "libspd: launch of the attention kernel: %s\n", cudaGetErrorString(err));
     return err == cudaSuccess ? SPD_OK : SPD_ERR_CUDA;
 }
 
@@ -431,7 +446,7 @@ static spd_status partial_attn_impl(const spd_shape *shape, const void *q, const
 
 static spd_status service_attn_merge_impl(const spd_shape *shape, const void *q, const spd_paged_kv *pub, spd_partial in,
                                           void *out, spd_dtype out_dtype, int plan, void *ws, size_t ws_bytes,
-                                          void *cuda_stream) {
+                                          void *cuda_stream, const void *k_new = nullptr, const void *v_new = nullptr) {
     spd_status rc = check_shape(shape);
     if (rc != SPD_OK) return rc;
     if ((rc = check_kv(shape, pub)) != SPD_OK) return rc;
@@ -443,6 +458,11 @@ static spd_status service_attn_merge_impl(const spd_shape *shape, const void *q,
     job.mode = OUT_FINAL; job.pin = &in; job.out = out; job.out_dtype = out_dtype;
     job.epoch = next_epoch();
     job.plan_mode = plan;
+    if (k_new) {     // an appending launch reads lengths that the previous call of its kind bumps as its last act
+        job.k_new = k_new; job.v_new = v_new;
+        job.plain_order = true;
+        job.wait_first = true;
+    }
     return run_job(job, ws, ws_bytes, cuda_stream);
 }
 
@@ -522,6 +542,13 @@ spd_status spd_decode_step_append(const spd_shape *shape, const void *q, const v
     // which adds one to the lengths as its last act: nothing is read before that kernel has finished.
     return decode_step_impl(shape, q, priv, pub, out, out_dtype, 1, plan, true, ws, ws_bytes, cuda_stream, k_new, v_new,
                             true);
+}
+
+spd_status spd_service_attn_merge_append(const spd_shape *shape, const void *q, const void *k_new, const void *v_new,
+                                         const spd_paged_kv *pub, spd_partial in, void *out, spd_dtype out_dtype,
+                                         spd_plan_mode plan, void *ws, size_t ws_bytes, void *cuda_stream) {
+    if (check_plan(plan) != SPD_OK || !k_new || !v_new) return SPD_ERR_INVALID_ARG;
+    return service_attn_merge_impl(shape, q, pub, in, out, out_dtype, plan, ws, ws_bytes, cuda_stream, k_new, v_new);
 }
 
 spd_status spd_decode_step_planned(const spd_shape *shape, const void *q, const spd_paged_kv *priv,

@@ -267,6 +267,26 @@ def test_append_inside_the_decode_launch(dtype, hq, hkv, d):
         ok = [u for u in range(B) if done[u]]
         assert bool((out[full] == 0).all())
         assert_close(out[ok].cpu().numpy(), ref[ok], w.dtype, f"attention over the grown cache, step {step}")
+    # the paper's split with the append at the head of the service call: the per-user process computes the private
+    # partial (it never sees the public cache), the service appends, computes the public partial and merges
+    k_new = torch.randn((B, hkv, d), generator=gen).to(w.dtype)
+    v_new = torch.randn((B, hkv, d), generator=gen).to(w.dtype)
+    done = orc.append(kout, orc.q_from_torch(k_new), orc.q_from_torch(v_new))
+    ref = orc.full(q, kin, kout, w.sm_scale)
+    part = spd.alloc_partial(shape)
+    spd.spd_partial_attn(shape, wg.q, wg.priv, part, ws)
+    out = torch.full((B, hq, d), float("nan"), dtype=torch.float32, device="cuda")
+    spd.spd_service_attn_merge_append(shape, wg.q, k_new.cuda(), v_new.cuda(), wg.pub, part, out, ws)
+    assert spd.spd_query_device_status(ws)[0] == 4
+    ok = [u for u in range(B) if done[u]]
+    assert np.array_equal(wg.pub.seq_lens.cpu().numpy(), kout.seq_lens)
+    assert np.array_equal(bits(wg.pub.k_pool), kout.k_pool.view(bits(wg.pub.k_pool).dtype))
+    assert np.array_equal(bits(wg.pub.v_pool), kout.v_pool.view(bits(wg.pub.v_pool).dtype))
+    assert bool((out[[u for u in range(B) if not done[u]]] == 0).all())
+    assert_close(out[ok].cpu().numpy(), ref[ok], w.dtype, "service call with the append at its head")
+    wg.pub.seq_lens.copy_(torch.clamp(wg.pub.seq_lens - 1, min=0))            # back to the storing call's lengths + 1
+    kout.seq_lens[:] = np.maximum(kout.seq_lens - 1, 0)
+    wg.pub.seq_lens[-1] = int(lout[-1]); kout.seq_lens[-1] = int(lout[-1])
     # the stored plan serves another cache with the lengths this one had before the storing call's append
     # (same arrays moved back by one), values of the rows that are appended again differ
     wg.pub.seq_lens.copy_(torch.clamp(wg.pub.seq_lens - 1, min=0))

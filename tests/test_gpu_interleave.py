@@ -101,3 +101,32 @@ def test_per_layer_calls_without_a_kernel_in_between():
     torch.cuda.synchronize()
     _check(wa, ref_a, outs_a, ws_a, sa, "layer-by-layer calls, batch A")
     _check(wb, ref_b, outs_b, ws_b, sb, "layer-by-layer calls, batch B")
+
+
+def test_two_host_threads_two_workspaces():
+    """Calls may come from several host threads as long as each workspace is driven by one of them: two threads, each
+    with its own batch, workspace and stream, issue their steps at the same time (ctypes releases the interpreter
+    lock during a call, so the launches really interleave in the library)."""
+    import threading
+    batches = [_batch(A_CFG), _batch(B_CFG)]
+    streams = [torch.cuda.Stream(), torch.cuda.Stream()]
+    torch.cuda.synchronize()
+    errors = []
+
+    def serve(k):
+        try:
+            w, g, ref, shape, ws, outs = batches[k]
+            for r in range(ROUNDS):
+                spd.spd_decode_step(shape, g.q, g.priv, g.pub, outs[r], ws, fused=(k == 0 or r % 2 == 0), stream=streams[k])
+        except Exception as e:          # noqa: BLE001  (reported by the main thread)
+            errors.append(e)
+    threads = [threading.Thread(target=serve, args=(k,)) for k in range(2)]
+    for t in threads:
+        t.start()
+    for t in threads:
+        t.join()
+    torch.cuda.synchronize()
+    assert not errors, errors
+    for k, what in enumerate(("thread 0, batch A", "thread 1, batch B")):
+        w, g, ref, shape, ws, outs = batches[k]
+        _check(w, ref, outs, ws, streams[k], what)
