@@ -6,6 +6,8 @@ by element at the bf16 tolerances (max-abs 2e-3, relative L2 1e-3):
   - spd_decode_step, fused (what the benchmark times) and chained (the paper's two calls through a partial);
   - spd_partial_attn: gauge-free A = O / l and lse = m + ln l, and m itself against the true maximum;
   - spd_service_attn_merge fed with the oracle's private partial rounded to fp32 (a message produced elsewhere).
+  - spd_decode_step_append (append and attention in one launch) deriving and storing its plan, then once more on the
+    stored plan: every row, the lengths, and the appended rows in the cache bit for bit.
 The measured errors are appended to gpurun_out/full_size_errors.jsonl when that folder can be written.
 """
 import json
@@ -84,4 +86,32 @@ def test_full_size_every_row_of_every_entry_point(name):
     out.fill_(float("nan"))
     spd.spd_service_attn_merge(shape, w.q, w.pub, ext, out, ws)
     check_out("service_attn_merge")
+
+    # the append inside the launch, twice: once deriving and storing the plan, once more on the stored plan after the
+    # lengths have been moved back (what the layers of a token step do).  The listed pages have room for one more
+    # token for every user whose public length is not a multiple of 16; the others are full: zeros, no append, flagged.
+    gen = torch.Generator(device="cuda").manual_seed(77)
+    k_new = torch.randn((B, w.num_kv_heads, D), generator=gen, device="cuda").to(w.dtype)
+    v_new = torch.randn((B, w.num_kv_heads, D), generator=gen, device="cuda").to(w.dtype)
+    lens_before = w.pub.seq_lens.clone()
+    done = orc.append(kout, orc.q_from_torch(k_new.cpu()), orc.q_from_torch(v_new.cpu()))
+    ref = orc.full(q, kin, kout, w.sm_scale)
+    ok = torch.from_numpy(np.flatnonzero(done)).cuda()
+    full = torch.from_numpy(np.flatnonzero(~done)).cuda()
+    assert len(ok) > B // 2
+    for plan in (spd.SPD_PLAN_STORE, spd.SPD_PLAN_REUSE):
+        w.pub.seq_lens.copy_(lens_before)
+        out.fill_(float("nan"))
+        spd.spd_decode_step_append(shape, w.q, k_new, v_new, w.priv, w.pub, out, ws, plan=plan)
+        code, first_bad = spd.spd_query_device_status(ws)
+        assert (code, first_bad) == ((4, int(full.min())) if len(full) else (spd.SPD_OK, -1))
+        assert np.array_equal(w.pub.seq_lens.cpu().numpy(), kout.seq_lens)
+        assert bool((out[full] == 0).all())
+        got = out[ok].cpu().numpy()
+        report[f"decode_step_append_plan{plan}"] = dict(zip(("max_abs", "rel_l2"), errors(got, ref[ok.cpu().numpy()])))
+        assert_close(got, ref[ok.cpu().numpy()], w.dtype, f"{name} append inside the launch, plan mode {plan}")
+    # the appended rows sit in the cache bit for bit: position lens_before of every user that had room
+    pos = lens_before[ok].long()
+    pages = w.pub.page_indices[(w.pub.page_indptr[ok].long() + pos // 16)].long()
+    assert torch.equal(w.pub.k_pool[pages, :, pos % 16], k_new[ok]) and torch.equal(w.pub.v_pool[pages, :, pos % 16], v_new[ok])
     _record(report)
