@@ -8,7 +8,7 @@ by element at the bf16 tolerances (max-abs 2e-3, relative L2 1e-3):
   - spd_service_attn_merge fed with the oracle's private partial rounded to fp32 (a message produced elsewhere).
   - spd_decode_step_append (append and attention in one launch) deriving and storing its plan, then once more on the
     stored plan: every row, the lengths, and the appended rows in the cache bit for bit.
-The measured errors are appended to gpurun_out/full_size_errors.jsonl when that folder can be written.
+The measured errors are appended to full_size_errors.jsonl in the folder that SPD_TEST_RECORD_DIR names, if it is set.
 """
 import json
 import os
@@ -29,9 +29,12 @@ ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
 
 
 def _record(entry):
+    folder = os.environ.get("SPD_TEST_RECORD_DIR")
+    if not folder:
+        return
     try:
-        os.makedirs(os.path.join(ROOT, "gpurun_out"), exist_ok=True)
-        with open(os.path.join(ROOT, "gpurun_out", "full_size_errors.jsonl"), "a") as f:
+        os.makedirs(folder, exist_ok=True)
+        with open(os.path.join(folder, "full_size_errors.jsonl"), "a") as f:
             f.write(json.dumps(entry) + "\n")
     except OSError:
         pass

@@ -177,14 +177,15 @@ def test_prefill_at_the_benchmark_size_on_sampled_rows():
         ma, rl = float(np.abs(g2 - ref2).max()), float(np.linalg.norm(g2 - ref2) / np.linalg.norm(ref2))
         record[f"rows{rows_per_cta}"] = {"max_abs": ma, "rel_l2": rl}
         assert ma <= TOL_ABS and rl <= TOL_REL, (rows_per_cta, ma, rl)
-    try:
-        import json, os
-        root = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
-        os.makedirs(os.path.join(root, "gpurun_out"), exist_ok=True)
-        with open(os.path.join(root, "gpurun_out", "prefill_errors.jsonl"), "a") as f:
-            f.write(json.dumps(record) + "\n")
-    except OSError:
-        pass
+    import json, os
+    folder = os.environ.get("SPD_TEST_RECORD_DIR")       # where to leave the measured errors, if anywhere
+    if folder:
+        try:
+            os.makedirs(folder, exist_ok=True)
+            with open(os.path.join(folder, "prefill_errors.jsonl"), "a") as f:
+                f.write(json.dumps(record) + "\n")
+        except OSError:
+            pass
     pc = wl.PagedKV(part.k_pool.cpu(), part.v_pool.cpu(), part.page_indptr.cpu(), part.page_indices.cpu(), torch.zeros(len(lens), dtype=torch.int32))
     pc.k_pool.zero_(), pc.v_pool.zero_()
     okv = orc.kv_from_torch(pc)
