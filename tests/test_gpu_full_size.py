@@ -25,7 +25,6 @@ from tests.test_gpu_parity import TOL, assert_close, errors
 pytestmark = pytest.mark.gpu
 
 FULL = ["c2_llama2_7b", "c3_llama3_8b_gqa", "c4_long_prompt", "c5_many_user"]
-ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
 
 
 def _record(entry):
