@@ -711,7 +711,7 @@ def run_cuda(args):
 # captures summarised under profiles/; configs without a capture of the current kernel report None.  The largest
 # configuration holds too much memory for a capture: its figure is that of its first 256 users (2 615 303 936 bytes
 # for 2 590 486 528 algorithmic) scaled to all 512 by the KV bytes, traffic being proportional to the tokens streamed.
-TRAFFIC_BYTES = {"c2_llama2_7b": 1340836608, "c3_llama3_8b_gqa": 3021949696, "c5_many_user": 5084278250}
+TRAFFIC_BYTES = {"c2_llama2_7b": 1340836608, "c3_llama3_8b_gqa": 3021949696, "c4_long_prompt": 2587209728, "c5_many_user": 5084278250}
 
 
 def main():
