@@ -373,7 +373,7 @@ spd_status spd_profile_end(int32_t *calls, double *kernel_ms);
  *   - Limit: the shape must need no more than SPD_STATIC_WS_BYTES of workspace (what
  *     spd_workspace_size() reports); otherwise the call launches nothing, prints one line to stderr
  *     and returns SPD_ERR_WORKSPACE.  On a 148-SM B200 that admits roughly
- *     batch * num_q_heads <= 13000 at head_dim 128.
+ *     batch * num_q_heads <= 12000 at head_dim 128.
  *   - The first call on each device looks up the array's device address (with that device current).
  *     Make that first call outside any stream capture.
  *   - All calls share the one array, and it keeps what the previous call left, laid out for the
