@@ -95,9 +95,10 @@ typedef struct {
 
 /*
  * Bytes of device workspace the calls below need for `shape` on the current device.
- * The workspace holds the sticky status words, per-user flags, merge tickets, split-K scratch and
- * the partial of a chained step; zero it once (cudaMemset) before first use, and again after an
- * SPD_ERR_CUDA.  One workspace serves one stream at a time.
+ * The workspace holds the sticky status words, the table of streaming rates, the stored plans, per-user
+ * flags, merge tickets, split-K scratch and the partial of a chained step; it does not depend on how many
+ * tokens are cached.  Zero it once (cudaMemset) before first use, and again after an SPD_ERR_CUDA.  One
+ * workspace serves one stream at a time.
  */
 spd_status spd_workspace_size(const spd_shape *shape, size_t *bytes);
 
