@@ -156,7 +156,8 @@ spd_status spd_decode_step(const spd_shape *shape, const void *q, const spd_page
  *                       pools, q may differ).  A plan that was never stored, or was stored for another shape,
  *                       raises SPD_ERR_PLAN and the call writes nothing (a plain or PER_CALL call of the same
  *                       kind in between discards the stored plan); lengths that changed silently give
- *                       wrong results for the users concerned (never a fault: every index is still checked).
+ *                       wrong results for the users concerned, possibly with SPD_ERR_PLAN or SPD_ERR_BAD_PAGE
+ *                       raised (never a fault: every index is still checked).
  * Reuse pays for small calls, where deriving the plan is most of the time; large calls hide it anyway.
  */
 typedef enum { SPD_PLAN_PER_CALL = 0, SPD_PLAN_STORE = 1, SPD_PLAN_REUSE = 2 } spd_plan_mode;
