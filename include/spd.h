@@ -318,6 +318,10 @@ spd_status spd_token_step(const spd_shape *shape, int32_t num_layers, const spd_
  * device: `priv_pools` and `pub_pools` carry k_pool, v_pool and num_pages only (their table pointers
  * are ignored).  `device_blob` is device memory of layout->total_bytes, 256-byte aligned.
  *
+ * A batch whose q or output comes to megabytes is served in two parts inside the call, so that the second part's q
+ * goes up and the first part's output comes down (on a copy stream that the library keeps per host thread) while the
+ * other part's kernel runs; the result is the same, row for row.
+ *
  * The call copies host_blob[0, in_bytes) to the device, runs the step, copies status and output back
  * (the output to host_blob + layout->out), waits for the stream and returns the device status of
  * this step (*first_bad_user: lowest flagged user or -1; may be NULL).  The workspace's own sticky

@@ -115,6 +115,32 @@ spd_status device_info(DeviceInfo *out) {
     return SPD_OK;
 }
 
+// A copy stream and two events per host thread and device for the host-buffer entry point, made at the thread's
+// first large call on the device and kept (no device memory is involved).
+constexpr int kHostStepParts = 2;     // a large batch is served in this many parts (8 status words each: at most 8); four measured no faster than two
+struct HostStepStreams {
+    cudaStream_t copy = nullptr;
+    cudaEvent_t q_up[kHostStepParts] = {}, done[kHostStepParts] = {};   // part i's q is on the device; part i's kernel has finished
+};
+
+spd_status host_step_streams(HostStepStreams *out) {
+    static thread_local HostStepStreams cache[64];     // per host thread: two threads may serve two batches at once
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return SPD_ERR_CUDA;
+    HostStepStreams &h = cache[dev];
+    if (!h.copy) {
+        HostStepStreams n;
+        if (cudaStreamCreateWithFlags(&n.copy, cudaStreamNonBlocking) != cudaSuccess) return SPD_ERR_CUDA;
+        for (int i = 0; i < kHostStepParts; ++i)
+            if (cudaEventCreateWithFlags(&n.q_up[i], cudaEventDisableTiming) != cudaSuccess ||
+                cudaEventCreateWithFlags(&n.done[i], cudaEventDisableTiming) != cudaSuccess)
+                return SPD_ERR_CUDA;
+        h = n;
+    }
+    *out = h;
+    return SPD_OK;
+}
+
 #ifndef SPD_TMA_L2_PROMOTION
 #define SPD_TMA_L2_PROMOTION CU_TENSOR_MAP_L2_PROMOTION_L2_256B
 #endif
@@ -284,6 +310,7 @@ struct Job {
     bool plain_order;              // launch in plain stream order (an input was written by the kernel just before)
     const void *k_new, *v_new;     // optional append of the new token's rows to part[1] inside the launch
     bool wait_first;               // read nothing before the previous kernel on the stream has finished, not even a stored plan
+    const spd_shape *layout_shape; // shape that lays the workspace out, if not `shape` (a call served in two halves keeps the whole batch's layout)
 };
 
 // The stored plan of a call is tagged with what it was cut for besides the lengths, so that a launch told to load a
@@ -301,7 +328,7 @@ spd_status run_job(const Job &job, void *ws, size_t ws_bytes, void *stream) {
     DeviceInfo di;
     spd_status rc = device_info(&di);
     if (rc != SPD_OK) return rc;
-    const WsLayout L = ws_layout(s, di.sms);
+    const WsLayout L = ws_layout(job.layout_shape ? *job.layout_shape : s, di.sms);
     if (!ws || misaligned(ws, 256)) return SPD_ERR_INVALID_ARG;
     if (ws_bytes < L.total) return SPD_ERR_WORKSPACE;
     if (!job.q || misaligned(job.q, 16)) return SPD_ERR_INVALID_ARG;
@@ -817,7 +844,7 @@ spd_status spd_decode_step_host(const spd_shape *shape, const spd_step_blob *lay
         return SPD_ERR_INVALID_ARG;
     cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
     uint8_t *db = static_cast<uint8_t *>(device_blob);
-    if (cudaMemcpyAsync(db, hb, layout->in_bytes, cudaMemcpyHostToDevice, st) != cudaSuccess) return SPD_ERR_CUDA;
+    uint8_t *hbw = static_cast<uint8_t *>(host_blob);
     spd_paged_kv a = *priv_pools, b = *pub_pools;
     a.page_indptr = reinterpret_cast<const int32_t *>(db + layout->priv_indptr);
     a.seq_lens = reinterpret_cast<const int32_t *>(db + layout->priv_lens);
@@ -827,22 +854,84 @@ spd_status spd_decode_step_host(const spd_shape *shape, const spd_step_blob *lay
     b.page_indices = reinterpret_cast<const int32_t *>(db + layout->pub_indices);
     if ((rc = check_kv(shape, &a)) != SPD_OK || (rc = check_kv(shape, &b)) != SPD_OK) return rc;
     if (out_dtype != SPD_F32 && out_dtype != SPD_BF16) return SPD_ERR_UNSUPPORTED;
-    // The step raises its status in the blob (uploaded as zeros a moment ago), right in front of the
-    // output, so that one copy brings both back.
-    Job job{};
-    job.shape = shape; job.q = db + layout->q; job.part[0] = &a; job.part[1] = &b;
-    job.mode = OUT_FINAL; job.pin = nullptr; job.out = db + layout->out; job.out_dtype = out_dtype;
-    job.epoch = next_epoch();
-    job.status_words = reinterpret_cast<int32_t *>(db + layout->status);
-    if ((rc = run_job(job, ws, ws_bytes, cuda_stream)) != SPD_OK) return rc;
-    uint8_t *hs = static_cast<uint8_t *>(host_blob) + layout->status;
-    if (cudaMemcpyAsync(hs, db + layout->status, layout->total_bytes - layout->status, cudaMemcpyDeviceToHost, st) != cudaSuccess)
-        return SPD_ERR_CUDA;
-    if (cudaStreamSynchronize(st) != cudaSuccess) return SPD_ERR_CUDA;
+    const size_t row_in = static_cast<size_t>(shape->num_q_heads) * shape->head_dim * (shape->dtype == SPD_BF16 ? 2 : 4);
+    const size_t row_out = static_cast<size_t>(shape->num_q_heads) * shape->head_dim * (out_dtype == SPD_BF16 ? 2 : 4);
+    uint8_t *hs = hbw + layout->status;
     int32_t *hdr = reinterpret_cast<int32_t *>(hs);
-    const int32_t code = hdr[HDR_STATUS], enc = hdr[HDR_BAD_ENC];
+    int32_t code = 0, bad_user = -1;
+
+    // A large batch is served in parts so that the copies hide behind the kernels: while one part's kernel runs, the
+    // next parts' q go up on a copy stream of the library's own and the previous part's output comes down.  The
+    // tables of all parts travel with the first one.  Each part raises its status in words of its own of the blob's
+    // status block.  Parts hold at least a megabyte of q or of output; smaller batches go as one.
+    const size_t per_mb = ((row_in > row_out ? row_in : row_out) * B) >> 20;
+    const int want_parts = per_mb >= 2 ? kHostStepParts : 1;
+    const int parts = static_cast<size_t>(want_parts) <= B ? want_parts : 1;
+    HostStepStreams hss;
+    if (parts == 1 || host_step_streams(&hss) != SPD_OK) {
+        if (cudaMemcpyAsync(db, hb, layout->in_bytes, cudaMemcpyHostToDevice, st) != cudaSuccess) return SPD_ERR_CUDA;
+        // The step raises its status in the blob (uploaded as zeros a moment ago), right in front of the
+        // output, so that one copy brings both back.
+        Job job{};
+        job.shape = shape; job.q = db + layout->q; job.part[0] = &a; job.part[1] = &b;
+        job.mode = OUT_FINAL; job.pin = nullptr; job.out = db + layout->out; job.out_dtype = out_dtype;
+        job.epoch = next_epoch();
+        job.status_words = reinterpret_cast<int32_t *>(db + layout->status);
+        if ((rc = run_job(job, ws, ws_bytes, cuda_stream)) != SPD_OK) return rc;
+        if (cudaMemcpyAsync(hs, db + layout->status, layout->total_bytes - layout->status, cudaMemcpyDeviceToHost, st) != cudaSuccess)
+            return SPD_ERR_CUDA;
+        if (cudaStreamSynchronize(st) != cudaSuccess) return SPD_ERR_CUDA;
+        code = hdr[HDR_STATUS];
+        if (hdr[HDR_BAD_ENC]) bad_user = 0x7fffffff - hdr[HDR_BAD_ENC];
+    } else {
+        size_t first[kHostStepParts + 1];              // part i serves users [first[i], first[i + 1])
+        for (int i = 0; i <= parts; ++i) first[i] = B * i / parts;
+        const size_t q_all = B * row_in;
+        // the first part's q, then everything behind q (tables of all parts, the zeroed status block), on the caller's stream
+        if (cudaMemcpyAsync(db + layout->q, hb + layout->q, first[1] * row_in, cudaMemcpyHostToDevice, st) != cudaSuccess ||
+            cudaMemcpyAsync(db + layout->q + q_all, hb + layout->q + q_all, layout->in_bytes - (layout->q + q_all), cudaMemcpyHostToDevice, st) != cudaSuccess)
+            return SPD_ERR_CUDA;
+        // the other parts' q on the copy stream, in order
+        for (int i = 1; i < parts; ++i)
+            if (cudaMemcpyAsync(db + layout->q + first[i] * row_in, hb + layout->q + first[i] * row_in, (first[i + 1] - first[i]) * row_in,
+                                cudaMemcpyHostToDevice, hss.copy) != cudaSuccess ||
+                cudaEventRecord(hss.q_up[i], hss.copy) != cudaSuccess)
+                return SPD_ERR_CUDA;
+        int32_t *status = reinterpret_cast<int32_t *>(db + layout->status);
+        for (int i = 0; i < parts; ++i) {
+            spd_shape si = *shape;
+            si.batch = static_cast<int32_t>(first[i + 1] - first[i]);
+            spd_paged_kv ai = a, bi = b;                // this part's users: the same tables, entered further in
+            ai.page_indptr += first[i]; ai.seq_lens += first[i];
+            bi.page_indptr += first[i]; bi.seq_lens += first[i];
+            Job job{};
+            job.shape = &si; job.q = db + layout->q + first[i] * row_in; job.part[0] = &ai; job.part[1] = &bi;
+            job.mode = OUT_FINAL; job.out = db + layout->out + first[i] * row_out; job.out_dtype = out_dtype;
+            job.epoch = next_epoch();
+            job.status_words = status + 8 * i;
+            job.layout_shape = shape;                   // every part lays the workspace out as the whole batch does
+            if (i > 0 && cudaStreamWaitEvent(st, hss.q_up[i], 0) != cudaSuccess) return SPD_ERR_CUDA;
+            if ((rc = run_job(job, ws, ws_bytes, cuda_stream)) != SPD_OK) return rc;
+            if (i + 1 < parts) {                        // this part's output comes down under the next part's kernel
+                if (cudaEventRecord(hss.done[i], st) != cudaSuccess || cudaStreamWaitEvent(hss.copy, hss.done[i], 0) != cudaSuccess ||
+                    cudaMemcpyAsync(hbw + layout->out + first[i] * row_out, db + layout->out + first[i] * row_out,
+                                    (first[i + 1] - first[i]) * row_out, cudaMemcpyDeviceToHost, hss.copy) != cudaSuccess)
+                    return SPD_ERR_CUDA;
+            }
+        }
+        const size_t last = first[parts - 1];
+        if (cudaMemcpyAsync(hs, db + layout->status, HDR_WORDS * 4, cudaMemcpyDeviceToHost, st) != cudaSuccess ||
+            cudaMemcpyAsync(hbw + layout->out + last * row_out, db + layout->out + last * row_out, (B - last) * row_out, cudaMemcpyDeviceToHost, st) != cudaSuccess)
+            return SPD_ERR_CUDA;
+        if (cudaStreamSynchronize(st) != cudaSuccess || cudaStreamSynchronize(hss.copy) != cudaSuccess) return SPD_ERR_CUDA;
+        for (int i = parts - 1; i >= 0; --i) {         // the lowest part that reports anything names the lowest user
+            const int32_t c = hdr[8 * i + HDR_STATUS], enc = hdr[8 * i + HDR_BAD_ENC];
+            if (c == SPD_ERR_TIMEOUT || (c != 0 && code != SPD_ERR_TIMEOUT)) code = c;
+            if (enc) bad_user = static_cast<int32_t>(first[i]) + (0x7fffffff - enc);
+        }
+    }
     memset(hs, 0, HDR_WORDS * 4);              // ready for the next upload
-    if (first_bad_user) *first_bad_user = enc ? 0x7fffffff - enc : -1;
+    if (first_bad_user) *first_bad_user = bad_user;
     if (code == SPD_ERR_TIMEOUT) {             // a kernel that gave up may have left merge tickets drawn
         DeviceInfo di;
         if (device_info(&di) != SPD_OK) return SPD_ERR_CUDA;

@@ -164,6 +164,54 @@ def test_host_blob_step_matches_oracle(name):
         spd.spd_decode_step_host(shape, lay, host, devb, pools[0], pools[1], torch.float32, ws)
 
 
+@pytest.mark.parametrize("batch,out_dtype", [(161, torch.float32), (300, torch.bfloat16), (601, torch.float32)])
+def test_host_blob_step_in_parts(batch, out_dtype):
+    """A batch whose q and output are megabytes is served in two parts inside the call (the second part's q goes up
+    and the first part's output comes down on a copy stream, under the other part's kernel).  Every row against
+    the oracle, three steps in a row on the same buffers, odd batches (unequal parts), and a page index outside the
+    pool planted in the last part: reported with the user's index in the whole batch."""
+    cfg = dict(name="halves", batch=batch, hq=32, hkv=8, d=128, dtype="bf16", lin=("uniform", 1, 400), lout=("uniform", 0, 60), seed=71)
+    w = wl.make_workload(cfg)
+    q, kin, kout = oracle_inputs(w)
+    ref = orc.full(q, kin, kout, w.sm_scale)
+    shape = spd.make_shape(w.batch, w.num_q_heads, w.num_kv_heads, w.head_dim, w.dtype, w.sm_scale)
+    ws = spd.alloc_workspace(shape)
+    lay = spd.spd_step_blob_layout(shape, int(w.priv.page_indices.numel()), int(w.pub.page_indices.numel()), out_dtype)
+    host = torch.zeros(lay.total_bytes, dtype=torch.uint8).pin_memory()
+    spd.fill_step_blob(lay, host, w.q, w.priv, w.pub)
+    devb = torch.empty(lay.total_bytes, dtype=torch.uint8, device="cuda")
+    pools = [(p.k_pool.cuda(), p.v_pool.cuda()) for p in (w.priv, w.pub)]
+    n = w.batch * w.num_q_heads * w.head_dim
+    es = 4 if out_dtype == torch.float32 else 2
+    tol = 2e-3 if out_dtype == torch.float32 else 2e-3 + 2.0 ** -8 * float(np.max(np.abs(ref)))
+
+    def result():
+        return host[lay.out:lay.out + es * n].view(out_dtype).reshape(w.batch, w.num_q_heads, w.head_dim).float().numpy()
+    for _ in range(3):
+        host[lay.out:] = 0xFF
+        assert spd.spd_decode_step_host(shape, lay, host, devb, pools[0], pools[1], out_dtype, ws) == (spd.SPD_OK, -1)
+        got = result()
+        assert np.all(np.isfinite(got)) and np.max(np.abs(got - ref)) <= tol
+    victim = batch - 7                                   # in the last part
+    idx = host[lay.priv_indices:lay.priv_indices + 4 * w.priv.page_indices.numel()].view(torch.int32)
+    at = int(w.priv.page_indptr[victim])
+    keep = int(idx[at])
+    idx[at] = w.priv.num_pages + 11
+    assert spd.spd_decode_step_host(shape, lay, host, devb, pools[0], pools[1], out_dtype, ws) == (4, victim)
+    got = result()
+    others = [u for u in range(batch) if u != victim]
+    assert np.all(got[victim] == 0) and np.max(np.abs(got[others] - ref[others])) <= tol
+    idx[at] = keep
+    assert spd.spd_decode_step_host(shape, lay, host, devb, pools[0], pools[1], out_dtype, ws) == (spd.SPD_OK, -1)
+    assert np.max(np.abs(result() - ref)) <= tol
+    # the plain entry point on the same workspace afterwards: the halves left it clean
+    out = torch.full((w.batch, w.num_q_heads, w.head_dim), float("nan"), dtype=torch.float32, device="cuda")
+    wg = w.to("cuda")
+    spd.spd_decode_step(shape, wg.q, wg.priv, wg.pub, out, ws, fused=True)
+    assert spd.spd_query_device_status(ws) == (spd.SPD_OK, -1)
+    assert_close(out.cpu().numpy(), ref, w.dtype, "plain step after steps in parts")
+
+
 @pytest.mark.parametrize("dtype", ["bf16", "f32"])
 def test_append_kv_is_bit_exact_and_feeds_the_next_step(dtype):
     """Step 3a: the new token's K/V rows go into the public cache, then attention sees them."""
