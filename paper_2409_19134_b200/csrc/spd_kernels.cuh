@@ -651,7 +651,7 @@ struct MathF32 {
         float s[GE];
 #pragma unroll
         for (int hh = 0; hh < GE; ++hh) s[hh] = 0.f;
-#pragma unroll
+#pragma unroll(NCH > 8 ? 4 : NCH)      // head_dim 128: fully unrolled, sixteen steps times eight heads overflow the register file
         for (int j = 0; j < NCH; ++j) {
             const int c = (j + t) & (NCH - 1);
             const float4 k4 = *reinterpret_cast<const float4 *>(krow + 4 * c);
